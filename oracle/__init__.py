@@ -1,0 +1,6 @@
+"""CPU oracle for block-quantised low-bit linear layers.
+
+TEST INFRASTRUCTURE ONLY.  Nothing in the product path may import this
+package: only the tests, the smoke check and the benchmark's CPU-baseline /
+reference arm call it.  It shares no code with the CUDA path.
+"""
