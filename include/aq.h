@@ -1,0 +1,195 @@
+/*
+ * libaq -- low-bit block-quantised linear layers for NVIDIA B200 (sm_100a).
+ *
+ * C ABI.  Every pointer argument says whether it is HOST or DEVICE memory.
+ * Citations name passages of "ActQuant: Sub-4-bit Action-Guided Quantization
+ * for Vision-Language-Action Models" (the paper).
+ *
+ * The format (Section 3, "Weight quantization", Eq. 1): a weight matrix W of
+ * N rows (output features) by K columns (input features) is cut, along each
+ * row, into blocks of 32 consecutive elements; a block has a scale and a zero
+ * point and all its elements are coded with the same number of bits n; one
+ * matrix has one n (Section 1: "a single bit-width per matrix").  Eq. 1's
+ * decode s_b (q_i - z_b) is stored as  scale * q_i + min  (min = -s_b z_b),
+ * scale and min in IEEE binary16, q_i in {0 .. 2^n - 1}, n in {2, 3, 4}.
+ *
+ * Canonical bytes (the container of Appendix D: packed codes, per-block
+ * scales and zero points; byte order is this library's choice): blocks in
+ * row-major order over (row, block); a block record is
+ *     [scale: binary16 LE][min: binary16 LE][codes: 4n bytes]
+ * where the codes form one little-endian integer of 32 n bits with code i at
+ * bits [n i, n i + n).  N*K*(n+1)/8 bytes in total.
+ *
+ * Errors: every call returns an aq_status_t; nothing throws, aborts or traps
+ * the device.  Arguments are checked on the host before any launch.
+ * All launches are asynchronous on the given stream unless stated otherwise.
+ * The library runs only on compute capability 10.x devices (AQ_ERR_ARCH).
+ */
+#ifndef AQ_H_
+#define AQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct aq_handle_s* aq_handle_t;   /* opaque; owns its device memory */
+typedef void* aq_stream_t;                 /* a cudaStream_t (0 = default stream) */
+
+typedef enum {
+    AQ_OK = 0,
+    AQ_ERR_INVALID_ARG = 1,   /* null / misaligned pointer, bad size, bad enum */
+    AQ_ERR_UNSUPPORTED = 2,   /* bits not in {2,3,4}, block != 32, dtype not allowed here */
+    AQ_ERR_ALLOC = 3,         /* device or host allocation failed */
+    AQ_ERR_CUDA = 4,          /* a CUDA runtime call failed (see aq_last_cuda_error) */
+    AQ_ERR_TIMEOUT = 5,       /* a bounded device-side wait ran out */
+    AQ_ERR_ARCH = 6,          /* current device is not sm_100 */
+    AQ_ERR_RANGE = 7          /* non-finite weight, or a block's scale/min overflows binary16 */
+} aq_status_t;
+
+typedef enum { AQ_F16 = 0, AQ_BF16 = 1, AQ_F32 = 2 } aq_dtype_t;
+
+/* Largest token count M of one aq_linear / aq_stack_forward call. */
+#define AQ_MAX_M 4096
+/* Token counts up to this run the weight-streaming (decode) kernel. */
+#define AQ_DECODE_MAX_M 8
+
+/*
+ * aq_pack -- quantise and pack (Eq. 1, the argmin over a uniform codebook:
+ * round-to-nearest; the "RTN block quantization" row of the ablation table).
+ *   bits   : n in {2,3,4};  block : must be 32
+ *   W_dev  : DEVICE, float32, row-major [N][K], 16-byte aligned; read during
+ *            the call's stream work, not retained
+ *   N, K   : N >= 1; K >= 32 and K % 32 == 0
+ *   out    : HOST pointer receiving the new handle
+ * Per block, in binary32 with one rounding per operation:
+ *   scale = f16((max - min) / (2^n - 1)), min = f16(min),
+ *   q = clamp(rint((w - min) / scale), 0, 2^n - 1)   (rint: ties to even),
+ *   q = 0 everywhere when scale rounds to 0.
+ * A non-finite weight or an overflowing scale/min is recorded in the handle
+ * and reported as AQ_ERR_RANGE by aq_info / aq_export.
+ */
+aq_status_t aq_pack(int bits, int block, const float* W_dev, int64_t N, int64_t K,
+                    aq_stream_t stream, aq_handle_t* out);
+
+/*
+ * aq_import -- build a handle from canonical bytes (Appendix D container).
+ *   canon_host : HOST, nbytes == N*K*(bits+1)/8 bytes in the layout above
+ * Synchronises `stream` before returning (the host buffer may be reused).
+ */
+aq_status_t aq_import(int bits, int block, int64_t N, int64_t K, const void* canon_host,
+                      size_t nbytes, aq_stream_t stream, aq_handle_t* out);
+
+/*
+ * aq_export -- canonical bytes of a handle (Appendix D container).
+ *   canon_host : HOST buffer of capacity cap (may be NULL to query the size)
+ *   nbytes     : HOST, receives N*K*(bits+1)/8
+ * Synchronises the handle's last stream.  AQ_ERR_RANGE if packing saw a
+ * non-finite weight or an overflow (the bytes are still written).
+ */
+aq_status_t aq_export(aq_handle_t h, void* canon_host, size_t cap, size_t* nbytes);
+
+/*
+ * aq_info -- shape and sizes; any out pointer may be NULL.
+ *   packed_bytes : N*K*(bits+1)/8, the closed form
+ *   device_bytes : bytes the handle holds on the device for the weights
+ *                  (the closed form plus padding of N to 16 and K to 256)
+ * Synchronises the handle's last stream; AQ_ERR_RANGE as for aq_export.
+ */
+aq_status_t aq_info(aq_handle_t h, int* bits, int* block, int64_t* N, int64_t* K,
+                    size_t* packed_bytes, size_t* device_bytes);
+
+/*
+ * aq_dequant -- the whole dequantised matrix (Eq. 1).
+ *   out_dev : DEVICE, row-major [N][K] of out_dtype, 16-byte aligned
+ * Each element is fmaf(f32(scale), f32(q), f32(min)) rounded once to
+ * out_dtype (nearest even); bit-exact with that definition.
+ */
+aq_status_t aq_dequant(aq_handle_t h, void* out_dev, aq_dtype_t out_dtype, aq_stream_t stream);
+
+/*
+ * aq_linear -- y = x W_hat^T on the packed weights (Section 4.3 / Appendix D:
+ * each matmul of the converted model runs as one low-bit kernel that
+ * dequantises on the fly; activations stay in half precision).
+ *   x_dev : DEVICE, row-major [M][K], AQ_F16 or AQ_BF16, 16-byte aligned
+ *   y_dev : DEVICE, row-major [M][N], same dtype (AQ_F32 output is accepted
+ *           with xy_dtype's input type via aq_linear_f32out)
+ *   M     : 1 .. AQ_MAX_M.  M <= AQ_DECODE_MAX_M runs the weight-streaming
+ *           kernel, larger M the tensor-core GEMM.
+ * Accumulation is binary32.  Calls on one handle must be ordered on a stream
+ * (the handle owns accumulation scratch that concurrent calls would share).
+ */
+aq_status_t aq_linear(aq_handle_t h, const void* x_dev, void* y_dev, int M,
+                      aq_dtype_t xy_dtype, aq_stream_t stream);
+
+/* As aq_linear but y_dev is float32 [M][N] holding the unrounded accumulators. */
+aq_status_t aq_linear_f32out(aq_handle_t h, const void* x_dev, float* y_dev, int M,
+                             aq_dtype_t x_dtype, aq_stream_t stream);
+
+/*
+ * A program over a list of handles: the linears of a stack of transformer
+ * blocks (Section 3: each block holds W_Q, W_K, W_V, W_O, W_gate, W_up,
+ * W_down) with the glue between them.  Activations live in float32 buffers
+ * [M][width] inside the caller's workspace; the vector a linear consumes is
+ * formed from them and rounded to the activation dtype:
+ *   AQ_IN_PLAIN    : x = src
+ *   AQ_IN_RMSNORM  : x = src / sqrt(mean_k(src^2) + 1e-6)      (no gain)
+ *   AQ_IN_SILU_MUL : x = silu(src) * src2,  silu(g) = g / (1 + exp(-g))
+ * and the result is dst = W x (AQ_OUT_STORE) or dst = res + W x (AQ_OUT_ADD).
+ * Buffer 0 is the program input.  Handles are borrowed, not owned.
+ */
+typedef enum { AQ_IN_PLAIN = 0, AQ_IN_RMSNORM = 1, AQ_IN_SILU_MUL = 2 } aq_in_op_t;
+typedef enum { AQ_OUT_STORE = 0, AQ_OUT_ADD = 1 } aq_out_op_t;
+
+typedef struct {
+    aq_handle_t w;      /* the packed matrix, N = width[dst], K = width[src] */
+    int32_t src;        /* input buffer index */
+    int32_t src2;       /* second input for AQ_IN_SILU_MUL, else ignored */
+    int32_t dst;        /* output buffer index (> 0; written by this op only) */
+    int32_t res;        /* residual buffer for AQ_OUT_ADD, else ignored */
+    int32_t in_op;      /* aq_in_op_t */
+    int32_t out_op;     /* aq_out_op_t */
+} aq_stack_op_t;
+
+typedef struct {
+    int32_t n_ops;
+    int32_t n_bufs;
+    const aq_stack_op_t* ops;     /* HOST, n_ops entries, in execution order */
+    const int64_t* buf_width;     /* HOST, n_bufs entries */
+} aq_stack_t;
+
+/* Bytes of workspace aq_stack_forward needs for M tokens (0 on a bad program). */
+size_t aq_stack_workspace_bytes(const aq_stack_t* prog, int M);
+
+/*
+ * aq_stack_forward -- run the program (Section 4.3: the deployed forward pass
+ * dispatches every quantised matmul to a low-bit kernel).
+ *   x0_dev        : DEVICE [M][width[0]] of `dtype` (AQ_F16 / AQ_BF16)
+ *   out_dev       : DEVICE [M][width[out_buf]] of `dtype`, the rounded contents
+ *                   of buffer out_buf after the last op (may be NULL)
+ *   workspace_dev : DEVICE, 256-byte aligned, >= aq_stack_workspace_bytes();
+ *                   afterwards buffer b is float32 [M][width[b]] at byte
+ *                   offset aq_stack_buffer_offset(prog, M, b): every op's
+ *                   input and output stay readable for per-op checks
+ */
+aq_status_t aq_stack_forward(const aq_stack_t* prog, const void* x0_dev, void* out_dev, int out_buf,
+                             int M, aq_dtype_t dtype, void* workspace_dev, size_t ws_bytes,
+                             aq_stream_t stream);
+
+/* Byte offset of buffer b inside the workspace ((size_t)-1 on a bad argument). */
+size_t aq_stack_buffer_offset(const aq_stack_t* prog, int M, int b);
+
+/* Releases the handle and its device memory (synchronises its last stream). */
+void aq_free(aq_handle_t h);
+
+const char* aq_status_string(aq_status_t s);
+
+/* Text of the last CUDA error this thread's libaq call saw ("" if none). */
+const char* aq_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AQ_H_ */

@@ -1,0 +1,242 @@
+"""ctypes binding over libaq.so: same names as the C ABI, argument marshalling only.
+
+Every step of the path runs in the library's CUDA kernels; torch is used by
+callers for device memory and streams.  Importing this module loads the
+library and raises if it is missing (there is no fallback path).
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libaq.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} not found: build it with `python -m paper_2605_24011_b200.build` "
+        "(libaq has no CPU or PyTorch fallback)")
+
+_lib = C.CDLL(LIB_PATH)
+
+AQ_OK, AQ_ERR_INVALID_ARG, AQ_ERR_UNSUPPORTED, AQ_ERR_ALLOC, AQ_ERR_CUDA, AQ_ERR_TIMEOUT, AQ_ERR_ARCH, AQ_ERR_RANGE = range(8)
+AQ_F16, AQ_BF16, AQ_F32 = 0, 1, 2
+AQ_IN_PLAIN, AQ_IN_RMSNORM, AQ_IN_SILU_MUL = 0, 1, 2
+AQ_OUT_STORE, AQ_OUT_ADD = 0, 1
+AQ_MAX_M, AQ_DECODE_MAX_M = 4096, 8
+
+SYMBOLS = ("aq_pack", "aq_import", "aq_export", "aq_info", "aq_dequant", "aq_linear", "aq_linear_f32out",
+           "aq_stack_workspace_bytes", "aq_stack_forward", "aq_stack_buffer_offset", "aq_free",
+           "aq_status_string", "aq_last_cuda_error")
+
+_H = C.c_void_p
+
+
+class StackOp(C.Structure):
+    _fields_ = [("w", _H), ("src", C.c_int32), ("src2", C.c_int32), ("dst", C.c_int32), ("res", C.c_int32),
+                ("in_op", C.c_int32), ("out_op", C.c_int32)]
+
+
+class Stack(C.Structure):
+    _fields_ = [("n_ops", C.c_int32), ("n_bufs", C.c_int32), ("ops", C.POINTER(StackOp)),
+                ("buf_width", C.POINTER(C.c_int64))]
+
+
+_lib.aq_pack.argtypes = [C.c_int, C.c_int, C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.POINTER(_H)]
+_lib.aq_import.argtypes = [C.c_int, C.c_int, C.c_int64, C.c_int64, C.c_void_p, C.c_size_t, C.c_void_p, C.POINTER(_H)]
+_lib.aq_export.argtypes = [_H, C.c_void_p, C.c_size_t, C.POINTER(C.c_size_t)]
+_lib.aq_info.argtypes = [_H, C.POINTER(C.c_int), C.POINTER(C.c_int), C.POINTER(C.c_int64), C.POINTER(C.c_int64),
+                         C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
+_lib.aq_dequant.argtypes = [_H, C.c_void_p, C.c_int, C.c_void_p]
+_lib.aq_linear.argtypes = [_H, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p]
+_lib.aq_linear_f32out.argtypes = [_H, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p]
+_lib.aq_stack_workspace_bytes.argtypes = [C.POINTER(Stack), C.c_int]
+_lib.aq_stack_workspace_bytes.restype = C.c_size_t
+_lib.aq_stack_buffer_offset.argtypes = [C.POINTER(Stack), C.c_int, C.c_int]
+_lib.aq_stack_buffer_offset.restype = C.c_size_t
+_lib.aq_stack_forward.argtypes = [C.POINTER(Stack), C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p,
+                                  C.c_size_t, C.c_void_p]
+_lib.aq_free.argtypes = [_H]
+_lib.aq_free.restype = None
+_lib.aq_status_string.argtypes = [C.c_int]
+_lib.aq_status_string.restype = C.c_char_p
+_lib.aq_last_cuda_error.argtypes = []
+_lib.aq_last_cuda_error.restype = C.c_char_p
+for _n in ("aq_pack", "aq_import", "aq_export", "aq_info", "aq_dequant", "aq_linear", "aq_linear_f32out",
+           "aq_stack_forward"):
+    getattr(_lib, _n).restype = C.c_int
+
+
+class AqError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = f"{where}: {status_string(status)}"
+        if status == AQ_ERR_CUDA:
+            msg += f" ({_lib.aq_last_cuda_error().decode()})"
+        super().__init__(msg)
+
+
+def status_string(status: int) -> str:
+    return _lib.aq_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str):
+    if status != AQ_OK:
+        raise AqError(status, where)
+
+
+def _ptr(t) -> int:
+    """Address of a torch tensor's storage (0 for None)."""
+    return 0 if t is None else int(t.data_ptr())
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        import torch
+        return int(torch.cuda.current_stream().cuda_stream)
+    return int(getattr(stream, "cuda_stream", stream))
+
+
+_DT = {"f16": AQ_F16, "bf16": AQ_BF16, "f32": AQ_F32}
+
+
+def dtype_code(t) -> int:
+    """aq_dtype_t of a torch tensor / dtype / short name."""
+    if isinstance(t, str):
+        return _DT[t]
+    import torch
+    dt = t.dtype if hasattr(t, "data_ptr") else t
+    return {torch.float16: AQ_F16, torch.bfloat16: AQ_BF16, torch.float32: AQ_F32}[dt]
+
+
+class Handle:
+    """Owns one aq_handle_t."""
+
+    def __init__(self, raw: int):
+        self._h = raw
+
+    @property
+    def raw(self):
+        return self._h
+
+    def free(self):
+        if self._h:
+            _lib.aq_free(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.free()
+        except Exception:
+            pass
+
+
+def aq_pack(bits: int, block: int, W, stream=None) -> Handle:
+    """W: CUDA float32 tensor [N][K] (contiguous)."""
+    N, K = W.shape
+    h = _H()
+    _check(_lib.aq_pack(bits, block, _ptr(W), N, K, _stream(stream), C.byref(h)), "aq_pack")
+    return Handle(h.value)
+
+
+def aq_pack_raw(bits, block, w_ptr, N, K, stream_ptr=0):
+    """Direct call with raw addresses; returns (status, handle value or None)."""
+    h = _H()
+    st = _lib.aq_pack(bits, block, w_ptr, N, K, stream_ptr, C.byref(h))
+    return st, h.value
+
+
+def aq_import(bits: int, block: int, N: int, K: int, canon, stream=None) -> Handle:
+    """canon: host bytes / numpy uint8 array holding the canonical stream."""
+    import numpy as np
+    buf = np.ascontiguousarray(np.frombuffer(canon, dtype=np.uint8) if isinstance(canon, (bytes, bytearray)) else canon,
+                               dtype=np.uint8)
+    h = _H()
+    _check(_lib.aq_import(bits, block, N, K, buf.ctypes.data, buf.size, _stream(stream), C.byref(h)), "aq_import")
+    return Handle(h.value)
+
+
+def aq_export(h: Handle, allow_range_error: bool = False):
+    """Canonical bytes as a numpy uint8 array."""
+    import numpy as np
+    n = C.c_size_t()
+    _check(_lib.aq_export(h.raw, None, 0, C.byref(n)), "aq_export(size)")
+    out = np.empty(n.value, dtype=np.uint8)
+    st = _lib.aq_export(h.raw, out.ctypes.data, out.size, C.byref(n))
+    if not (allow_range_error and st == AQ_ERR_RANGE):
+        _check(st, "aq_export")
+    return out
+
+
+def aq_info(h: Handle):
+    bits, block = C.c_int(), C.c_int()
+    N, K = C.c_int64(), C.c_int64()
+    pb, db = C.c_size_t(), C.c_size_t()
+    st = _lib.aq_info(h.raw, C.byref(bits), C.byref(block), C.byref(N), C.byref(K), C.byref(pb), C.byref(db))
+    return {"status": st, "bits": bits.value, "block": block.value, "N": N.value, "K": K.value,
+            "packed_bytes": pb.value, "device_bytes": db.value}
+
+
+def aq_dequant(h: Handle, out, stream=None):
+    """out: CUDA tensor [N][K] of float16 / bfloat16 / float32."""
+    _check(_lib.aq_dequant(h.raw, _ptr(out), dtype_code(out), _stream(stream)), "aq_dequant")
+    return out
+
+
+def aq_linear(h: Handle, x, y, M: int | None = None, stream=None):
+    """x: CUDA [M][K] float16/bfloat16; y: CUDA [M][N] of the same dtype, or float32."""
+    M = int(x.shape[0]) if M is None else M
+    if dtype_code(y) == AQ_F32:
+        _check(_lib.aq_linear_f32out(h.raw, _ptr(x), _ptr(y), M, dtype_code(x), _stream(stream)), "aq_linear_f32out")
+    else:
+        if dtype_code(y) != dtype_code(x):
+            raise AqError(AQ_ERR_INVALID_ARG, "aq_linear: y dtype must equal x dtype (or float32)")
+        _check(_lib.aq_linear(h.raw, _ptr(x), _ptr(y), M, dtype_code(x), _stream(stream)), "aq_linear")
+    return y
+
+
+class Program:
+    """Host-side aq_stack_t builder.  ops: dicts with keys w (Handle), src, dst
+    and optionally src2, res, in_op, out_op."""
+
+    def __init__(self, buf_width, ops):
+        self.handles = [o["w"] for o in ops]           # keep alive
+        self._ops = (StackOp * len(ops))()
+        for i, o in enumerate(ops):
+            self._ops[i] = StackOp(o["w"].raw, o["src"], o.get("src2", -1), o["dst"], o.get("res", -1),
+                                   o.get("in_op", AQ_IN_PLAIN), o.get("out_op", AQ_OUT_STORE))
+        self._w = (C.c_int64 * len(buf_width))(*buf_width)
+        self.c = Stack(len(ops), len(buf_width), self._ops, self._w)
+        self.buf_width = list(buf_width)
+        self.ops = ops
+
+    def workspace_bytes(self, M: int) -> int:
+        return int(_lib.aq_stack_workspace_bytes(C.byref(self.c), M))
+
+    def buffer_offset(self, M: int, b: int) -> int:
+        return int(_lib.aq_stack_buffer_offset(C.byref(self.c), M, b))
+
+
+def aq_stack_workspace_bytes(prog: Program, M: int) -> int:
+    return prog.workspace_bytes(M)
+
+
+def aq_stack_forward(prog: Program, x0, out, out_buf: int, M: int, workspace, stream=None):
+    """x0: CUDA [M][width0] f16/bf16; out: CUDA [M][width[out_buf]] same dtype or None;
+    workspace: CUDA uint8 tensor of at least workspace_bytes(M)."""
+    _check(_lib.aq_stack_forward(C.byref(prog.c), _ptr(x0), _ptr(out), out_buf, M, dtype_code(x0), _ptr(workspace),
+                                 workspace.numel() * workspace.element_size(), _stream(stream)), "aq_stack_forward")
+    return out
+
+
+def stack_buffer(prog: Program, workspace, M: int, b: int):
+    """float32 view [M][width[b]] of buffer b inside the workspace."""
+    import torch
+    off = prog.buffer_offset(M, b)
+    n = M * prog.buf_width[b]
+    return workspace[off:off + 4 * n].view(torch.float32).view(M, prog.buf_width[b])
+
+
+def raw_lib():
+    """The ctypes library object (tests of the ABI itself)."""
+    return _lib

@@ -1,0 +1,232 @@
+// C-ABI entry points of libaq: argument checks, handle ownership, dispatch.
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "aq_internal.h"
+#include "aq_layout.cuh"
+
+namespace aq {
+
+static thread_local char g_last_err[256] = "";
+
+aq_status_t cuda_fail(cudaError_t e) {
+    snprintf(g_last_err, sizeof(g_last_err), "%s: %s", cudaGetErrorName(e), cudaGetErrorString(e));
+    return AQ_ERR_CUDA;
+}
+
+bool handle_ok(aq_handle_t h) { return h != nullptr && h->magic == AQ_HANDLE_MAGIC; }
+
+int sm_count() {
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+    }
+    return n;
+}
+
+static aq_status_t check_arch(int* dev_out) {
+    int dev = 0, major = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (major != 10) return AQ_ERR_ARCH;
+    if (dev_out) *dev_out = dev;
+    return AQ_OK;
+}
+
+static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static aq_status_t new_handle(int bits, int block, int64_t N, int64_t K, aq_handle_t* out) {
+    if (!out) return AQ_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (block != 32 || bits < 2 || bits > 4) return AQ_ERR_UNSUPPORTED;
+    if (N < 1 || K < 32 || (K % 32) != 0 || N > (int64_t)1 << 24 || K > (int64_t)1 << 24) return AQ_ERR_INVALID_ARG;
+    int dev = 0;
+    aq_status_t st = check_arch(&dev);
+    if (st != AQ_OK) return st;
+    aq_handle_s* h = new (std::nothrow) aq_handle_s();
+    if (!h) return AQ_ERR_ALLOC;
+    h->magic = AQ_HANDLE_MAGIC;
+    h->bits = bits; h->device = dev; h->N = N; h->K = K;
+    h->NT = (int)((N + 15) / 16);
+    h->KP = (int)((K + 255) / 256);
+    h->n_frags = (int64_t)h->NT * h->KP * 2;
+    h->dev_bytes = (size_t)h->n_frags * frag_bytes(bits);
+    h->frags = nullptr; h->acc = nullptr; h->flags = nullptr; h->last_stream = nullptr;
+    const size_t acc_bytes = (size_t)AQ_DECODE_MAX_M * h->NT * 16 * sizeof(float);
+    if (cudaMalloc(&h->frags, h->dev_bytes) != cudaSuccess || cudaMalloc(&h->acc, acc_bytes) != cudaSuccess ||
+        cudaMalloc(&h->flags, 256) != cudaSuccess) {
+        cudaGetLastError();
+        cudaFree(h->frags); cudaFree(h->acc); cudaFree(h->flags);
+        delete h;
+        return AQ_ERR_ALLOC;
+    }
+    *out = h;
+    return AQ_OK;
+}
+
+static void destroy(aq_handle_s* h) {
+    cudaFree(h->frags); cudaFree(h->acc); cudaFree(h->flags);
+    h->magic = 0;
+    delete h;
+}
+
+}  // namespace aq
+
+using namespace aq;
+
+extern "C" {
+
+aq_status_t aq_pack(int bits, int block, const float* W_dev, int64_t N, int64_t K, aq_stream_t stream,
+                    aq_handle_t* out) {
+    if (!out) return AQ_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!W_dev || !aligned16(W_dev)) return AQ_ERR_INVALID_ARG;
+    aq_handle_t h = nullptr;
+    aq_status_t st = new_handle(bits, block, N, K, &h);
+    if (st != AQ_OK) return st;
+    cudaStream_t s = (cudaStream_t)stream;
+    cudaError_t e = cudaMemsetAsync(h->acc, 0, (size_t)AQ_DECODE_MAX_M * h->NT * 16 * sizeof(float), s);
+    if (e == cudaSuccess) e = cudaMemsetAsync(h->flags, 0, 256, s);
+    if (e == cudaSuccess) e = launch_pack(h, W_dev, s);
+    if (e != cudaSuccess) { destroy(h); return cuda_fail(e); }
+    h->last_stream = s;
+    *out = h;
+    return AQ_OK;
+}
+
+aq_status_t aq_import(int bits, int block, int64_t N, int64_t K, const void* canon_host, size_t nbytes,
+                      aq_stream_t stream, aq_handle_t* out) {
+    if (!out) return AQ_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!canon_host) return AQ_ERR_INVALID_ARG;
+    aq_handle_t h = nullptr;
+    aq_status_t st = new_handle(bits, block, N, K, &h);
+    if (st != AQ_OK) return st;
+    if (nbytes != (size_t)N * (size_t)(K / 32) * (size_t)(4 + 4 * bits)) { destroy(h); return AQ_ERR_INVALID_ARG; }
+    cudaStream_t s = (cudaStream_t)stream;
+    uint8_t* tmp = nullptr;
+    if (cudaMalloc(&tmp, nbytes) != cudaSuccess) { cudaGetLastError(); destroy(h); return AQ_ERR_ALLOC; }
+    cudaError_t e = cudaMemcpyAsync(tmp, canon_host, nbytes, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaMemsetAsync(h->acc, 0, (size_t)AQ_DECODE_MAX_M * h->NT * 16 * sizeof(float), s);
+    if (e == cudaSuccess) e = cudaMemsetAsync(h->flags, 0, 256, s);
+    if (e == cudaSuccess) e = launch_import(h, tmp, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    cudaFree(tmp);
+    if (e != cudaSuccess) { destroy(h); return cuda_fail(e); }
+    h->last_stream = s;
+    *out = h;
+    return AQ_OK;
+}
+
+static aq_status_t range_status(aq_handle_t h) {
+    int flag = 0;
+    cudaError_t e = cudaStreamSynchronize(h->last_stream);
+    if (e == cudaSuccess) e = cudaMemcpy(&flag, h->flags, sizeof(int), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(e);
+    return (flag & 1) ? AQ_ERR_RANGE : AQ_OK;
+}
+
+aq_status_t aq_export(aq_handle_t h, void* canon_host, size_t cap, size_t* nbytes) {
+    if (!handle_ok(h)) return AQ_ERR_INVALID_ARG;
+    const size_t need = (size_t)h->N * (size_t)(h->K / 32) * (size_t)(4 + 4 * h->bits);
+    if (nbytes) *nbytes = need;
+    if (!canon_host) return nbytes ? AQ_OK : AQ_ERR_INVALID_ARG;
+    if (cap < need) return AQ_ERR_INVALID_ARG;
+    uint8_t* tmp = nullptr;
+    if (cudaMalloc(&tmp, need) != cudaSuccess) { cudaGetLastError(); return AQ_ERR_ALLOC; }
+    cudaStream_t s = h->last_stream;
+    cudaError_t e = launch_export(h, tmp, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(canon_host, tmp, need, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    cudaFree(tmp);
+    if (e != cudaSuccess) return cuda_fail(e);
+    return range_status(h);
+}
+
+aq_status_t aq_info(aq_handle_t h, int* bits, int* block, int64_t* N, int64_t* K, size_t* packed_bytes,
+                    size_t* device_bytes) {
+    if (!handle_ok(h)) return AQ_ERR_INVALID_ARG;
+    if (bits) *bits = h->bits;
+    if (block) *block = 32;
+    if (N) *N = h->N;
+    if (K) *K = h->K;
+    if (packed_bytes) *packed_bytes = (size_t)h->N * (size_t)(h->K / 32) * (size_t)(4 + 4 * h->bits);
+    if (device_bytes) *device_bytes = h->dev_bytes;
+    return range_status(h);
+}
+
+aq_status_t aq_dequant(aq_handle_t h, void* out_dev, aq_dtype_t out_dtype, aq_stream_t stream) {
+    if (!handle_ok(h) || !out_dev || !aligned16(out_dev)) return AQ_ERR_INVALID_ARG;
+    if (out_dtype != AQ_F16 && out_dtype != AQ_BF16 && out_dtype != AQ_F32) return AQ_ERR_INVALID_ARG;
+    cudaStream_t s = (cudaStream_t)stream;
+    cudaError_t e = launch_dequant(h, out_dev, out_dtype, s);
+    if (e != cudaSuccess) return cuda_fail(e);
+    h->last_stream = s;
+    return AQ_OK;
+}
+
+static aq_status_t linear_common(aq_handle_t h, const void* x_dev, void* y_dev, int M, aq_dtype_t xdt,
+                                 aq_dtype_t ydt, aq_stream_t stream) {
+    if (!handle_ok(h) || !x_dev || !y_dev || !aligned16(x_dev) || !aligned16(y_dev)) return AQ_ERR_INVALID_ARG;
+    if (M < 1 || M > AQ_MAX_M) return AQ_ERR_INVALID_ARG;
+    if (xdt != AQ_F16 && xdt != AQ_BF16) return (xdt == AQ_F32) ? AQ_ERR_UNSUPPORTED : AQ_ERR_INVALID_ARG;
+    cudaStream_t s = (cudaStream_t)stream;
+    cudaError_t e;
+    if (M <= AQ_DECODE_MAX_M) {
+        const int64_t ld = (int64_t)h->NT * 16;
+        e = launch_gemv(h, x_dev, xdt, M, h->acc, ld, s);
+        if (e == cudaSuccess) e = launch_finalize(h->acc, h->acc, ld, y_dev, ydt, M, h->N, s);
+    } else if (ydt == AQ_F32) {
+        e = launch_gemm(h, x_dev, xdt, M, (float*)y_dev, h->N, false, s);
+    } else {
+        float* tmp = nullptr;
+        e = cudaMallocAsync(&tmp, (size_t)M * h->N * sizeof(float), s);
+        if (e != cudaSuccess) { cudaGetLastError(); return AQ_ERR_ALLOC; }
+        e = launch_gemm(h, x_dev, xdt, M, tmp, h->N, false, s);
+        if (e == cudaSuccess) e = launch_finalize(tmp, nullptr, h->N, y_dev, ydt, M, h->N, s);
+        cudaFreeAsync(tmp, s);
+    }
+    if (e != cudaSuccess) return cuda_fail(e);
+    h->last_stream = s;
+    return AQ_OK;
+}
+
+aq_status_t aq_linear(aq_handle_t h, const void* x_dev, void* y_dev, int M, aq_dtype_t xy_dtype,
+                      aq_stream_t stream) {
+    return linear_common(h, x_dev, y_dev, M, xy_dtype, xy_dtype, stream);
+}
+
+aq_status_t aq_linear_f32out(aq_handle_t h, const void* x_dev, float* y_dev, int M, aq_dtype_t x_dtype,
+                             aq_stream_t stream) {
+    return linear_common(h, x_dev, y_dev, M, x_dtype, AQ_F32, stream);
+}
+
+void aq_free(aq_handle_t h) {
+    if (!handle_ok(h)) return;
+    cudaStreamSynchronize(h->last_stream);
+    destroy(h);
+}
+
+const char* aq_status_string(aq_status_t s) {
+    switch (s) {
+        case AQ_OK: return "AQ_OK";
+        case AQ_ERR_INVALID_ARG: return "AQ_ERR_INVALID_ARG";
+        case AQ_ERR_UNSUPPORTED: return "AQ_ERR_UNSUPPORTED";
+        case AQ_ERR_ALLOC: return "AQ_ERR_ALLOC";
+        case AQ_ERR_CUDA: return "AQ_ERR_CUDA";
+        case AQ_ERR_TIMEOUT: return "AQ_ERR_TIMEOUT";
+        case AQ_ERR_ARCH: return "AQ_ERR_ARCH";
+        case AQ_ERR_RANGE: return "AQ_ERR_RANGE";
+    }
+    return "AQ_ERR_?";
+}
+
+const char* aq_last_cuda_error(void) { return g_last_err; }
+
+}  // extern "C"

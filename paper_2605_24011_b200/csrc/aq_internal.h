@@ -1,0 +1,49 @@
+// Host-side internals shared by the .cu files of libaq (not part of the ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include "../../include/aq.h"
+
+#define AQ_HANDLE_MAGIC 0x41514831u   /* "AQH1" */
+
+struct aq_handle_s {
+    uint32_t magic;
+    int bits;
+    int device;
+    int64_t N, K;
+    int NT;            // row tiles of 16
+    int KP;            // pair slabs of 256 k
+    int64_t n_frags;   // NT * KP * 2
+    size_t dev_bytes;  // n_frags * frag_bytes
+    uint8_t* frags;    // DEVICE: fragment layout
+    float* acc;        // DEVICE: [AQ_DECODE_MAX_M][NT*16] accumulation scratch, zero between calls
+    int* flags;        // DEVICE: bit 0 = range error seen while packing
+    cudaStream_t last_stream;
+};
+
+namespace aq {
+
+// status helpers (aq_api.cu)
+aq_status_t cuda_fail(cudaError_t e);
+bool handle_ok(aq_handle_t h);
+
+// launchers (each checks nothing: arguments are validated by the API layer)
+cudaError_t launch_pack(const aq_handle_s* h, const float* W, cudaStream_t s);
+cudaError_t launch_import(const aq_handle_s* h, const uint8_t* canon_dev, cudaStream_t s);
+cudaError_t launch_export(const aq_handle_s* h, uint8_t* canon_dev, cudaStream_t s);
+cudaError_t launch_dequant(const aq_handle_s* h, void* out, aq_dtype_t dt, cudaStream_t s);
+
+// decode path: accumulate x W^T into acc (fp32 [M][ldacc]); x is [M][K] of xdt
+cudaError_t launch_gemv(const aq_handle_s* h, const void* x, aq_dtype_t xdt, int M, float* acc,
+                        int64_t ldacc, cudaStream_t s);
+// y[m][n] = cast(acc[m][n]) for n < N, then acc = 0
+cudaError_t launch_finalize(const float* acc_in, float* acc_zero, int64_t ldacc, void* y, aq_dtype_t ydt,
+                            int M, int64_t N, cudaStream_t s);
+
+// prefill path: out[m][n] (+)= sum_k x[m][k] w[n][k]; out fp32 [M][ldo]
+cudaError_t launch_gemm(const aq_handle_s* h, const void* x, aq_dtype_t xdt, int M, float* out,
+                        int64_t ldo, bool accumulate, cudaStream_t s);
+
+int sm_count();
+
+}  // namespace aq

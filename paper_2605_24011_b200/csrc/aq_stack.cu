@@ -1,0 +1,191 @@
+// aq_stack_forward: a program of linears over packed weights with the glue
+// between them (Section 3: the matrices of a transformer block; Section 4.3:
+// every quantised matmul of the deployed graph runs as a low-bit kernel).
+//
+// Activations are float32 buffers in the caller's workspace.  Consecutive ops
+// that consume the same input vector form a phase; per phase the input is
+// formed once (RMS scaling / SiLU*up / plain) and rounded to the activation
+// dtype, then each op of the phase accumulates W x into its output buffer.
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+#include <vector>
+
+#include "aq_internal.h"
+
+namespace aq {
+
+static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct StackPlan {
+    std::vector<size_t> buf_off;
+    size_t stage_off = 0;   // [M][maxK] activation-dtype staging of a phase input
+    size_t total = 0;
+};
+
+static bool plan_stack(const aq_stack_t* p, int M, StackPlan& plan) {
+    if (!p || !p->ops || !p->buf_width || p->n_ops < 1 || p->n_bufs < 2 || M < 1 || M > AQ_MAX_M) return false;
+    plan.buf_off.resize(p->n_bufs);
+    size_t off = 0;
+    int64_t maxw = 0;
+    for (int b = 0; b < p->n_bufs; ++b) {
+        if (p->buf_width[b] < 1) return false;
+        plan.buf_off[b] = off;
+        off += align_up((size_t)M * p->buf_width[b] * sizeof(float), 256);
+        if (p->buf_width[b] > maxw) maxw = p->buf_width[b];
+    }
+    plan.stage_off = off;
+    off += align_up((size_t)M * maxw * 2, 256);
+    plan.total = off;
+    std::vector<char> written(p->n_bufs, 0);
+    written[0] = 1;
+    for (int i = 0; i < p->n_ops; ++i) {
+        const aq_stack_op_t& o = p->ops[i];
+        if (!handle_ok(o.w)) return false;
+        if (o.src < 0 || o.src >= p->n_bufs || o.dst < 1 || o.dst >= p->n_bufs) return false;
+        if (!written[o.src] || written[o.dst]) return false;
+        if (o.in_op < AQ_IN_PLAIN || o.in_op > AQ_IN_SILU_MUL || o.out_op < AQ_OUT_STORE || o.out_op > AQ_OUT_ADD) return false;
+        if (o.in_op == AQ_IN_SILU_MUL) {
+            if (o.src2 < 0 || o.src2 >= p->n_bufs || !written[o.src2] || p->buf_width[o.src2] != p->buf_width[o.src]) return false;
+        }
+        if (o.out_op == AQ_OUT_ADD) {
+            if (o.res < 0 || o.res >= p->n_bufs || !written[o.res] || p->buf_width[o.res] != p->buf_width[o.dst]) return false;
+        }
+        if (o.w->K != p->buf_width[o.src] || o.w->N != p->buf_width[o.dst]) return false;
+        written[o.dst] = 1;
+    }
+    return true;
+}
+
+// ---- glue kernels ----------------------------------------------------------
+template <typename T> __device__ __forceinline__ float to_f32(T v);
+template <> __device__ __forceinline__ float to_f32<__half>(__half v) { return __half2float(v); }
+template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f32(float v);
+template <> __device__ __forceinline__ __half from_f32<__half>(float v) { return __float2half_rn(v); }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+template <typename T>
+__global__ void widen_kernel(const T* __restrict__ x, float* __restrict__ out, int64_t n) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) out[i] = to_f32<T>(x[i]);
+}
+
+template <typename T>
+__global__ void narrow_kernel(const float* __restrict__ x, T* __restrict__ out, int64_t n) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) out[i] = from_f32<T>(x[i]);
+}
+
+// One CTA per token row: x[m][k] = round(transform(src[m][k])).
+template <typename T>
+__global__ void __launch_bounds__(256) stage_kernel(const float* __restrict__ src, const float* __restrict__ src2,
+                                                    int in_op, int64_t K, T* __restrict__ x) {
+    const int64_t m = blockIdx.x;
+    const float* s = src + m * K;
+    T* o = x + m * K;
+    float scale = 1.f;
+    if (in_op == AQ_IN_RMSNORM) {
+        __shared__ float red[8];
+        float ss = 0.f;
+        for (int64_t k = threadIdx.x; k < K; k += 256) ss = fmaf(s[k], s[k], ss);
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, d);
+        if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+        __syncthreads();
+        float tot = 0.f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) tot += red[i];
+        scale = rsqrtf(tot / (float)K + 1e-6f);
+    }
+    if (in_op == AQ_IN_SILU_MUL) {
+        const float* s2 = src2 + m * K;
+        for (int64_t k = threadIdx.x; k < K; k += 256) {
+            const float g = s[k];
+            o[k] = from_f32<T>(g / (1.f + expf(-g)) * s2[k]);
+        }
+    } else {
+        for (int64_t k = threadIdx.x; k < K; k += 256) o[k] = from_f32<T>(s[k] * scale);
+    }
+}
+
+template <typename T>
+static cudaError_t run_stack(const aq_stack_t* p, const StackPlan& plan, const T* x0, T* out, int out_buf, int M,
+                             aq_dtype_t dt, uint8_t* ws, cudaStream_t s) {
+    cudaError_t e = cudaMemsetAsync(ws, 0, plan.stage_off, s);
+    if (e != cudaSuccess) return e;
+    auto buf = [&](int b) { return reinterpret_cast<float*>(ws + plan.buf_off[b]); };
+    T* stage = reinterpret_cast<T*>(ws + plan.stage_off);
+    {
+        const int64_t n = (int64_t)M * p->buf_width[0];
+        widen_kernel<T><<<(unsigned)((n + 255) / 256), 256, 0, s>>>(x0, buf(0), n);
+    }
+    int i = 0;
+    while (i < p->n_ops) {
+        const aq_stack_op_t& f = p->ops[i];
+        const int64_t K = p->buf_width[f.src];
+        stage_kernel<T><<<M, 256, 0, s>>>(buf(f.src), f.in_op == AQ_IN_SILU_MUL ? buf(f.src2) : nullptr, f.in_op, K, stage);
+        int j = i;
+        while (j < p->n_ops && p->ops[j].src == f.src && p->ops[j].in_op == f.in_op &&
+               (f.in_op != AQ_IN_SILU_MUL || p->ops[j].src2 == f.src2)) {
+            const aq_stack_op_t& o = p->ops[j];
+            const int64_t N = p->buf_width[o.dst];
+            if (o.out_op == AQ_OUT_ADD) {
+                e = cudaMemcpyAsync(buf(o.dst), buf(o.res), (size_t)M * N * sizeof(float), cudaMemcpyDeviceToDevice, s);
+                if (e != cudaSuccess) return e;
+            }
+            if (M <= AQ_DECODE_MAX_M) e = launch_gemv(o.w, stage, dt, M, buf(o.dst), N, s);
+            else e = launch_gemm(o.w, stage, dt, M, buf(o.dst), N, true, s);
+            if (e != cudaSuccess) return e;
+            o.w->last_stream = s;
+            ++j;
+        }
+        i = j;
+    }
+    if (out) {
+        const int64_t n = (int64_t)M * p->buf_width[out_buf];
+        narrow_kernel<T><<<(unsigned)((n + 255) / 256), 256, 0, s>>>(buf(out_buf), out, n);
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace aq
+
+using namespace aq;
+
+extern "C" {
+
+size_t aq_stack_workspace_bytes(const aq_stack_t* prog, int M) {
+    StackPlan plan;
+    if (!plan_stack(prog, M, plan)) return 0;
+    return plan.total;
+}
+
+size_t aq_stack_buffer_offset(const aq_stack_t* prog, int M, int b) {
+    StackPlan plan;
+    if (!plan_stack(prog, M, plan) || b < 0 || b >= prog->n_bufs) return (size_t)-1;
+    return plan.buf_off[b];
+}
+
+aq_status_t aq_stack_forward(const aq_stack_t* prog, const void* x0_dev, void* out_dev, int out_buf, int M,
+                             aq_dtype_t dtype, void* workspace_dev, size_t ws_bytes, aq_stream_t stream) {
+    StackPlan plan;
+    if (!plan_stack(prog, M, plan)) return AQ_ERR_INVALID_ARG;
+    if (!x0_dev || !workspace_dev || (reinterpret_cast<uintptr_t>(workspace_dev) & 255u) ||
+        (reinterpret_cast<uintptr_t>(x0_dev) & 15u) || (reinterpret_cast<uintptr_t>(out_dev) & 15u))
+        return AQ_ERR_INVALID_ARG;
+    if (ws_bytes < plan.total) return AQ_ERR_INVALID_ARG;
+    if (out_dev && (out_buf < 0 || out_buf >= prog->n_bufs)) return AQ_ERR_INVALID_ARG;
+    if (dtype != AQ_F16 && dtype != AQ_BF16) return (dtype == AQ_F32) ? AQ_ERR_UNSUPPORTED : AQ_ERR_INVALID_ARG;
+    cudaStream_t s = (cudaStream_t)stream;
+    cudaError_t e;
+    if (dtype == AQ_F16)
+        e = run_stack<__half>(prog, plan, (const __half*)x0_dev, (__half*)out_dev, out_buf, M, dtype, (uint8_t*)workspace_dev, s);
+    else
+        e = run_stack<__nv_bfloat16>(prog, plan, (const __nv_bfloat16*)x0_dev, (__nv_bfloat16*)out_dev, out_buf, M, dtype,
+                                     (uint8_t*)workspace_dev, s);
+    if (e != cudaSuccess) return cuda_fail(e);
+    return AQ_OK;
+}
+
+}  // extern "C"
