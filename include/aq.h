@@ -181,6 +181,22 @@ aq_status_t aq_stack_forward(const aq_stack_t* prog, const void* x0_dev, void* o
 /* Byte offset of buffer b inside the workspace ((size_t)-1 on a bad argument). */
 size_t aq_stack_buffer_offset(const aq_stack_t* prog, int M, int b);
 
+/*
+ * Byte offset, inside the workspace, of the rounded input vector op `op`
+ * consumed: [M][K] of the activation dtype, kept after the call so that each
+ * linear can be checked against exactly what it read ((size_t)-1 on a bad
+ * argument).  Ops that share an input share the region.
+ */
+size_t aq_stack_input_offset(const aq_stack_t* prog, int M, int op);
+
+/*
+ * aq_check -- synchronises `stream`, then reports whether any kernel of this
+ * library gave up on a bounded device-side wait since the last aq_check
+ * (AQ_ERR_TIMEOUT; the record is cleared) or the stream saw a CUDA error
+ * (AQ_ERR_CUDA).  Outputs of a call that timed out are undefined.
+ */
+aq_status_t aq_check(aq_stream_t stream);
+
 /* Releases the handle and its device memory (synchronises its last stream). */
 void aq_free(aq_handle_t h);
 

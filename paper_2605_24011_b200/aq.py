@@ -26,7 +26,7 @@ AQ_OUT_STORE, AQ_OUT_ADD = 0, 1
 AQ_MAX_M, AQ_DECODE_MAX_M = 4096, 8
 
 SYMBOLS = ("aq_pack", "aq_import", "aq_export", "aq_info", "aq_dequant", "aq_linear", "aq_linear_f32out",
-           "aq_stack_workspace_bytes", "aq_stack_forward", "aq_stack_buffer_offset", "aq_free",
+           "aq_stack_workspace_bytes", "aq_stack_forward", "aq_stack_buffer_offset", "aq_stack_input_offset", "aq_check", "aq_free",
            "aq_status_string", "aq_last_cuda_error")
 
 _H = C.c_void_p
@@ -54,8 +54,12 @@ _lib.aq_stack_workspace_bytes.argtypes = [C.POINTER(Stack), C.c_int]
 _lib.aq_stack_workspace_bytes.restype = C.c_size_t
 _lib.aq_stack_buffer_offset.argtypes = [C.POINTER(Stack), C.c_int, C.c_int]
 _lib.aq_stack_buffer_offset.restype = C.c_size_t
+_lib.aq_stack_input_offset.argtypes = [C.POINTER(Stack), C.c_int, C.c_int]
+_lib.aq_stack_input_offset.restype = C.c_size_t
 _lib.aq_stack_forward.argtypes = [C.POINTER(Stack), C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p,
                                   C.c_size_t, C.c_void_p]
+_lib.aq_check.argtypes = [C.c_void_p]
+_lib.aq_check.restype = C.c_int
 _lib.aq_free.argtypes = [_H]
 _lib.aq_free.restype = None
 _lib.aq_status_string.argtypes = [C.c_int]
@@ -216,6 +220,9 @@ class Program:
     def buffer_offset(self, M: int, b: int) -> int:
         return int(_lib.aq_stack_buffer_offset(C.byref(self.c), M, b))
 
+    def input_offset(self, M: int, op: int) -> int:
+        return int(_lib.aq_stack_input_offset(C.byref(self.c), M, op))
+
 
 def aq_stack_workspace_bytes(prog: Program, M: int) -> int:
     return prog.workspace_bytes(M)
@@ -235,6 +242,19 @@ def stack_buffer(prog: Program, workspace, M: int, b: int):
     off = prog.buffer_offset(M, b)
     n = M * prog.buf_width[b]
     return workspace[off:off + 4 * n].view(torch.float32).view(M, prog.buf_width[b])
+
+
+def aq_check(stream=None) -> int:
+    """Synchronise the stream; raise if a device-side wait timed out or CUDA failed."""
+    _check(_lib.aq_check(_stream(stream)), "aq_check")
+    return AQ_OK
+
+
+def stack_input(prog: Program, workspace, M: int, op: int, dtype):
+    """[M][K] view (activation dtype) of the rounded input vector op `op` consumed."""
+    off = prog.input_offset(M, op)
+    K = prog.buf_width[prog.ops[op]["src"]]
+    return workspace[off:off + 2 * M * K].view(dtype).view(M, K)
 
 
 def raw_lib():

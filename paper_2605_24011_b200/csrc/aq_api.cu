@@ -207,6 +207,12 @@ aq_status_t aq_linear_f32out(aq_handle_t h, const void* x_dev, float* y_dev, int
     return linear_common(h, x_dev, y_dev, M, x_dtype, AQ_F32, stream);
 }
 
+aq_status_t aq_check(aq_stream_t stream) {
+    cudaError_t e = cudaStreamSynchronize((cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(e);
+    return read_gemm_status(true) ? AQ_ERR_TIMEOUT : AQ_OK;
+}
+
 void aq_free(aq_handle_t h) {
     if (!handle_ok(h)) return;
     cudaStreamSynchronize(h->last_stream);

@@ -45,5 +45,6 @@ cudaError_t launch_gemm(const aq_handle_s* h, const void* x, aq_dtype_t xdt, int
                         int64_t ldo, bool accumulate, cudaStream_t s);
 
 int sm_count();
+int read_gemm_status(bool clear);   // nonzero: a bounded wait in the GEMM kernel ran out
 
 }  // namespace aq

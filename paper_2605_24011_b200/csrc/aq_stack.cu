@@ -19,9 +19,15 @@ static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; 
 
 struct StackPlan {
     std::vector<size_t> buf_off;
-    size_t stage_off = 0;   // [M][maxK] activation-dtype staging of a phase input
+    std::vector<size_t> in_off;     // per op: its phase's staged input [M][K] (activation dtype)
+    std::vector<int> phase_first;   // first op of each phase
+    size_t stage_off = 0;           // end of the float32 buffers
     size_t total = 0;
 };
+
+static inline bool same_input(const aq_stack_op_t& a, const aq_stack_op_t& b) {
+    return a.src == b.src && a.in_op == b.in_op && (a.in_op != AQ_IN_SILU_MUL || a.src2 == b.src2);
+}
 
 static bool plan_stack(const aq_stack_t* p, int M, StackPlan& plan) {
     if (!p || !p->ops || !p->buf_width || p->n_ops < 1 || p->n_bufs < 2 || M < 1 || M > AQ_MAX_M) return false;
@@ -35,8 +41,6 @@ static bool plan_stack(const aq_stack_t* p, int M, StackPlan& plan) {
         if (p->buf_width[b] > maxw) maxw = p->buf_width[b];
     }
     plan.stage_off = off;
-    off += align_up((size_t)M * maxw * 2, 256);
-    plan.total = off;
     std::vector<char> written(p->n_bufs, 0);
     written[0] = 1;
     for (int i = 0; i < p->n_ops; ++i) {
@@ -54,6 +58,15 @@ static bool plan_stack(const aq_stack_t* p, int M, StackPlan& plan) {
         if (o.w->K != p->buf_width[o.src] || o.w->N != p->buf_width[o.dst]) return false;
         written[o.dst] = 1;
     }
+    plan.in_off.resize(p->n_ops);
+    for (int i = 0; i < p->n_ops; ++i) {
+        if (i > 0 && same_input(p->ops[i], p->ops[i - 1])) { plan.in_off[i] = plan.in_off[i - 1]; continue; }
+        plan.phase_first.push_back(i);
+        plan.in_off[i] = off;
+        off += align_up((size_t)M * p->buf_width[p->ops[i].src] * 2, 256);
+    }
+    plan.total = off;
+    (void)maxw;
     return true;
 }
 
@@ -115,7 +128,6 @@ static cudaError_t run_stack(const aq_stack_t* p, const StackPlan& plan, const T
     cudaError_t e = cudaMemsetAsync(ws, 0, plan.stage_off, s);
     if (e != cudaSuccess) return e;
     auto buf = [&](int b) { return reinterpret_cast<float*>(ws + plan.buf_off[b]); };
-    T* stage = reinterpret_cast<T*>(ws + plan.stage_off);
     {
         const int64_t n = (int64_t)M * p->buf_width[0];
         widen_kernel<T><<<(unsigned)((n + 255) / 256), 256, 0, s>>>(x0, buf(0), n);
@@ -124,10 +136,10 @@ static cudaError_t run_stack(const aq_stack_t* p, const StackPlan& plan, const T
     while (i < p->n_ops) {
         const aq_stack_op_t& f = p->ops[i];
         const int64_t K = p->buf_width[f.src];
+        T* stage = reinterpret_cast<T*>(ws + plan.in_off[i]);
         stage_kernel<T><<<M, 256, 0, s>>>(buf(f.src), f.in_op == AQ_IN_SILU_MUL ? buf(f.src2) : nullptr, f.in_op, K, stage);
         int j = i;
-        while (j < p->n_ops && p->ops[j].src == f.src && p->ops[j].in_op == f.in_op &&
-               (f.in_op != AQ_IN_SILU_MUL || p->ops[j].src2 == f.src2)) {
+        while (j < p->n_ops && same_input(p->ops[j], f)) {
             const aq_stack_op_t& o = p->ops[j];
             const int64_t N = p->buf_width[o.dst];
             if (o.out_op == AQ_OUT_ADD) {
@@ -165,6 +177,12 @@ size_t aq_stack_buffer_offset(const aq_stack_t* prog, int M, int b) {
     StackPlan plan;
     if (!plan_stack(prog, M, plan) || b < 0 || b >= prog->n_bufs) return (size_t)-1;
     return plan.buf_off[b];
+}
+
+size_t aq_stack_input_offset(const aq_stack_t* prog, int M, int op) {
+    StackPlan plan;
+    if (!plan_stack(prog, M, plan) || op < 0 || op >= prog->n_ops) return (size_t)-1;
+    return plan.in_off[op];
 }
 
 aq_status_t aq_stack_forward(const aq_stack_t* prog, const void* x0_dev, void* out_dev, int out_buf, int M,
