@@ -1,0 +1,321 @@
+#!/usr/bin/env python
+"""Benchmark of the low-bit linear hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One step = one pass of the 7B-class decoder linear stack (32 layers x
+{q,k,v,o,gate,up,down}, per-matrix 2/3/4-bit codes with mean width 2.5,
+blocks of 32 with fp16 scale+min) for M = 1 action decode: every packed weight
+byte is streamed once, with the glue (RMS scale, SiLU*up, residual adds)
+between the linears.  The headline metric is weight-stream GB/s.  The same
+JSON line carries the prefill (M = 512) TFLOP/s of the same stack, the
+standalone dequant GB/s, roofline fractions and the CPU oracle timed on the
+host cores.  With N > 1 every rank runs an independent replica (the path does
+not shard); value is the sum over ranks over the slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+NOMINAL_HBM_GBS = 8000.0
+NOMINAL_BF16_TFLOPS = 2250.0
+
+
+def _peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"], "bf16_tflops_sustained": d.get("bf16_tflops_sustained"),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while a region runs."""
+
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.index), "-lms", "100"], stdout=subprocess.PIPE, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons, power = [], [], set(), []
+        for ln in self.lines:
+            f = [s.strip() for s in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2])); power.append(float(f[3]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                "power_w_max": max(power), "samples": len(sm)}
+
+
+def _timed(fn, steps, warmup, torch):
+    """CUDA-event time of `steps` calls after `warmup` calls, in ms (total)."""
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1)
+
+
+def oracle_layer_sample(which=("q", "k", "v", "o", "gate", "up", "down")):
+    """Host-side inputs for the oracle timing: one 7B-shaped layer (or part of it)."""
+    import numpy as np
+    from oracle import aq_oracle as O
+    from paper_2605_24011_b200 import synth
+    shapes = [s for s in synth.llama7b_layer() if s[0] in which]
+    bits = {"q": 2, "k": 2, "v": 3, "o": 3, "gate": 2, "up": 2, "down": 4}
+    mats = []
+    for i, (name, N, K) in enumerate(shapes):
+        W = synth.weights(N, K, 77, i, outliers=True)
+        d, m, q = O.quantize(W, bits[name])
+        x = synth.activations(1, K, 77, i).astype(np.float16).astype(np.float64)
+        mats.append((d, m, q, x, N * K * (bits[name] + 1) // 8))
+    return mats
+
+
+def time_oracle(mats, repeats=1):
+    from oracle import aq_oracle as O
+    t0 = time.perf_counter()
+    for _ in range(repeats):
+        for (d, m, q, x, _) in mats:
+            O.linear(d, m, q, x)
+    dt = time.perf_counter() - t0
+    return dt, sum(b for *_, b in mats) * repeats
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle, as it stands, on the host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cores = len(os.sched_getaffinity(0))
+    mats = oracle_layer_sample(which=("q",))
+    for _ in range(args.warmup):
+        time_oracle(mats)
+    t, nbytes = 0.0, 0
+    for _ in range(args.steps):
+        dt, nb = time_oracle(mats)
+        t += dt; nbytes += nb
+    val = nbytes / t / 1e9
+    sample = "per step: oracle dequant + fp64 mat-vec of one 4096x4096 2-bit matrix of the stack (M=1)"
+    line = {"impl": "reference", "metric": "decode_weight_stream", "value": val, "unit": "GB/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "sample": sample},
+            "cpu_baseline": {"value": val, "unit": "GB/s", "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": val, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+WORKLOAD = ("7B-class decoder linear stack, M=1 decode: 32 layers x {q,k,v,o 4096x4096; gate,up 11008x4096; "
+            "down 4096x11008}, per-matrix 2/3/4-bit (mean 2.5), blocks of 32 + fp16 scale/min, N(0,0.02) weights "
+            "with 0.1% x20 outliers, x fp16 N(0,1)")
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
+    ap.add_argument("--layers", type=int, default=32, help="decoder layers (32 = the full workload)")
+    ap.add_argument("--no-extras", action="store_true", help="skip prefill / dequant / oracle legs")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import numpy as np
+    import torch
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    from paper_2605_24011_b200 import aq, synth, workloads
+    peaks = _peaks()
+    warm = max(3, args.warmup)
+
+    # ---- set-up (untimed): generate, pack, wire --------------------------------------------------
+    prog, out_buf, names, _, info = workloads.llama7b_decode_stack(n_layers=args.layers, seed=0)
+    M = 1
+    ws = torch.empty(prog.workspace_bytes(M), dtype=torch.uint8, device="cuda")
+    x0 = workloads.activations_device(M, 4096, torch.float16, 3, 0)
+    out = torch.empty((M, 4096), dtype=torch.float16, device="cuda")
+    x0_host = x0.cpu().pin_memory()
+    out_host = torch.empty_like(out, device="cpu").pin_memory()
+    packed = info["packed_bytes"]
+
+    def step():
+        aq.aq_stack_forward(prog, x0, out, out_buf, M, ws)
+
+    def step_e2e():
+        x0.copy_(x0_host, non_blocking=True)
+        aq.aq_stack_forward(prog, x0, out, out_buf, M, ws)
+        out_host.copy_(out, non_blocking=True)
+
+    # ---- timed: device-resident, then end to end ---------------------------------------------------
+    sampler = ClockSampler(local)
+    for _ in range(warm):
+        step()
+    torch.cuda.synchronize()
+    if dist:
+        dist.barrier()
+    sampler.start()
+    l0 = aq.aq_kernel_launches()
+    ms = _timed(step, args.steps, 0, torch)
+    launches = aq.aq_kernel_launches() - l0
+    if dist:
+        dist.barrier()
+    ms_e2e = _timed(step_e2e, args.steps, 3, torch)
+    clocks = sampler.stop()
+    aq.aq_check()
+    if dist:
+        t = torch.tensor([ms, ms_e2e], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, ms_e2e = float(t[0]), float(t[1])
+    ms_step = ms / args.steps
+    value = world * packed / (ms_step * 1e-3) / 1e9
+    e2e = world * packed / (ms_e2e / args.steps * 1e-3) / 1e9
+
+    line = {
+        "metric": "decode_weight_stream", "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+        "warmup": warm, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f16", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "layers": args.layers, "M": 1, "packed_bytes_per_step": packed,
+                   "mean_code_bits": info["mean_code_bits"], "stored_bits_per_weight": 8.0 * packed / info["weights"],
+                   "l2": "inputs larger than L2: every step streams all packed weights (>> 126 MB) once",
+                   "parallelism": "replicas only (one GPU per replica, no collective)"},
+        "clocks": clocks,
+        "e2e": {"value": e2e, "unit": "GB/s", "h2d_bytes_per_step": int(x0_host.numel() * 2),
+                "d2h_bytes_per_step": int(out_host.numel() * 2), "ms_per_step": ms_e2e / args.steps},
+        "gpu_launches": int(launches),
+        "us_per_decode_pass": 1e3 * ms_step,
+        "pct_of_nominal_hbm": 100.0 * (value / world) / NOMINAL_HBM_GBS,
+        "roofline": {"bound": "hbm", "achieved": value / world, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": (value / world) / peaks["hbm_gbs"], "traffic": DECODE_TRAFFIC_BYTES,
+                     "peak_source": peaks["source"], "kernel": "gemv_kernel (all launches of one stack pass)",
+                     "algorithmic_bytes_per_step": packed},
+    }
+
+    if world == 1 and rank == 0 and not args.no_extras:
+        line["prefill"] = prefill_leg(aq, workloads, prog, out_buf, info, peaks, torch)
+        line["dequant"] = dequant_leg(aq, synth, peaks, torch)
+        cores = len(os.sched_getaffinity(0))
+        mats = oracle_layer_sample()
+        dt, nb = time_oracle(mats)
+        line["cpu_baseline"] = {"value": nb / dt / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
+                                "seconds": dt,
+                                "sample": "one 7B-shaped layer (7 matrices, 202M weights, M=1): oracle dequant + fp64 mat-vec"}
+    if rank == 0:
+        print(json.dumps(line))
+    if dist:
+        dist.destroy_process_group()
+
+
+# dram__bytes_read.sum + dram__bytes_write.sum of the decode kernel per stack pass, from the ncu
+# capture summarised under profiles/ (None until a capture has been taken).
+DECODE_TRAFFIC_BYTES = None
+PREFILL_TRAFFIC_BYTES = None
+
+
+def prefill_leg(aq, workloads, prog, out_buf, info, peaks, torch):
+    """Same stack, M = 512 prefill: 256 vision-like rows + 256 text rows, bf16."""
+    M = 512
+    ws = torch.empty(prog.workspace_bytes(M), dtype=torch.uint8, device="cuda")
+    x0 = workloads.activations_device(M, 4096, torch.bfloat16, 4, 0, kind="vision_text")
+    out = torch.empty((M, 4096), dtype=torch.bfloat16, device="cuda")
+
+    def step():
+        aq.aq_stack_forward(prog, x0, out, out_buf, M, ws)
+
+    l0 = aq.aq_kernel_launches()
+    ms = _timed(step, 5, 3, torch) / 5
+    launches = (aq.aq_kernel_launches() - l0) // 8
+    aq.aq_check()
+    flops = 2.0 * M * info["weights"]
+    tf = flops / (ms * 1e-3) / 1e12
+    return {"workload": "same stack, M=512 (256 vision rows N(0,1)*U(0.5,2) + 256 text rows), bf16, dequant->tcgen05 GEMM",
+            "ms_per_pass": ms, "tflops": tf, "pct_of_nominal_bf16": 100.0 * tf / NOMINAL_BF16_TFLOPS,
+            "gpu_launches_per_pass": int(launches),
+            "roofline": {"bound": "tensor", "achieved": tf, "peak": peaks["bf16_tflops_sustained"] or peaks["bf16_tflops"],
+                         "unit": "TFLOP/s", "frac": tf / (peaks["bf16_tflops_sustained"] or peaks["bf16_tflops"]),
+                         "traffic": PREFILL_TRAFFIC_BYTES, "peak_source": peaks["source"] + " (sustained: timed inside a long step)",
+                         "kernel": "gemm_kernel (all launches of one stack pass, glue kernels included in the time)"}}
+
+
+def dequant_leg(aq, synth, peaks, torch):
+    """Standalone dequant, K = N = 4096 4-bit, rotating over 24 packed copies so that every call misses L2."""
+    N = K = 4096
+    W = synth.weights_device(N, K, 1)
+    hs = [aq.aq_pack(4, 32, W) for _ in range(24)]
+    outs = [torch.empty((N, K), dtype=torch.float16, device="cuda") for _ in range(8)]
+    i = [0]
+
+    def step():
+        aq.aq_dequant(hs[i[0] % 24], outs[i[0] % 8])
+        i[0] += 1
+
+    ms = _timed(step, 48, 8, torch) / 48
+    nbytes = N * K * 5 // 8 + N * K * 2
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    for h in hs:
+        h.free()
+    return {"workload": "aq_dequant 4096x4096 4-bit -> fp16, cold L2 (24 packed copies, 8 outputs in rotation)",
+            "us_per_call": 1e3 * ms, "gbs": gbs,
+            "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": gbs / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"]}}
+
+
+if __name__ == "__main__":
+    main()

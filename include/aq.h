@@ -205,6 +205,9 @@ const char* aq_status_string(aq_status_t s);
 /* Text of the last CUDA error this thread's libaq call saw ("" if none). */
 const char* aq_last_cuda_error(void);
 
+/* Number of CUDA kernels this library has launched in this process so far. */
+uint64_t aq_kernel_launches(void);
+
 #ifdef __cplusplus
 }
 #endif

@@ -27,7 +27,7 @@ AQ_MAX_M, AQ_DECODE_MAX_M = 4096, 8
 
 SYMBOLS = ("aq_pack", "aq_import", "aq_export", "aq_info", "aq_dequant", "aq_linear", "aq_linear_f32out",
            "aq_stack_workspace_bytes", "aq_stack_forward", "aq_stack_buffer_offset", "aq_stack_input_offset", "aq_check", "aq_free",
-           "aq_status_string", "aq_last_cuda_error")
+           "aq_status_string", "aq_last_cuda_error", "aq_kernel_launches")
 
 _H = C.c_void_p
 
@@ -64,6 +64,8 @@ _lib.aq_free.argtypes = [_H]
 _lib.aq_free.restype = None
 _lib.aq_status_string.argtypes = [C.c_int]
 _lib.aq_status_string.restype = C.c_char_p
+_lib.aq_kernel_launches.argtypes = []
+_lib.aq_kernel_launches.restype = C.c_uint64
 _lib.aq_last_cuda_error.argtypes = []
 _lib.aq_last_cuda_error.restype = C.c_char_p
 for _n in ("aq_pack", "aq_import", "aq_export", "aq_info", "aq_dequant", "aq_linear", "aq_linear_f32out",
@@ -255,6 +257,10 @@ def stack_input(prog: Program, workspace, M: int, op: int, dtype):
     off = prog.input_offset(M, op)
     K = prog.buf_width[prog.ops[op]["src"]]
     return workspace[off:off + 2 * M * K].view(dtype).view(M, K)
+
+
+def aq_kernel_launches() -> int:
+    return int(_lib.aq_kernel_launches())
 
 
 def raw_lib():

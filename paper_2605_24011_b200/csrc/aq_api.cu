@@ -2,6 +2,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <atomic>
 #include <new>
 
 #include "aq_internal.h"
@@ -17,6 +18,9 @@ aq_status_t cuda_fail(cudaError_t e) {
 }
 
 bool handle_ok(aq_handle_t h) { return h != nullptr && h->magic == AQ_HANDLE_MAGIC; }
+
+static std::atomic<uint64_t> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
 
 int sm_count() {
     static int n = 0;
@@ -234,5 +238,7 @@ const char* aq_status_string(aq_status_t s) {
 }
 
 const char* aq_last_cuda_error(void) { return g_last_err; }
+
+uint64_t aq_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
 
 }  // extern "C"

@@ -91,6 +91,7 @@ static cudaError_t launch_bits(const aq_handle_s* h, void* out, aq_dtype_t dt, c
         dequant_kernel<BITS, __nv_bfloat16><<<grid, 256, 0, s>>>(h->frags, h->N, h->K, h->NT, h->n_frags, (__nv_bfloat16*)out);
     else
         dequant_kernel<BITS, float><<<grid, 256, 0, s>>>(h->frags, h->N, h->K, h->NT, h->n_frags, (float*)out);
+    count_launch();
     return cudaGetLastError();
 }
 

@@ -348,6 +348,7 @@ static cudaError_t launch_one(const CUtensorMap& tm, const GemmArgs& a, dim3 gri
         configured = true;
     }
     kern<<<grid, GM_THREADS, SMEM, s>>>(tm, a);
+    count_launch();
     return cudaGetLastError();
 }
 

@@ -263,6 +263,7 @@ static cudaError_t launch_one(const GemvArgs& a, cudaStream_t s) {
     const int64_t need = (warps_wanted + GEMV_WARPS - 1) / GEMV_WARPS;
     if (need < grid) grid = (int)need;
     kern<<<grid, GEMV_WARPS * 32, SMEM, s>>>(a);
+    count_launch();
     return cudaGetLastError();
 }
 
@@ -307,6 +308,7 @@ cudaError_t launch_finalize(const float* acc_in, float* acc_zero, int64_t ldacc,
     if (ydt == AQ_F16) finalize_kernel<__half><<<grid, 256, 0, s>>>(acc_in, acc_zero, ldacc, (__half*)y, M, N);
     else if (ydt == AQ_BF16) finalize_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>(acc_in, acc_zero, ldacc, (__nv_bfloat16*)y, M, N);
     else finalize_kernel<float><<<grid, 256, 0, s>>>(acc_in, acc_zero, ldacc, (float*)y, M, N);
+    count_launch();
     return cudaGetLastError();
 }
 

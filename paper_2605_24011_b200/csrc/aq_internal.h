@@ -45,6 +45,7 @@ cudaError_t launch_gemm(const aq_handle_s* h, const void* x, aq_dtype_t xdt, int
                         int64_t ldo, bool accumulate, cudaStream_t s);
 
 int sm_count();
+void count_launch(int n = 1);       // process-wide count of this library's kernel launches
 int read_gemm_status(bool clear);   // nonzero: a bounded wait in the GEMM kernel ran out
 
 }  // namespace aq

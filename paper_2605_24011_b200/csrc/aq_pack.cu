@@ -177,6 +177,7 @@ cudaError_t launch_pack(const aq_handle_s* h, const float* W, cudaStream_t s) {
         case 3: pack_kernel<3><<<grid, 128, 0, s>>>(W, h->N, h->K, h->NT, h->n_frags, h->frags, h->flags); break;
         default: pack_kernel<4><<<grid, 128, 0, s>>>(W, h->N, h->K, h->NT, h->n_frags, h->frags, h->flags); break;
     }
+    count_launch();
     return cudaGetLastError();
 }
 
@@ -187,6 +188,7 @@ cudaError_t launch_import(const aq_handle_s* h, const uint8_t* canon_dev, cudaSt
         case 3: import_kernel<3><<<grid, 128, 0, s>>>(canon_dev, h->N, h->K, h->NT, h->n_frags, h->frags); break;
         default: import_kernel<4><<<grid, 128, 0, s>>>(canon_dev, h->N, h->K, h->NT, h->n_frags, h->frags); break;
     }
+    count_launch();
     return cudaGetLastError();
 }
 
@@ -194,6 +196,7 @@ cudaError_t launch_export(const aq_handle_s* h, uint8_t* canon_dev, cudaStream_t
     const int64_t n = h->N * (h->K / 32);
     const unsigned grid = (unsigned)((n + 127) / 128);
     export_kernel<<<grid, 128, 0, s>>>(h->frags, h->bits, h->N, h->K, h->NT, canon_dev);
+    count_launch();
     return cudaGetLastError();
 }
 

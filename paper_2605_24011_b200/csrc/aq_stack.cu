@@ -125,12 +125,17 @@ __global__ void __launch_bounds__(256) stage_kernel(const float* __restrict__ sr
 template <typename T>
 static cudaError_t run_stack(const aq_stack_t* p, const StackPlan& plan, const T* x0, T* out, int out_buf, int M,
                              aq_dtype_t dt, uint8_t* ws, cudaStream_t s) {
-    cudaError_t e = cudaMemsetAsync(ws, 0, plan.stage_off, s);
-    if (e != cudaSuccess) return e;
+    cudaError_t e = cudaSuccess;
+    const bool decode = (M <= AQ_DECODE_MAX_M);
+    if (decode) {   // the streaming kernel accumulates with red.add: outputs start at zero
+        e = cudaMemsetAsync(ws, 0, plan.stage_off, s);
+        if (e != cudaSuccess) return e;
+    }
     auto buf = [&](int b) { return reinterpret_cast<float*>(ws + plan.buf_off[b]); };
     {
         const int64_t n = (int64_t)M * p->buf_width[0];
         widen_kernel<T><<<(unsigned)((n + 255) / 256), 256, 0, s>>>(x0, buf(0), n);
+        count_launch();
     }
     int i = 0;
     while (i < p->n_ops) {
@@ -138,6 +143,7 @@ static cudaError_t run_stack(const aq_stack_t* p, const StackPlan& plan, const T
         const int64_t K = p->buf_width[f.src];
         T* stage = reinterpret_cast<T*>(ws + plan.in_off[i]);
         stage_kernel<T><<<M, 256, 0, s>>>(buf(f.src), f.in_op == AQ_IN_SILU_MUL ? buf(f.src2) : nullptr, f.in_op, K, stage);
+        count_launch();
         int j = i;
         while (j < p->n_ops && same_input(p->ops[j], f)) {
             const aq_stack_op_t& o = p->ops[j];
@@ -146,8 +152,8 @@ static cudaError_t run_stack(const aq_stack_t* p, const StackPlan& plan, const T
                 e = cudaMemcpyAsync(buf(o.dst), buf(o.res), (size_t)M * N * sizeof(float), cudaMemcpyDeviceToDevice, s);
                 if (e != cudaSuccess) return e;
             }
-            if (M <= AQ_DECODE_MAX_M) e = launch_gemv(o.w, stage, dt, M, buf(o.dst), N, s);
-            else e = launch_gemm(o.w, stage, dt, M, buf(o.dst), N, true, s);
+            if (decode) e = launch_gemv(o.w, stage, dt, M, buf(o.dst), N, s);
+            else e = launch_gemm(o.w, stage, dt, M, buf(o.dst), N, o.out_op == AQ_OUT_ADD, s);
             if (e != cudaSuccess) return e;
             o.w->last_stream = s;
             ++j;
@@ -157,6 +163,7 @@ static cudaError_t run_stack(const aq_stack_t* p, const StackPlan& plan, const T
     if (out) {
         const int64_t n = (int64_t)M * p->buf_width[out_buf];
         narrow_kernel<T><<<(unsigned)((n + 255) / 256), 256, 0, s>>>(buf(out_buf), out, n);
+        count_launch();
     }
     return cudaGetLastError();
 }
