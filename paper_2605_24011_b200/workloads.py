@@ -13,8 +13,16 @@ import numpy as np
 from . import aq, programs, synth
 
 
+def _flat(key):
+    for k in key:
+        if isinstance(k, (tuple, list)):
+            yield from _flat(k)
+        else:
+            yield int(k) & 0xFFFFFFFF
+
+
 def _seed(*key) -> int:
-    return int(np.random.SeedSequence([int(k) & 0xFFFFFFFF for k in key]).generate_state(1)[0])
+    return int(np.random.SeedSequence(list(_flat(key))).generate_state(1)[0])
 
 
 def build_stack(layer_shapes, n_layers, bits, key, outliers=False, sample_rows=0, device="cuda"):
