@@ -129,6 +129,35 @@ aq_status_t aq_linear_f32out(aq_handle_t h, const void* x_dev, float* y_dev, int
                              aq_dtype_t x_dtype, aq_stream_t stream);
 
 /*
+ * aq_linear_noalloc -- aq_linear for M <= AQ_DECODE_MAX_M that reserves no
+ * memory.  (No counterpart in the paper: this entry point exists for the
+ * library's users, not for the method.)
+ *
+ * Who needs it: code that runs where device allocation is forbidden or
+ * unaffordable -- a control loop with a hard deadline that may not take the
+ * allocator's locks or an implicit device synchronisation, a process whose
+ * memory budget was fixed at start-up, a plug-in that is handed a stream and
+ * told not to touch the allocator.  aq_linear itself allocates nothing per
+ * call either, but its accumulation scratch was allocated when the handle was
+ * made; here the scratch is a fixed array of AQ_DECODE_MAX_M *
+ * AQ_NOALLOC_MAX_N float32 (512 KiB) in the library's device image, which every
+ * GPU that loads the library holds until the process exits.
+ *
+ *   arguments as aq_linear (x_dev, y_dev DEVICE, 16-byte aligned, same dtype)
+ *   AQ_ERR_UNSUPPORTED when M > AQ_DECODE_MAX_M or N (rounded up to 16) >
+ *   AQ_NOALLOC_MAX_N: the fixed scratch cannot hold the sums.
+ * The first call on each device looks up the array's device address (with that
+ * device current); make that first call before any stream capture begins.
+ * All calls on a device share the one array: it is cleared on the stream at the
+ * start of every call, and two calls that overlap on the GPU (different
+ * streams, no ordering) race on it and corrupt each other's result.
+ * Calls no cudaMalloc/cudaFree and no allocating library routine.
+ */
+#define AQ_NOALLOC_MAX_N 16384
+aq_status_t aq_linear_noalloc(aq_handle_t h, const void* x_dev, void* y_dev, int M,
+                              aq_dtype_t xy_dtype, aq_stream_t stream);
+
+/*
  * A program over a list of handles: the linears of a stack of transformer
  * blocks (Section 3: each block holds W_Q, W_K, W_V, W_O, W_gate, W_up,
  * W_down) with the glue between them.  Activations live in float32 buffers

@@ -25,7 +25,7 @@ AQ_IN_PLAIN, AQ_IN_RMSNORM, AQ_IN_SILU_MUL = 0, 1, 2
 AQ_OUT_STORE, AQ_OUT_ADD = 0, 1
 AQ_MAX_M, AQ_DECODE_MAX_M = 4096, 8
 
-SYMBOLS = ("aq_pack", "aq_import", "aq_export", "aq_info", "aq_dequant", "aq_linear", "aq_linear_f32out",
+SYMBOLS = ("aq_pack", "aq_import", "aq_export", "aq_info", "aq_dequant", "aq_linear", "aq_linear_f32out", "aq_linear_noalloc",
            "aq_stack_workspace_bytes", "aq_stack_forward", "aq_stack_buffer_offset", "aq_stack_input_offset", "aq_check", "aq_free",
            "aq_status_string", "aq_last_cuda_error", "aq_kernel_launches")
 
@@ -50,6 +50,8 @@ _lib.aq_info.argtypes = [_H, C.POINTER(C.c_int), C.POINTER(C.c_int), C.POINTER(C
 _lib.aq_dequant.argtypes = [_H, C.c_void_p, C.c_int, C.c_void_p]
 _lib.aq_linear.argtypes = [_H, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p]
 _lib.aq_linear_f32out.argtypes = [_H, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p]
+_lib.aq_linear_noalloc.argtypes = [_H, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p]
+_lib.aq_linear_noalloc.restype = C.c_int
 _lib.aq_stack_workspace_bytes.argtypes = [C.POINTER(Stack), C.c_int]
 _lib.aq_stack_workspace_bytes.restype = C.c_size_t
 _lib.aq_stack_buffer_offset.argtypes = [C.POINTER(Stack), C.c_int, C.c_int]
@@ -198,6 +200,17 @@ def aq_linear(h: Handle, x, y, M: int | None = None, stream=None):
         if dtype_code(y) != dtype_code(x):
             raise AqError(AQ_ERR_INVALID_ARG, "aq_linear: y dtype must equal x dtype (or float32)")
         _check(_lib.aq_linear(h.raw, _ptr(x), _ptr(y), M, dtype_code(x), _stream(stream)), "aq_linear")
+    return y
+
+
+def aq_linear_noalloc(h: Handle, x, y, M: int | None = None, stream=None):
+    """aq_linear for M <= 8 that reserves no memory: the sums are built in a fixed
+    512 KiB array inside the library instead of scratch owned by the handle.  For
+    callers that may not allocate on the device (deadline loops, fixed memory
+    budgets).  x, y: CUDA tensors of the same half-precision dtype.  Calls on one
+    GPU share the array, so they must not overlap."""
+    M = int(x.shape[0]) if M is None else M
+    _check(_lib.aq_linear_noalloc(h.raw, _ptr(x), _ptr(y), M, dtype_code(x), _stream(stream)), "aq_linear_noalloc")
     return y
 
 
