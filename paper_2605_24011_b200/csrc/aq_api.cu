@@ -214,12 +214,14 @@ aq_status_t aq_linear_f32out(aq_handle_t h, const void* x_dev, float* y_dev, int
 aq_status_t aq_check(aq_stream_t stream) {
     cudaError_t e = cudaStreamSynchronize((cudaStream_t)stream);
     if (e != cudaSuccess) return cuda_fail(e);
-    return read_gemm_status(true) ? AQ_ERR_TIMEOUT : AQ_OK;
+    const int g = read_gemm_status(true), d = read_decode_status(true);
+    return (g || d) ? AQ_ERR_TIMEOUT : AQ_OK;
 }
 
 void aq_free(aq_handle_t h) {
     if (!handle_ok(h)) return;
     cudaStreamSynchronize(h->last_stream);
+    decode_stack_forget(h);
     destroy(h);
 }
 

@@ -1,0 +1,664 @@
+// Decode path for a whole program of linears (M = 1..8) in ONE persistent
+// kernel launch (Section 4.3: the deployed forward pass dispatches every
+// quantised matmul to a low-bit kernel; Appendix D: dequantise on the fly).
+//
+// Bound: HBM -- every packed byte of every matrix is read once per pass.  A
+// 4096 x 4096 matrix is about a microsecond of HBM time, less than a kernel
+// launch, so the pass runs as one cooperative grid of one CTA per SM:
+//
+//   * Work.  Consecutive ops that read the same input vector form a phase.
+//     The units (16 rows x 256 k) of a phase's matrices are concatenated and
+//     dealt as contiguous runs: first to CTAs, then to the warps of a CTA.
+//   * Weight stream.  Which bytes a warp will need does not depend on any
+//     activation, so every warp keeps a private ring of bulk copies
+//     (cp.async.bulk + mbarrier, L2 evict-first) running ahead of what it
+//     consumes, across op and phase boundaries.
+//   * Dependencies.  Sums leave the warps as fp32 red.add into the output
+//     buffer.  Every op has an arrival counter in global memory; a CTA arrives
+//     once all its warps have committed their share of the op.  Before a phase
+//     a CTA waits (bounded) until the ops that wrote the buffers it reads have
+//     been arrived at by every CTA.  Ops nobody waits for soon (k and v of an
+//     attention block) therefore overlap the wait of the ops that follow.
+//   * Glue.  At the start of a phase each CTA forms, in shared memory, the
+//     rounded input vector for the k-slabs its warps will touch (RMS scaling /
+//     SiLU(g)*u / plain), and writes its share of the vector to the caller's
+//     workspace, where every op's input stays readable after the call.
+//
+// Every wait is bounded: when one runs out the kernel raises a status word,
+// waits (bounded) for its own copies in flight and returns.
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+#include <cstring>
+#include <mutex>
+#include <vector>
+
+#include "aq_gemv_core.cuh"
+#include "aq_internal.h"
+
+namespace aq {
+
+constexpr int DS_WARPS = 16;
+constexpr int DS_THREADS = DS_WARPS * 32;
+constexpr int DS_SLOTS = 5;                 // ring depth per warp (units)
+constexpr int DS_SLOT_BYTES = 2560;         // the largest unit (4-bit: 2 fragments of 1280 B)
+constexpr int DS_XS_BYTES = 16384;          // staged input: tokens x slabs <= 32 (a slab = 256 k = 512 B per token)
+constexpr int DS_MAX_PHASE_OPS = 8;
+constexpr int DS_MAX_DEPS = 12;
+constexpr uint64_t DS_WAIT_NS = 2000000000ull;   // every wait gives up after two seconds
+
+__device__ int g_decode_status = 0;   // nonzero: a bounded wait ran out (1 = counter, 2 = copy)
+
+struct DsOp {
+    const uint8_t* frags;
+    float* dst;            // float32 [M][N]
+    const float* res;      // float32 [M][N] added once (by the k-slab-0 units), or null
+    int32_t N;             // true rows
+    int32_t NT;            // 16-row tiles
+    int32_t n_units;       // KP * NT
+    int32_t unit_off;      // offset of this op's units inside its phase
+    int32_t bits;
+    int32_t pad_;
+};
+
+struct DsPhase {
+    const float* src;      // float32 [M][K]
+    const float* src2;     // second input of AQ_IN_SILU_MUL, else null
+    void* stage;           // [M][K] of the activation dtype: the rounded input, kept for the caller
+    int32_t K;
+    int32_t in_op;
+    int32_t op_first;      // index of ops[0] in the program (names its arrival counter)
+    int32_t op_count;
+    int32_t units_total;
+    int32_t n_deps;
+    int16_t deps[DS_MAX_DEPS];   // ops that must be complete before this phase reads its inputs
+    int32_t pad_[2];
+    DsOp ops[DS_MAX_PHASE_OPS];
+};
+static_assert(sizeof(DsOp) == 48, "DsOp layout");
+static_assert(sizeof(DsPhase) % 16 == 0, "a phase record is fetched with one bulk copy");
+
+struct DsArgs {
+    const DsPhase* phases;
+    uint32_t* cnt;         // per-op arrival counters, zero at launch
+    int n_phases;
+    int M;
+};
+
+// ---- small PTX wrappers ---------------------------------------------------------
+__device__ __forceinline__ uint32_t ds_smem(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void ds_mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void ds_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool ds_mbar_try(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ void ds_bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, uint64_t pol) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(pol) : "memory");
+}
+__device__ __forceinline__ uint64_t ds_now_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait on a shared-memory barrier; false when DS_WAIT_NS passed.
+__device__ __forceinline__ bool ds_mbar_wait(uint32_t bar, uint32_t parity) {
+    if (ds_mbar_try(bar, parity)) return true;
+    const uint64_t t0 = ds_now_ns();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 64; ++i)
+            if (ds_mbar_try(bar, parity)) return true;
+        if (ds_now_ns() - t0 > DS_WAIT_NS) return false;
+    }
+}
+__device__ __forceinline__ uint32_t ds_ld_acquire(const uint32_t* p) {
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// ---- the warp's position in its stream of units ---------------------------------
+struct DsCursor {
+    int ph;                // phase (n_phases: past the end)
+    int oi;                // op inside the phase
+    int wa, wb;            // the warp's run inside the phase's concatenated units
+    int u, u_end;          // position inside the current op
+    const uint8_t* base;   // the op's fragments
+    int ub;                // bytes per unit
+};
+
+// The run of units warp `warp` of CTA `cta` owns in a phase of `total` units.
+__device__ __forceinline__ void ds_warp_run(int total, int cta, int ncta, int warp, int& wa, int& wb) {
+    const int a = (int)(((int64_t)total * cta) / ncta), b = (int)(((int64_t)total * (cta + 1)) / ncta);
+    const int n = b - a;
+    wa = a + (int)(((int64_t)n * warp) / DS_WARPS);
+    wb = a + (int)(((int64_t)n * (warp + 1)) / DS_WARPS);
+}
+
+// Moves the cursor to the next op (from (ph, oi) on) in which the warp owns units.
+__device__ __forceinline__ void ds_seek(DsCursor& c, const DsArgs& a, int warp, bool new_phase) {
+    while (c.ph < a.n_phases) {
+        const DsPhase* P = a.phases + c.ph;
+        if (new_phase) {
+            ds_warp_run(__ldg(&P->units_total), blockIdx.x, gridDim.x, warp, c.wa, c.wb);
+            c.oi = 0;
+            new_phase = false;
+        }
+        const int oc = __ldg(&P->op_count);
+        while (c.oi < oc) {
+            const DsOp* op = P->ops + c.oi;
+            const int off = __ldg(&op->unit_off), n = __ldg(&op->n_units);
+            const int u0 = max(c.wa, off) - off, u1 = min(c.wb, off + n) - off;
+            if (u0 < u1) {
+                c.u = u0; c.u_end = u1;
+                c.ub = 2 * frag_bytes(__ldg(&op->bits));
+                c.base = reinterpret_cast<const uint8_t*>(__ldg(reinterpret_cast<const unsigned long long*>(&op->frags)));
+                return;
+            }
+            ++c.oi;
+        }
+        ++c.ph;
+        new_phase = true;
+    }
+}
+
+// ---- glue arithmetic --------------------------------------------------------------
+__device__ __forceinline__ float ds_silu_mul(float g, float u) { return g / (1.f + expf(-g)) * u; }
+
+template <bool BF16>
+__device__ __forceinline__ uint2 ds_round4(const float4& v) {
+    uint2 r;
+    if constexpr (BF16) {
+        __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y), b = __floats2bfloat162_rn(v.z, v.w);
+        r.x = *reinterpret_cast<uint32_t*>(&a); r.y = *reinterpret_cast<uint32_t*>(&b);
+    } else {
+        __half2 a = __floats2half2_rn(v.x, v.y), b = __floats2half2_rn(v.z, v.w);
+        r.x = *reinterpret_cast<uint32_t*>(&a); r.y = *reinterpret_cast<uint32_t*>(&b);
+    }
+    return r;
+}
+
+// Four consecutive elements of the rounded input vector of token m at k (k % 4 == 0, k < K).
+template <bool BF16>
+__device__ __forceinline__ uint2 ds_form4(const DsPhase& P, int m, int k, float scale) {
+    const float4 s = *reinterpret_cast<const float4*>(P.src + (int64_t)m * P.K + k);
+    float4 v;
+    if (P.in_op == AQ_IN_SILU_MUL) {
+        const float4 t = *reinterpret_cast<const float4*>(P.src2 + (int64_t)m * P.K + k);
+        v = make_float4(ds_silu_mul(s.x, t.x), ds_silu_mul(s.y, t.y), ds_silu_mul(s.z, t.z), ds_silu_mul(s.w, t.w));
+    } else {
+        v = make_float4(s.x * scale, s.y * scale, s.z * scale, s.w * scale);
+    }
+    return ds_round4<BF16>(v);
+}
+
+// The x operand of pair-slab P from the staged vector in shared memory:
+// xs points at [slab - slab_lo][M][256] halves of the op's segment.
+template <int MT, bool BF16>
+__device__ __forceinline__ void ds_load_x_operand(XOperand<MT>& xo, const uint16_t* xs, int M, int lane) {
+    constexpr int BG = XOperand<MT>::BG, NG = XOperand<MT>::NG;
+    const int g = lane >> 2, t = lane & 3;
+    const int tok = g % MT, bs = g / MT;
+#pragma unroll
+    for (int fi = 0; fi < 2; ++fi) {
+#pragma unroll
+        for (int gi = 0; gi < NG; ++gi) {
+            const int jb = gi * BG + bs;
+            uint4 v = make_uint4(0, 0, 0, 0);
+            if (tok < M) v = *reinterpret_cast<const uint4*>(xs + tok * 256 + fi * 128 + 32 * jb + 8 * t);
+            float s = sum8<BF16>(v);
+            s += __shfl_xor_sync(0xffffffffu, s, 1);
+            s += __shfl_xor_sync(0xffffffffu, s, 2);
+            xo.X0[fi][gi] = __shfl_sync(0xffffffffu, s, (2 * t) * 4);
+            xo.X1[fi][gi] = __shfl_sync(0xffffffffu, s, (2 * t + 1) * 4);
+#pragma unroll
+            for (int b2 = 0; b2 < BG; ++b2) {
+                const bool on = (b2 == bs);
+                xo.b[fi][gi * BG + b2][0] = on ? v.x : 0u;
+                xo.b[fi][gi * BG + b2][1] = on ? v.y : 0u;
+                xo.b[fi][gi * BG + b2][2] = on ? v.z : 0u;
+                xo.b[fi][gi * BG + b2][3] = on ? v.w : 0u;
+            }
+        }
+    }
+}
+
+// ---- the kernel ---------------------------------------------------------------------
+struct DsShared {
+    alignas(128) uint8_t ring[DS_WARPS][DS_SLOTS][DS_SLOT_BYTES];
+    alignas(16) uint16_t xs[DS_XS_BYTES / 2];
+    alignas(16) DsPhase rec[2];             // descriptors of the current and the next phase
+    alignas(8) uint64_t bar[DS_WARPS][DS_SLOTS];
+    alignas(8) uint64_t rec_bar[2];
+    float red[AQ_DECODE_MAX_M][DS_WARPS];
+    float scale[AQ_DECODE_MAX_M];
+    int seg_slab_lo[2][DS_MAX_PHASE_OPS];   // per op of the phase: first pair-slab staged for this CTA
+    int seg_xoff[2][DS_MAX_PHASE_OPS + 1];  // ... and where its slabs start in xs (in slabs); [op_count] = total
+    int done[32];                           // warps of this CTA that finished op (index & 31)
+    int abort_flag;
+};
+
+template <int MT, bool BF16>
+__global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArgs a) {
+    extern __shared__ __align__(128) uint8_t ds_smem_raw[];
+    DsShared& sh = *reinterpret_cast<DsShared*>(ds_smem_raw);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int M = a.M;
+
+    if (threadIdx.x < 32) sh.done[threadIdx.x] = 0;
+    if (threadIdx.x == 0) {
+        sh.abort_flag = 0;
+        ds_mbar_init(ds_smem(&sh.rec_bar[0]), 1);
+        ds_mbar_init(ds_smem(&sh.rec_bar[1]), 1);
+    }
+    if (lane == 0) {
+#pragma unroll
+        for (int s = 0; s < DS_SLOTS; ++s) ds_mbar_init(ds_smem(&sh.bar[warp][s]), 1);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    __syncthreads();
+
+    uint64_t pol, pol_keep;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
+
+    // descriptors of phase q -> rec[q & 1] (one bulk copy; waited for at the start of phase q)
+    auto fetch_record = [&](int q) {
+        const uint32_t bar = ds_smem(&sh.rec_bar[q & 1]);
+        ds_expect_tx(bar, (uint32_t)sizeof(DsPhase));
+        ds_bulk_load(ds_smem(&sh.rec[q & 1]), a.phases + q, (uint32_t)sizeof(DsPhase), bar, pol_keep);
+    };
+    if (threadIdx.x == 0) {
+        fetch_record(0);
+        if (a.n_phases > 1) fetch_record(1);
+    }
+
+    // the copy stream: `iss` runs ahead of consumption by up to DS_SLOTS units
+    DsCursor iss;
+    iss.ph = 0; iss.oi = 0; iss.wa = iss.wb = 0; iss.u = iss.u_end = 0; iss.base = nullptr; iss.ub = 0;
+    ds_seek(iss, a, warp, true);
+    uint32_t iseq = 0, cseq = 0;   // units issued / consumed by this warp
+    auto issue_next = [&]() {
+        if (iss.ph >= a.n_phases) return;
+        const uint32_t slot = iseq % DS_SLOTS;
+        if (lane == 0) {
+            const uint32_t bar = ds_smem(&sh.bar[warp][slot]);
+            ds_expect_tx(bar, (uint32_t)iss.ub);
+            ds_bulk_load(ds_smem(&sh.ring[warp][slot][0]), iss.base + (int64_t)iss.u * iss.ub, (uint32_t)iss.ub, bar, pol);
+        }
+        ++iseq;
+        if (++iss.u == iss.u_end) { ++iss.oi; ds_seek(iss, a, warp, false); }
+    };
+#pragma unroll 1
+    for (int s = 0; s < DS_SLOTS; ++s) issue_next();
+
+    bool dead = false;   // this warp gave up on a wait
+    XOperand<MT> xo;
+
+#pragma unroll 1
+    for (int ph = 0; ph < a.n_phases; ++ph) {
+        const int pb = ph & 1;
+        const DsPhase& P = sh.rec[pb];
+        {   // -- the phase's descriptors (fetched one phase ahead) --
+            if (!ds_mbar_wait(ds_smem(&sh.rec_bar[pb]), (uint32_t)(ph >> 1) & 1u)) {
+                atomicCAS(&g_decode_status, 0, 2);
+                sh.abort_flag = 1;
+            }
+        }
+        if (*reinterpret_cast<volatile int*>(&sh.abort_flag) == 0) {
+            // -- which slabs of the input this CTA's warps will read (independent of the data) --
+            if (threadIdx.x == DS_THREADS - 1) {
+                const int ca = (int)(((int64_t)P.units_total * blockIdx.x) / gridDim.x);
+                const int cb = (int)(((int64_t)P.units_total * (blockIdx.x + 1)) / gridDim.x);
+                int tot = 0;
+                for (int oi = 0; oi < P.op_count; ++oi) {
+                    const int off = P.ops[oi].unit_off, n = P.ops[oi].n_units, NT = P.ops[oi].NT;
+                    const int u0 = max(ca, off) - off, u1 = min(cb, off + n) - off;
+                    sh.seg_xoff[pb][oi] = tot;
+                    if (u0 < u1) {
+                        const int lo = u0 / NT, hi = (u1 - 1) / NT;
+                        sh.seg_slab_lo[pb][oi] = lo;
+                        tot += hi - lo + 1;
+                    } else {
+                        sh.seg_slab_lo[pb][oi] = 0;
+                    }
+                }
+                sh.seg_xoff[pb][P.op_count] = tot;
+            }
+            // -- wait for the writers of what this phase reads --
+            if ((int)threadIdx.x < P.n_deps) {
+                const uint32_t* c = a.cnt + P.deps[threadIdx.x];
+                uint32_t i = 0;
+                uint64_t t0 = 0;
+                while (ds_ld_acquire(c) < gridDim.x) {
+                    if ((++i & 63u) == 0) {   // now and then: did another CTA give up, or has this wait run out?
+                        if (*reinterpret_cast<volatile int*>(&g_decode_status) != 0) { sh.abort_flag = 1; break; }
+                        const uint64_t t = ds_now_ns();
+                        if (t0 == 0) t0 = t;
+                        if (t - t0 > DS_WAIT_NS) { atomicCAS(&g_decode_status, 0, 1); sh.abort_flag = 1; break; }
+                    }
+                    __nanosleep(20);
+                }
+            }
+        }
+        __syncthreads();
+        if (*reinterpret_cast<volatile int*>(&sh.abort_flag)) break;
+        // every warp is past phase ph - 1: its record slot is free for phase ph + 1
+        if (threadIdx.x == 0 && ph >= 1 && ph + 1 < a.n_phases) fetch_record(ph + 1);
+
+        // -- form the rounded input: RMS scale first (needs the whole row) --
+        if (P.in_op == AQ_IN_RMSNORM) {
+            for (int m = 0; m < M; ++m) {
+                const float4* s4 = reinterpret_cast<const float4*>(P.src + (int64_t)m * P.K);
+                float ss = 0.f;
+                for (int i = threadIdx.x; i < P.K / 4; i += DS_THREADS) {
+                    const float4 v = __ldcg(s4 + i);
+                    ss = fmaf(v.x, v.x, ss); ss = fmaf(v.y, v.y, ss); ss = fmaf(v.z, v.z, ss); ss = fmaf(v.w, v.w, ss);
+                }
+#pragma unroll
+                for (int d = 16; d > 0; d >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, d);
+                if (lane == 0) sh.red[m][warp] = ss;
+            }
+            __syncthreads();
+            if ((int)threadIdx.x < M) {
+                float tot = 0.f;
+#pragma unroll
+                for (int w = 0; w < DS_WARPS; ++w) tot += sh.red[threadIdx.x][w];
+                sh.scale[threadIdx.x] = rsqrtf(tot / (float)P.K + 1e-6f);
+            }
+            __syncthreads();
+        }
+        {
+            // slabs this CTA's warps read -> shared memory, laid out [slab][token][256]
+            const int n_slabs = sh.seg_xoff[pb][P.op_count];
+            const int items = n_slabs * M * 64;   // groups of 4 elements
+            for (int it = threadIdx.x; it < items; it += DS_THREADS) {
+                const int k4 = it & 63, sm_ = it >> 6, m = sm_ % M, sl = sm_ / M;
+                int oi = 0;
+                while (oi + 1 < P.op_count && sl >= sh.seg_xoff[pb][oi + 1]) ++oi;
+                const int k = (sh.seg_slab_lo[pb][oi] + sl - sh.seg_xoff[pb][oi]) * 256 + k4 * 4;
+                uint2 r = make_uint2(0u, 0u);
+                if (k < P.K) r = ds_form4<BF16>(P, m, k, P.in_op == AQ_IN_RMSNORM ? sh.scale[m] : 1.f);
+                *reinterpret_cast<uint2*>(sh.xs + (size_t)it * 4) = r;
+            }
+            // this CTA's share of the vector -> the caller's workspace
+            const int q4 = P.K / 4;
+            const int g0 = (int)(((int64_t)q4 * blockIdx.x) / gridDim.x), g1 = (int)(((int64_t)q4 * (blockIdx.x + 1)) / gridDim.x);
+            const int span = g1 - g0;
+            for (int it = threadIdx.x; it < span * M; it += DS_THREADS) {
+                const int m = it / span, k = (g0 + it - m * span) * 4;
+                const uint2 r = ds_form4<BF16>(P, m, k, P.in_op == AQ_IN_RMSNORM ? sh.scale[m] : 1.f);
+                *reinterpret_cast<uint2*>(reinterpret_cast<uint16_t*>(P.stage) + (int64_t)m * P.K + k) = r;
+            }
+        }
+        __syncthreads();
+
+        // -- consume this warp's units of the phase --
+        int wa, wb;
+        ds_warp_run(P.units_total, blockIdx.x, gridDim.x, warp, wa, wb);
+#pragma unroll 1
+        for (int oi = 0; oi < P.op_count; ++oi) {
+            const int opx = P.op_first + oi;
+            const DsOp& op = P.ops[oi];
+            const int NT = op.NT, bits = op.bits;
+            const int u0 = max(wa, op.unit_off) - op.unit_off, u1 = min(wb, op.unit_off + op.n_units) - op.unit_off;
+            if (u0 < u1 && !dead) {
+                int Pk = u0 / NT, R = u0 - Pk * NT;
+                const int xbase = sh.seg_xoff[pb][oi] - sh.seg_slab_lo[pb][oi];   // slab Pk sits at xs[(xbase + Pk) M 256]
+                ds_load_x_operand<MT, BF16>(xo, sh.xs + (xbase + Pk) * M * 256, M, lane);
+#pragma unroll 1
+                for (int u = u0; u < u1; ++u) {
+                    const uint32_t slot = cseq % DS_SLOTS, parity = (cseq / DS_SLOTS) & 1u;
+                    const uint32_t bar = ds_smem(&sh.bar[warp][slot]);
+                    dead = __any_sync(0xffffffffu, !ds_mbar_wait(bar, parity));
+                    if (dead) {
+                        if (lane == 0) { atomicCAS(&g_decode_status, 0, 2); sh.abort_flag = 1; }
+                        break;
+                    }
+                    const uint8_t* unit = &sh.ring[warp][slot][0];
+                    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+                    if (bits == 2) unit_mac<2, MT, BF16>(unit, xo, lane, acc);
+                    else if (bits == 3) unit_mac<3, MT, BF16>(unit, xo, lane, acc);
+                    else unit_mac<4, MT, BF16>(unit, xo, lane, acc);
+                    ++cseq;
+                    __syncwarp();        // every lane has read its part of the slot
+                    issue_next();        // refill it
+                    unit_commit<MT>(acc, op.dst, op.N, R * 16, op.N, M, lane, Pk == 0 ? op.res : nullptr);
+                    if (++R == NT) {
+                        R = 0; ++Pk;
+                        if (u + 1 < u1) ds_load_x_operand<MT, BF16>(xo, sh.xs + (xbase + Pk) * M * 256, M, lane);
+                    }
+                }
+            }
+            // arrive: the CTA's last warp to finish the op publishes it
+            __syncwarp();
+            if (lane == 0) {
+                if (u0 < u1) __threadfence();
+                const int old = atomicAdd(&sh.done[opx & 31], 1);
+                if (old == DS_WARPS - 1) {
+                    sh.done[opx & 31] = 0;
+                    __threadfence();
+                    atomicAdd(a.cnt + opx, 1u);
+                }
+            }
+        }
+    }
+
+    // copies still in flight into this CTA's shared memory must land before it exits
+    if (*reinterpret_cast<volatile int*>(&sh.abort_flag)) {
+        for (uint32_t s = cseq; s < iseq; ++s) {
+            const uint32_t bar = ds_smem(&sh.bar[warp][s % DS_SLOTS]);
+            ds_mbar_wait(bar, (s / DS_SLOTS) & 1u);
+        }
+        __nanosleep(100000);   // ... and a descriptor record that may still be on its way
+    }
+}
+
+// ---- host: plan, cache, launch -----------------------------------------------------
+namespace {
+
+struct DecodePlan {
+    std::vector<uint8_t> key;
+    std::vector<aq_handle_t> handles;
+    uint8_t* dev = nullptr;       // [phase records][arrival counters]
+    size_t phases_bytes = 0, cnt_bytes = 0;
+    int n_phases = 0;
+    int device = 0;
+    uint64_t stamp = 0;
+};
+
+std::mutex g_plan_mutex;
+std::vector<DecodePlan*> g_plans;
+uint64_t g_plan_clock = 0;
+constexpr size_t MAX_PLANS = 16;
+
+void drop_plan(DecodePlan* p) {
+    if (p->dev) cudaFree(p->dev);
+    delete p;
+}
+
+template <typename T> void key_put(std::vector<uint8_t>& k, const T& v) {
+    const uint8_t* b = reinterpret_cast<const uint8_t*>(&v);
+    k.insert(k.end(), b, b + sizeof(T));
+}
+
+}  // namespace
+
+// Device tables of a program: one record per phase (at most DS_MAX_PHASE_OPS ops that
+// read the same input vector).  False when the program does not fit this kernel.
+bool build_decode_tables(const aq_stack_t* p, const StackPlan& plan, int M, int n_cta, uint8_t* ws,
+                         std::vector<DsPhase>& phases) {
+    if (M < 1 || M > AQ_DECODE_MAX_M || p->n_ops > 32000) return false;
+    phases.clear();
+    std::vector<int> writer(p->n_bufs, -1);
+    std::vector<char> waited(p->n_ops, 0);
+    const int n_ph = (int)plan.phase_first.size();
+    for (int ph = 0; ph < n_ph; ++ph) {
+        const int pfirst = plan.phase_first[ph];
+        const int plast = (ph + 1 < n_ph) ? plan.phase_first[ph + 1] : p->n_ops;
+        for (int first = pfirst; first < plast; first += DS_MAX_PHASE_OPS) {
+            const int last = std::min(plast, first + DS_MAX_PHASE_OPS);
+            const aq_stack_op_t& f = p->ops[first];
+            DsPhase P;
+            memset(&P, 0, sizeof(P));
+            const int64_t K = p->buf_width[f.src];
+            if (K > (int64_t)1 << 24) return false;
+            P.src = reinterpret_cast<const float*>(ws + plan.buf_off[f.src]);
+            P.src2 = (f.in_op == AQ_IN_SILU_MUL) ? reinterpret_cast<const float*>(ws + plan.buf_off[f.src2]) : nullptr;
+            P.stage = ws + plan.in_off[first];
+            P.K = (int32_t)K; P.in_op = f.in_op; P.op_first = first; P.op_count = last - first;
+            std::vector<int> deps;
+            auto need = [&](int buf) {
+                const int w = writer[buf];
+                if (w >= 0 && !waited[w]) { waited[w] = 1; deps.push_back(w); }
+            };
+            need(f.src);
+            if (f.in_op == AQ_IN_SILU_MUL) need(f.src2);
+            int64_t off = 0;
+            for (int i = first; i < last; ++i) {
+                const aq_stack_op_t& o = p->ops[i];
+                const aq_handle_s* h = o.w;
+                DsOp& d = P.ops[i - first];
+                d.frags = h->frags;
+                d.dst = reinterpret_cast<float*>(ws + plan.buf_off[o.dst]);
+                d.res = (o.out_op == AQ_OUT_ADD) ? reinterpret_cast<const float*>(ws + plan.buf_off[o.res]) : nullptr;
+                if (o.out_op == AQ_OUT_ADD) need(o.res);
+                const int64_t nu = (int64_t)h->KP * h->NT;
+                if (off + nu > (int64_t)1 << 26) return false;
+                d.N = (int32_t)h->N; d.NT = h->NT; d.n_units = (int32_t)nu; d.unit_off = (int32_t)off; d.bits = h->bits;
+                off += nu;
+            }
+            if ((int)deps.size() > DS_MAX_DEPS) return false;
+            P.units_total = (int32_t)off;
+            P.n_deps = (int)deps.size();
+            for (size_t j = 0; j < deps.size(); ++j) P.deps[j] = (int16_t)deps[j];
+            // every CTA's staged slabs must fit the shared-memory buffer
+            for (int c = 0; c < n_cta; ++c) {
+                const int64_t ca = off * c / n_cta, cb = off * (c + 1) / n_cta;
+                int64_t slabs = 0;
+                for (int i = 0; i < P.op_count; ++i) {
+                    const int64_t o0 = P.ops[i].unit_off, n = P.ops[i].n_units;
+                    const int64_t u0 = std::max(ca, o0) - o0, u1 = std::min(cb, o0 + n) - o0;
+                    if (u0 < u1) slabs += (u1 - 1) / P.ops[i].NT - u0 / P.ops[i].NT + 1;
+                }
+                if (slabs * M * 512 > DS_XS_BYTES) return false;
+            }
+            for (int i = first; i < last; ++i) writer[p->ops[i].dst] = i;
+            phases.push_back(P);
+        }
+    }
+    return true;
+}
+
+template <int MT, bool BF16>
+static cudaError_t launch_ds(const DsArgs& a, int grid, cudaStream_t s) {
+    auto kern = decode_stack_kernel<MT, BF16>;
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DsShared));
+        if (e != cudaSuccess) return e;
+        int per_sm = 0;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, DS_THREADS, sizeof(DsShared));
+        if (e != cudaSuccess) return e;
+        if (per_sm < 1) return cudaErrorCooperativeLaunchTooLarge;
+        configured = true;
+    }
+    DsArgs args = a;
+    void* params[1] = {&args};
+    cudaError_t e = cudaLaunchCooperativeKernel(reinterpret_cast<void*>(kern), dim3((unsigned)grid), dim3(DS_THREADS), params,
+                                                sizeof(DsShared), s);
+    if (e == cudaSuccess) count_launch();
+    return e;
+}
+
+int launch_decode_stack(const aq_stack_t* p, const StackPlan& plan, int M, aq_dtype_t dt, uint8_t* ws, cudaStream_t s,
+                        cudaError_t* err) {
+    *err = cudaSuccess;
+    const int grid = sm_count();
+    int dev = 0;
+    cudaGetDevice(&dev);
+    // key: everything the device tables are computed from
+    std::vector<uint8_t> key;
+    key_put(key, M); key_put(key, dev); key_put(key, grid); key_put(key, ws);
+    key_put(key, p->n_ops); key_put(key, p->n_bufs);
+    for (int i = 0; i < p->n_ops; ++i) {
+        key_put(key, p->ops[i]);
+        key_put(key, p->ops[i].w->frags);
+    }
+    for (int b = 0; b < p->n_bufs; ++b) key_put(key, p->buf_width[b]);
+
+    std::lock_guard<std::mutex> lock(g_plan_mutex);
+    DecodePlan* dp = nullptr;
+    for (DecodePlan* q : g_plans)
+        if (q->key == key) { dp = q; break; }
+    if (!dp) {
+        std::vector<DsPhase> phases;
+        if (!build_decode_tables(p, plan, M, grid, ws, phases)) return 1;
+        dp = new DecodePlan();
+        dp->key = key;
+        dp->device = dev;
+        for (int i = 0; i < p->n_ops; ++i) dp->handles.push_back(p->ops[i].w);
+        dp->phases_bytes = (phases.size() * sizeof(DsPhase) + 255) / 256 * 256;
+        dp->cnt_bytes = ((size_t)p->n_ops * sizeof(uint32_t) + 255) / 256 * 256;
+        dp->n_phases = (int)phases.size();
+        cudaError_t e = cudaMalloc(&dp->dev, dp->phases_bytes + dp->cnt_bytes);
+        if (e == cudaSuccess) e = cudaMemcpy(dp->dev, phases.data(), phases.size() * sizeof(DsPhase), cudaMemcpyHostToDevice);
+        if (e != cudaSuccess) { cudaGetLastError(); drop_plan(dp); *err = e; return -1; }
+        if (g_plans.size() >= MAX_PLANS) {
+            size_t oldest = 0;
+            for (size_t i = 1; i < g_plans.size(); ++i)
+                if (g_plans[i]->stamp < g_plans[oldest]->stamp) oldest = i;
+            drop_plan(g_plans[oldest]);
+            g_plans.erase(g_plans.begin() + oldest);
+        }
+        g_plans.push_back(dp);
+    }
+    dp->stamp = ++g_plan_clock;
+
+    DsArgs a;
+    a.phases = reinterpret_cast<const DsPhase*>(dp->dev);
+    a.cnt = reinterpret_cast<uint32_t*>(dp->dev + dp->phases_bytes);
+    a.n_phases = dp->n_phases;
+    a.M = M;
+    cudaError_t e = cudaMemsetAsync(a.cnt, 0, dp->cnt_bytes, s);
+    if (e == cudaSuccess) {
+        const bool bf = (dt == AQ_BF16);
+        if (M <= 2) e = bf ? launch_ds<2, true>(a, grid, s) : launch_ds<2, false>(a, grid, s);
+        else if (M <= 4) e = bf ? launch_ds<4, true>(a, grid, s) : launch_ds<4, false>(a, grid, s);
+        else e = bf ? launch_ds<8, true>(a, grid, s) : launch_ds<8, false>(a, grid, s);
+    }
+    if (e != cudaSuccess) { *err = e; return -1; }
+    return 0;
+}
+
+void decode_stack_forget(aq_handle_t h) {
+    std::lock_guard<std::mutex> lock(g_plan_mutex);
+    for (size_t i = 0; i < g_plans.size();) {
+        bool uses = false;
+        for (aq_handle_t x : g_plans[i]->handles)
+            if (x == h) { uses = true; break; }
+        if (uses) { drop_plan(g_plans[i]); g_plans.erase(g_plans.begin() + i); }
+        else ++i;
+    }
+}
+
+int read_decode_status(bool clear) {
+    int v = 0;
+    cudaMemcpyFromSymbol(&v, g_decode_status, sizeof(int));
+    if (clear && v) { int z = 0; cudaMemcpyToSymbol(g_decode_status, &z, sizeof(int)); }
+    return v;
+}
+
+}  // namespace aq

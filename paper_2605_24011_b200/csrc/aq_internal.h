@@ -2,6 +2,9 @@
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
+
+#include <vector>
+
 #include "../../include/aq.h"
 
 #define AQ_HANDLE_MAGIC 0x41514831u   /* "AQH1" */
@@ -43,6 +46,22 @@ cudaError_t launch_finalize(const float* acc_in, float* acc_zero, int64_t ldacc,
 // prefill path: out[m][n] (+)= sum_k x[m][k] w[n][k]; out fp32 [M][ldo]
 cudaError_t launch_gemm(const aq_handle_s* h, const void* x, aq_dtype_t xdt, int M, float* out,
                         int64_t ldo, bool accumulate, cudaStream_t s);
+
+// Where a program's buffers and staged inputs sit in the caller's workspace (aq_stack.cu).
+struct StackPlan {
+    std::vector<size_t> buf_off;    // per buffer: float32 [M][width]
+    std::vector<size_t> in_off;     // per op: its phase's staged input [M][K] (activation dtype)
+    std::vector<int> phase_first;   // first op of each phase (ops that share one input vector)
+    size_t stage_off = 0;           // end of the float32 buffers
+    size_t total = 0;
+};
+
+// whole-program decode (M <= AQ_DECODE_MAX_M) in one persistent kernel: 0 = launched,
+// 1 = the program does not fit that kernel (nothing launched), -1 = CUDA error in *err
+int launch_decode_stack(const aq_stack_t* p, const StackPlan& plan, int M, aq_dtype_t dt, uint8_t* ws, cudaStream_t s,
+                        cudaError_t* err);
+void decode_stack_forget(aq_handle_t h);   // drops cached device tables that name h
+int read_decode_status(bool clear);        // nonzero: a bounded wait in the decode-stack kernel ran out
 
 int sm_count();
 void count_launch(int n = 1);       // process-wide count of this library's kernel launches

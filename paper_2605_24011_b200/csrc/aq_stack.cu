@@ -17,14 +17,6 @@ namespace aq {
 
 static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-struct StackPlan {
-    std::vector<size_t> buf_off;
-    std::vector<size_t> in_off;     // per op: its phase's staged input [M][K] (activation dtype)
-    std::vector<int> phase_first;   // first op of each phase
-    size_t stage_off = 0;           // end of the float32 buffers
-    size_t total = 0;
-};
-
 static inline bool same_input(const aq_stack_op_t& a, const aq_stack_op_t& b) {
     return a.src == b.src && a.in_op == b.in_op && (a.in_op != AQ_IN_SILU_MUL || a.src2 == b.src2);
 }
@@ -136,6 +128,19 @@ static cudaError_t run_stack(const aq_stack_t* p, const StackPlan& plan, const T
         const int64_t n = (int64_t)M * p->buf_width[0];
         widen_kernel<T><<<(unsigned)((n + 255) / 256), 256, 0, s>>>(x0, buf(0), n);
         count_launch();
+    }
+    if (decode) {   // one persistent kernel for the whole program, when it fits
+        const int r = launch_decode_stack(p, plan, M, dt, ws, s, &e);
+        if (r < 0) return e;
+        if (r == 0) {
+            for (int k = 0; k < p->n_ops; ++k) p->ops[k].w->last_stream = s;
+        }
+        if (r == 0 && out) {
+            const int64_t n = (int64_t)M * p->buf_width[out_buf];
+            narrow_kernel<T><<<(unsigned)((n + 255) / 256), 256, 0, s>>>(buf(out_buf), out, n);
+            count_launch();
+        }
+        if (r == 0) return cudaGetLastError();
     }
     int i = 0;
     while (i < p->n_ops) {
