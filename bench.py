@@ -154,6 +154,58 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def run_micro(args):
+    """One kernel, small case, a few launches: what the ncu captures under profiles/ run."""
+    import torch
+    from paper_2605_24011_b200 import aq, synth, workloads
+    torch.cuda.set_device(0)
+    out = {"micro": args.micro, "bits": args.bits, "steps": args.steps, "warmup": args.warmup}
+    if args.micro in ("decode_linear", "prefill_linear", "dequant"):
+        decode = args.micro == "decode_linear"
+        M = args.M or (1 if decode else 512)
+        N = args.N or (65536 if decode else 11008)
+        K = args.K or (8192 if decode else 4096)
+        dt = torch.float16 if decode else torch.bfloat16
+        n_copies = 1 if decode else max(1, int(400e6 // (N * K * (args.bits + 1) // 8)))   # rotate past L2
+        W = synth.weights_device(N, K, 7)
+        hs = [aq.aq_pack(args.bits, 32, W) for _ in range(n_copies)]
+        del W
+        x = workloads.activations_device(M, K, dt, 9, M)
+        if args.micro == "dequant":
+            y = torch.empty((N, K), dtype=torch.float16, device="cuda")
+            fn = lambda i: aq.aq_dequant(hs[i % n_copies], y)
+            work, unit = N * K * (args.bits + 1) / 8 + 2.0 * N * K, "GB/s"
+        else:
+            y = torch.empty((M, N), dtype=torch.float32, device="cuda")
+            fn = lambda i: aq.aq_linear(hs[i % n_copies], x, y)
+            work, unit = (N * K * (args.bits + 1) / 8, "GB/s") if decode else (2.0 * M * N * K, "TFLOP/s")
+        out.update({"M": M, "N": N, "K": K, "copies": n_copies})
+    else:
+        decode = args.micro == "decode_stack"
+        M = args.M or (1 if decode else 512)
+        prog, out_buf, names, _, info = workloads.llama7b_decode_stack(n_layers=args.layers, seed=0)
+        ws = torch.empty(prog.workspace_bytes(M), dtype=torch.uint8, device="cuda")
+        dt = torch.float16 if decode else torch.bfloat16
+        x0 = workloads.activations_device(M, 4096, dt, 3, 0)
+        y = torch.empty((M, 4096), dtype=dt, device="cuda")
+        fn = lambda i: aq.aq_stack_forward(prog, x0, y, out_buf, M, ws)
+        work, unit = (info["packed_bytes"], "GB/s") if decode else (2.0 * M * info["weights"], "TFLOP/s")
+        out.update({"M": M, "layers": args.layers})
+    for i in range(args.warmup):
+        fn(i)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.steps):
+        fn(args.warmup + i)
+    e1.record()
+    torch.cuda.synchronize()
+    aq.aq_check()
+    ms = e0.elapsed_time(e1) / args.steps
+    out.update({"us_per_call": 1e3 * ms, "value": work / (ms * 1e-3) / (1e9 if unit == "GB/s" else 1e12), "unit": unit})
+    print(json.dumps(out))
+
+
 WORKLOAD = ("7B-class decoder linear stack, M=1 decode: 32 layers x {q,k,v,o 4096x4096; gate,up 11008x4096; "
             "down 4096x11008}, per-matrix 2/3/4-bit (mean 2.5), blocks of 32 + fp16 scale/min, N(0,0.02) weights "
             "with 0.1% x20 outliers, x fp16 N(0,1)")
@@ -167,9 +219,18 @@ def main():
     ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
     ap.add_argument("--layers", type=int, default=32, help="decoder layers (32 = the full workload)")
     ap.add_argument("--no-extras", action="store_true", help="skip prefill / dequant / oracle legs")
+    ap.add_argument("--micro", choices=("decode_linear", "prefill_linear", "dequant", "decode_stack", "prefill_stack"),
+                    help="time one kernel on a small case (the command ncu captures are taken from) instead of the benchmark")
+    ap.add_argument("--bits", type=int, default=2)
+    ap.add_argument("--M", type=int, default=None)
+    ap.add_argument("--N", type=int, default=None)
+    ap.add_argument("--K", type=int, default=None)
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.micro:
+        run_micro(args)
         return
 
     import numpy as np

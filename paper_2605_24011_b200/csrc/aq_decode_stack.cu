@@ -8,11 +8,12 @@
 //
 //   * Work.  Consecutive ops that read the same input vector form a phase.
 //     The units (16 rows x 256 k) of a phase's matrices are concatenated and
-//     dealt as contiguous runs: first to CTAs, then to the warps of a CTA.
+//     dealt as contiguous runs: first to CTAs, then to the 15 consumer warps
+//     of a CTA.
 //   * Weight stream.  Which bytes a warp will need does not depend on any
-//     activation, so every warp keeps a private ring of bulk copies
-//     (cp.async.bulk + mbarrier, L2 evict-first) running ahead of what it
-//     consumes, across op and phase boundaries.
+//     activation, so a 16th warp (lane w serves consumer warp w) keeps every
+//     consumer's private ring of bulk copies (cp.async.bulk + mbarrier, L2
+//     evict-first) full, running ahead across op and phase boundaries.
 //   * Dependencies.  Sums leave the warps as fp32 red.add into the output
 //     buffer.  Every op has an arrival counter in global memory; a CTA arrives
 //     once all its warps have committed their share of the op.  Before a phase
@@ -21,14 +22,18 @@
 //     attention block) therefore overlap the wait of the ops that follow.
 //   * Glue.  At the start of a phase each CTA forms, in shared memory, the
 //     rounded input vector for the k-slabs its warps will touch (RMS scaling /
-//     SiLU(g)*u / plain), and writes its share of the vector to the caller's
-//     workspace, where every op's input stays readable after the call.
+//     SiLU(g)*u / plain) with one round trip to L2, and writes its share of the
+//     vector to the caller's workspace, where every op's input stays readable.
+//     For one token the vector is stored already spread out as the B operand of
+//     the tensor-core instruction (non-zero only in the column of its block),
+//     so a warp picks its operand up with eight 16-byte loads.
 //
 // Every wait is bounded: when one runs out the kernel raises a status word,
-// waits (bounded) for its own copies in flight and returns.
+// gives copies in flight time to land and returns.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
+#include <algorithm>
 #include <cstring>
 #include <mutex>
 #include <vector>
@@ -38,14 +43,21 @@
 
 namespace aq {
 
-constexpr int DS_WARPS = 16;
-constexpr int DS_THREADS = DS_WARPS * 32;
+constexpr int DS_WARPS = 15;                // consumer warps (+ the copy warp = 4 warps per scheduler, 128 registers each)
+constexpr int DS_CTHREADS = DS_WARPS * 32;  // consumer threads
+constexpr int DS_THREADS = DS_CTHREADS + 32;   // + the copy warp
 constexpr int DS_SLOTS = 5;                 // ring depth per warp (units)
 constexpr int DS_SLOT_BYTES = 2560;         // the largest unit (4-bit: 2 fragments of 1280 B)
-constexpr int DS_XS_BYTES = 16384;          // staged input: tokens x slabs <= 32 (a slab = 256 k = 512 B per token)
+constexpr int DS_XS_BYTES = 6 * 4128;       // staged input: six one-token slabs (see ds_slab_bytes)
 constexpr int DS_MAX_PHASE_OPS = 8;
 constexpr int DS_MAX_DEPS = 12;
+constexpr int DS_RMS_HOLD = 4;              // float4 per thread kept in registers by the one-token RMS path
 constexpr uint64_t DS_WAIT_NS = 2000000000ull;   // every wait gives up after two seconds
+
+// Shared-memory bytes of one staged slab (256 k): one token is stored spread out
+// as B operands (32 lanes x 8 blocks x 16 B) plus 8 block sums; several tokens
+// are stored plainly, [token][256] halves.
+__host__ __device__ constexpr int ds_slab_bytes(int M) { return M == 1 ? 4096 + 32 : M * 512; }
 
 __device__ int g_decode_status = 0;   // nonzero: a bounded wait ran out (1 = counter, 2 = copy)
 
@@ -72,7 +84,7 @@ struct DsPhase {
     int32_t units_total;
     int32_t n_deps;
     int16_t deps[DS_MAX_DEPS];   // ops that must be complete before this phase reads its inputs
-    int32_t pad_[2];
+    int32_t units_q, units_r;    // units_total = units_q * (number of CTAs) + units_r
     DsOp ops[DS_MAX_PHASE_OPS];
 };
 static_assert(sizeof(DsOp) == 48, "DsOp layout");
@@ -90,6 +102,9 @@ __device__ __forceinline__ uint32_t ds_smem(const void* p) { return (uint32_t)__
 __device__ __forceinline__ void ds_mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
+__device__ __forceinline__ void ds_mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
 __device__ __forceinline__ void ds_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
@@ -98,6 +113,15 @@ __device__ __forceinline__ bool ds_mbar_try(uint32_t bar, uint32_t parity) {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool ds_mbar_test(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
@@ -128,6 +152,8 @@ __device__ __forceinline__ uint32_t ds_ld_acquire(const uint32_t* p) {
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
+// Barrier among the consumer warps only (the copy warp never joins).
+__device__ __forceinline__ void ds_consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(DS_CTHREADS) : "memory"); }
 
 // ---- the warp's position in its stream of units ---------------------------------
 struct DsCursor {
@@ -139,12 +165,19 @@ struct DsCursor {
     int ub;                // bytes per unit
 };
 
-// The run of units warp `warp` of CTA `cta` owns in a phase of `total` units.
-__device__ __forceinline__ void ds_warp_run(int total, int cta, int ncta, int warp, int& wa, int& wb) {
-    const int a = (int)(((int64_t)total * cta) / ncta), b = (int)(((int64_t)total * (cta + 1)) / ncta);
+// The run of units CTA `cta` owns in a phase of q * (number of CTAs) + r units:
+// the first r CTAs take q + 1 units, the others q.
+__device__ __forceinline__ void ds_cta_run(int q, int r, int cta, int& a, int& b) {
+    a = q * cta + min(cta, r);
+    b = a + q + (cta < r ? 1 : 0);
+}
+// ... and the run of one of its warps.
+__device__ __forceinline__ void ds_warp_run(int q, int r, int cta, int warp, int& wa, int& wb) {
+    int a, b;
+    ds_cta_run(q, r, cta, a, b);
     const int n = b - a;
-    wa = a + (int)(((int64_t)n * warp) / DS_WARPS);
-    wb = a + (int)(((int64_t)n * (warp + 1)) / DS_WARPS);
+    wa = a + (n * warp) / DS_WARPS;
+    wb = a + (n * (warp + 1)) / DS_WARPS;
 }
 
 // Moves the cursor to the next op (from (ph, oi) on) in which the warp owns units.
@@ -152,7 +185,7 @@ __device__ __forceinline__ void ds_seek(DsCursor& c, const DsArgs& a, int warp, 
     while (c.ph < a.n_phases) {
         const DsPhase* P = a.phases + c.ph;
         if (new_phase) {
-            ds_warp_run(__ldg(&P->units_total), blockIdx.x, gridDim.x, warp, c.wa, c.wb);
+            ds_warp_run(__ldg(&P->units_q), __ldg(&P->units_r), blockIdx.x, warp, c.wa, c.wb);
             c.oi = 0;
             new_phase = false;
         }
@@ -177,70 +210,41 @@ __device__ __forceinline__ void ds_seek(DsCursor& c, const DsArgs& a, int warp, 
 // ---- glue arithmetic --------------------------------------------------------------
 __device__ __forceinline__ float ds_silu_mul(float g, float u) { return g / (1.f + expf(-g)) * u; }
 
+// Rounds four values to the activation dtype; *sum gets the sum of the rounded values.
 template <bool BF16>
-__device__ __forceinline__ uint2 ds_round4(const float4& v) {
+__device__ __forceinline__ uint2 ds_round4(const float4& v, float* sum) {
     uint2 r;
     if constexpr (BF16) {
         __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y), b = __floats2bfloat162_rn(v.z, v.w);
         r.x = *reinterpret_cast<uint32_t*>(&a); r.y = *reinterpret_cast<uint32_t*>(&b);
+        const float2 fa = __bfloat1622float2(a), fb = __bfloat1622float2(b);
+        *sum = (fa.x + fa.y) + (fb.x + fb.y);
     } else {
         __half2 a = __floats2half2_rn(v.x, v.y), b = __floats2half2_rn(v.z, v.w);
         r.x = *reinterpret_cast<uint32_t*>(&a); r.y = *reinterpret_cast<uint32_t*>(&b);
+        const float2 fa = __half22float2(a), fb = __half22float2(b);
+        *sum = (fa.x + fa.y) + (fb.x + fb.y);
     }
     return r;
 }
 
-// Four consecutive elements of the rounded input vector of token m at k (k % 4 == 0, k < K).
-template <bool BF16>
-__device__ __forceinline__ uint2 ds_form4(const DsPhase& P, int m, int k, float scale) {
-    const float4 s = *reinterpret_cast<const float4*>(P.src + (int64_t)m * P.K + k);
-    float4 v;
+// Four consecutive elements of the input vector of token m at k (k % 4 == 0, k < K), before rounding.
+__device__ __forceinline__ float4 ds_form4(const DsPhase& P, int m, int k, float scale) {
+    const float4 s = __ldcg(reinterpret_cast<const float4*>(P.src + (int64_t)m * P.K + k));
     if (P.in_op == AQ_IN_SILU_MUL) {
-        const float4 t = *reinterpret_cast<const float4*>(P.src2 + (int64_t)m * P.K + k);
-        v = make_float4(ds_silu_mul(s.x, t.x), ds_silu_mul(s.y, t.y), ds_silu_mul(s.z, t.z), ds_silu_mul(s.w, t.w));
-    } else {
-        v = make_float4(s.x * scale, s.y * scale, s.z * scale, s.w * scale);
+        const float4 t = __ldcg(reinterpret_cast<const float4*>(P.src2 + (int64_t)m * P.K + k));
+        return make_float4(ds_silu_mul(s.x, t.x), ds_silu_mul(s.y, t.y), ds_silu_mul(s.z, t.z), ds_silu_mul(s.w, t.w));
     }
-    return ds_round4<BF16>(v);
+    return make_float4(s.x * scale, s.y * scale, s.z * scale, s.w * scale);
 }
 
-// The x operand of pair-slab P from the staged vector in shared memory:
-// xs points at [slab - slab_lo][M][256] halves of the op's segment.
-template <int MT, bool BF16>
-__device__ __forceinline__ void ds_load_x_operand(XOperand<MT>& xo, const uint16_t* xs, int M, int lane) {
-    constexpr int BG = XOperand<MT>::BG, NG = XOperand<MT>::NG;
-    const int g = lane >> 2, t = lane & 3;
-    const int tok = g % MT, bs = g / MT;
-#pragma unroll
-    for (int fi = 0; fi < 2; ++fi) {
-#pragma unroll
-        for (int gi = 0; gi < NG; ++gi) {
-            const int jb = gi * BG + bs;
-            uint4 v = make_uint4(0, 0, 0, 0);
-            if (tok < M) v = *reinterpret_cast<const uint4*>(xs + tok * 256 + fi * 128 + 32 * jb + 8 * t);
-            float s = sum8<BF16>(v);
-            s += __shfl_xor_sync(0xffffffffu, s, 1);
-            s += __shfl_xor_sync(0xffffffffu, s, 2);
-            xo.X0[fi][gi] = __shfl_sync(0xffffffffu, s, (2 * t) * 4);
-            xo.X1[fi][gi] = __shfl_sync(0xffffffffu, s, (2 * t + 1) * 4);
-#pragma unroll
-            for (int b2 = 0; b2 < BG; ++b2) {
-                const bool on = (b2 == bs);
-                xo.b[fi][gi * BG + b2][0] = on ? v.x : 0u;
-                xo.b[fi][gi * BG + b2][1] = on ? v.y : 0u;
-                xo.b[fi][gi * BG + b2][2] = on ? v.z : 0u;
-                xo.b[fi][gi * BG + b2][3] = on ? v.w : 0u;
-            }
-        }
-    }
-}
-
-// ---- the kernel ---------------------------------------------------------------------
+// ---- shared memory ------------------------------------------------------------------
 struct DsShared {
     alignas(128) uint8_t ring[DS_WARPS][DS_SLOTS][DS_SLOT_BYTES];
-    alignas(16) uint16_t xs[DS_XS_BYTES / 2];
+    alignas(128) uint8_t xs[DS_XS_BYTES];   // staged input slabs
     alignas(16) DsPhase rec[2];             // descriptors of the current and the next phase
-    alignas(8) uint64_t bar[DS_WARPS][DS_SLOTS];
+    alignas(8) uint64_t full[DS_WARPS][DS_SLOTS];    // copy landed
+    alignas(8) uint64_t empty[DS_WARPS][DS_SLOTS];   // consumer has read the slot
     alignas(8) uint64_t rec_bar[2];
     float red[AQ_DECODE_MAX_M][DS_WARPS];
     float scale[AQ_DECODE_MAX_M];
@@ -250,12 +254,51 @@ struct DsShared {
     int abort_flag;
 };
 
+// Where the 16-byte chunk (block bk, quarter t) of a one-token slab lives: in the
+// row of the lane (bk, t) that multiplies it, at a position rotated by the lane
+// so that the eight chunks a lane reads never collide on a bank.
+__device__ __forceinline__ int ds_spread_offset(int lane, int bk) { return lane * 128 + ((bk ^ (lane & 7)) * 16); }
+
+// Writes 4 rounded elements (k .. k+3 of slab-local index) of the staged vector.
+template <int MT>
+__device__ __forceinline__ void ds_store4(uint8_t* slab, int M, int m, int kl, uint2 r) {
+    if constexpr (MT == 1) {
+        const int bk = kl >> 5, t = (kl >> 3) & 3;
+        *reinterpret_cast<uint2*>(slab + ds_spread_offset(bk * 4 + t, bk) + (kl & 7) * 2) = r;
+    } else {
+        *reinterpret_cast<uint2*>(slab + ((size_t)m * 256 + kl) * 2) = r;
+    }
+}
+
+// The x operand of one pair-slab from its staged copy in shared memory.
+template <int MT, bool BF16>
+__device__ __forceinline__ void ds_load_x_operand(XOperand<MT>& xo, const uint8_t* slab, int M, int lane) {
+    if constexpr (MT == 1) {
+#pragma unroll
+        for (int bk = 0; bk < 8; ++bk) {
+            const uint4 v = *reinterpret_cast<const uint4*>(slab + ds_spread_offset(lane, bk));
+            xo.b[bk][0] = v.x; xo.b[bk][1] = v.y; xo.b[bk][2] = v.z; xo.b[bk][3] = v.w;
+        }
+        const float2 xs = *reinterpret_cast<const float2*>(slab + 4096 + (lane & 3) * 8);
+        xo.X0[0] = xs.x; xo.X1[0] = xs.y;
+    } else {
+        const uint16_t* x = reinterpret_cast<const uint16_t*>(slab);
+        fill_x_operand<MT, BF16>(xo, lane, [&](int tok, int kk) {
+            uint4 v = make_uint4(0, 0, 0, 0);
+            if (tok < M) v = *reinterpret_cast<const uint4*>(x + tok * 256 + kk);
+            return v;
+        });
+    }
+}
+
+// ---- the kernel ---------------------------------------------------------------------
 template <int MT, bool BF16>
 __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArgs a) {
     extern __shared__ __align__(128) uint8_t ds_smem_raw[];
     DsShared& sh = *reinterpret_cast<DsShared*>(ds_smem_raw);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int M = a.M;
+    const int slab_bytes = ds_slab_bytes(M);
 
     if (threadIdx.x < 32) sh.done[threadIdx.x] = 0;
     if (threadIdx.x == 0) {
@@ -263,10 +306,16 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArg
         ds_mbar_init(ds_smem(&sh.rec_bar[0]), 1);
         ds_mbar_init(ds_smem(&sh.rec_bar[1]), 1);
     }
-    if (lane == 0) {
+    if (warp < DS_WARPS && lane == 0) {
 #pragma unroll
-        for (int s = 0; s < DS_SLOTS; ++s) ds_mbar_init(ds_smem(&sh.bar[warp][s]), 1);
+        for (int s = 0; s < DS_SLOTS; ++s) {
+            ds_mbar_init(ds_smem(&sh.full[warp][s]), 1);
+            ds_mbar_init(ds_smem(&sh.empty[warp][s]), 1);
+        }
     }
+    // one-token slabs keep zeros everywhere but in the chunks the stagers rewrite every phase
+    for (int i = threadIdx.x; i < DS_XS_BYTES / 16; i += DS_THREADS)
+        reinterpret_cast<uint4*>(sh.xs)[i] = make_uint4(0, 0, 0, 0);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     __syncthreads();
 
@@ -274,7 +323,43 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArg
     asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
     asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
 
-    // descriptors of phase q -> rec[q & 1] (one bulk copy; waited for at the start of phase q)
+    if (warp == DS_WARPS) {
+        // ================= the copy warp: lane w keeps consumer warp w's ring full =================
+        DsCursor c;
+        c.ph = a.n_phases; c.oi = 0; c.wa = c.wb = 0; c.u = c.u_end = 0; c.base = nullptr; c.ub = 0;
+        if (lane < DS_WARPS) { c.ph = 0; ds_seek(c, a, lane, true); }
+        uint32_t iseq = 0;   // copies issued for this consumer
+        uint64_t t_progress = ds_now_ns();
+        uint32_t idle = 0;
+        for (;;) {
+            const bool active = c.ph < a.n_phases;
+            bool moved = false;
+            if (active) {
+                // the n-th copy into a slot (n >= 1) waits for the consumer's arrival after its (n-1)-th read
+                const uint32_t slot = iseq % DS_SLOTS, n = iseq / DS_SLOTS;
+                const bool is_free = (n == 0) || ds_mbar_test(ds_smem(&sh.empty[lane][slot]), (n - 1) & 1u);
+                if (is_free) {
+                    const uint32_t bar = ds_smem(&sh.full[lane][slot]);
+                    ds_expect_tx(bar, (uint32_t)c.ub);
+                    ds_bulk_load(ds_smem(&sh.ring[lane][slot][0]), c.base + (int64_t)c.u * c.ub, (uint32_t)c.ub, bar, pol);
+                    ++iseq;
+                    if (++c.u == c.u_end) { ++c.oi; ds_seek(c, a, lane, false); }
+                    moved = true;
+                }
+            }
+            if (!__any_sync(0xffffffffu, active)) break;
+            if (__any_sync(0xffffffffu, moved)) { idle = 0; continue; }
+            if ((++idle & 255u) == 0) {   // nothing to do for a while: stop if the CTA gave up, or after the time limit
+                if (*reinterpret_cast<volatile int*>(&sh.abort_flag)) break;
+                const uint64_t t = ds_now_ns();
+                if (idle == 256u) t_progress = t;
+                else if (t - t_progress > 2 * DS_WAIT_NS) { atomicCAS(&g_decode_status, 0, 2); sh.abort_flag = 1; break; }
+            }
+        }
+        return;
+    }
+
+    // ================= consumer warps =================
     auto fetch_record = [&](int q) {
         const uint32_t bar = ds_smem(&sh.rec_bar[q & 1]);
         ds_expect_tx(bar, (uint32_t)sizeof(DsPhase));
@@ -285,43 +370,24 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArg
         if (a.n_phases > 1) fetch_record(1);
     }
 
-    // the copy stream: `iss` runs ahead of consumption by up to DS_SLOTS units
-    DsCursor iss;
-    iss.ph = 0; iss.oi = 0; iss.wa = iss.wb = 0; iss.u = iss.u_end = 0; iss.base = nullptr; iss.ub = 0;
-    ds_seek(iss, a, warp, true);
-    uint32_t iseq = 0, cseq = 0;   // units issued / consumed by this warp
-    auto issue_next = [&]() {
-        if (iss.ph >= a.n_phases) return;
-        const uint32_t slot = iseq % DS_SLOTS;
-        if (lane == 0) {
-            const uint32_t bar = ds_smem(&sh.bar[warp][slot]);
-            ds_expect_tx(bar, (uint32_t)iss.ub);
-            ds_bulk_load(ds_smem(&sh.ring[warp][slot][0]), iss.base + (int64_t)iss.u * iss.ub, (uint32_t)iss.ub, bar, pol);
-        }
-        ++iseq;
-        if (++iss.u == iss.u_end) { ++iss.oi; ds_seek(iss, a, warp, false); }
-    };
-#pragma unroll 1
-    for (int s = 0; s < DS_SLOTS; ++s) issue_next();
-
-    bool dead = false;   // this warp gave up on a wait
+    uint32_t cslot = 0, cparity = 0;   // next ring slot to consume and the parity of its `full` barrier
+    bool dead = false;                 // this warp gave up on a wait
     XOperand<MT> xo;
 
 #pragma unroll 1
     for (int ph = 0; ph < a.n_phases; ++ph) {
         const int pb = ph & 1;
         const DsPhase& P = sh.rec[pb];
-        {   // -- the phase's descriptors (fetched one phase ahead) --
-            if (!ds_mbar_wait(ds_smem(&sh.rec_bar[pb]), (uint32_t)(ph >> 1) & 1u)) {
-                atomicCAS(&g_decode_status, 0, 2);
-                sh.abort_flag = 1;
-            }
+        // -- the phase's descriptors (fetched one phase ahead) --
+        if (!ds_mbar_wait(ds_smem(&sh.rec_bar[pb]), (uint32_t)(ph >> 1) & 1u)) {
+            atomicCAS(&g_decode_status, 0, 2);
+            sh.abort_flag = 1;
         }
         if (*reinterpret_cast<volatile int*>(&sh.abort_flag) == 0) {
             // -- which slabs of the input this CTA's warps will read (independent of the data) --
-            if (threadIdx.x == DS_THREADS - 1) {
-                const int ca = (int)(((int64_t)P.units_total * blockIdx.x) / gridDim.x);
-                const int cb = (int)(((int64_t)P.units_total * (blockIdx.x + 1)) / gridDim.x);
+            if (threadIdx.x == DS_CTHREADS - 1) {
+                int ca, cb;
+                ds_cta_run(P.units_q, P.units_r, blockIdx.x, ca, cb);
                 int tot = 0;
                 for (int oi = 0; oi < P.op_count; ++oi) {
                     const int off = P.ops[oi].unit_off, n = P.ops[oi].n_units, NT = P.ops[oi].NT;
@@ -349,65 +415,132 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArg
                         if (t0 == 0) t0 = t;
                         if (t - t0 > DS_WAIT_NS) { atomicCAS(&g_decode_status, 0, 1); sh.abort_flag = 1; break; }
                     }
-                    __nanosleep(20);
                 }
             }
         }
-        __syncthreads();
+        ds_consumer_sync();
         if (*reinterpret_cast<volatile int*>(&sh.abort_flag)) break;
         // every warp is past phase ph - 1: its record slot is free for phase ph + 1
         if (threadIdx.x == 0 && ph >= 1 && ph + 1 < a.n_phases) fetch_record(ph + 1);
 
-        // -- form the rounded input: RMS scale first (needs the whole row) --
-        if (P.in_op == AQ_IN_RMSNORM) {
-            for (int m = 0; m < M; ++m) {
-                const float4* s4 = reinterpret_cast<const float4*>(P.src + (int64_t)m * P.K);
+        // -- form the rounded input vector: slabs this CTA reads -> shared memory, its share -> workspace --
+        {
+            const int n_slabs = sh.seg_xoff[pb][P.op_count];
+            const int q4 = P.K >> 2;                                  // groups of 4 elements per token
+            const int g0 = (int)(((int64_t)q4 * blockIdx.x) / gridDim.x), g1 = (int)(((int64_t)q4 * (blockIdx.x + 1)) / gridDim.x);
+            uint16_t* rec_out = reinterpret_cast<uint16_t*>(P.stage);
+            // stores group i4 (elements 4 i4 ..) of token m where it is needed; whole warps call this together
+            auto place = [&](int m, int i4, float4 v, bool valid, bool with_record) {
+                float sum;
+                const uint2 r = ds_round4<BF16>(v, &sum);   // v is zero past the end of the row: padding stages zeros
+                if constexpr (MT == 1) {   // block sums: 8 consecutive groups = 8 consecutive lanes
+                    sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+                    sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+                    sum += __shfl_xor_sync(0xffffffffu, sum, 4);
+                }
+                const int k = i4 * 4, slab = k >> 8, kl = k & 255;
+                for (int oi = 0; oi < P.op_count; ++oi) {
+                    const int lo = sh.seg_slab_lo[pb][oi], xo0 = sh.seg_xoff[pb][oi], n = sh.seg_xoff[pb][oi + 1] - xo0;
+                    if (slab >= lo && slab < lo + n) {
+                        uint8_t* sl = sh.xs + (size_t)(xo0 + slab - lo) * slab_bytes;
+                        ds_store4<MT>(sl, M, m, kl, r);
+                        if constexpr (MT == 1) {
+                            if ((lane & 7) == 0) *reinterpret_cast<float*>(sl + 4096 + (kl >> 5) * 4) = sum;
+                        }
+                    }
+                }
+                if (with_record && valid && i4 >= g0 && i4 < g1) *reinterpret_cast<uint2*>(rec_out + (int64_t)m * P.K + k) = r;
+            };
+            if (P.in_op == AQ_IN_RMSNORM && MT == 1 && q4 <= DS_RMS_HOLD * DS_CTHREADS) {
+                // one token, row held in registers: one trip to L2
+                float4 v[DS_RMS_HOLD];
                 float ss = 0.f;
-                for (int i = threadIdx.x; i < P.K / 4; i += DS_THREADS) {
-                    const float4 v = __ldcg(s4 + i);
-                    ss = fmaf(v.x, v.x, ss); ss = fmaf(v.y, v.y, ss); ss = fmaf(v.z, v.z, ss); ss = fmaf(v.w, v.w, ss);
+#pragma unroll
+                for (int n = 0; n < DS_RMS_HOLD; ++n) {
+                    const int i4 = threadIdx.x + n * DS_CTHREADS;
+                    v[n] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (i4 < q4) v[n] = __ldcg(reinterpret_cast<const float4*>(P.src) + i4);
+                }
+#pragma unroll
+                for (int n = 0; n < DS_RMS_HOLD; ++n) {
+                    ss = fmaf(v[n].x, v[n].x, ss); ss = fmaf(v[n].y, v[n].y, ss);
+                    ss = fmaf(v[n].z, v[n].z, ss); ss = fmaf(v[n].w, v[n].w, ss);
                 }
 #pragma unroll
                 for (int d = 16; d > 0; d >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, d);
-                if (lane == 0) sh.red[m][warp] = ss;
-            }
-            __syncthreads();
-            if ((int)threadIdx.x < M) {
+                if (lane == 0) sh.red[0][warp] = ss;
+                ds_consumer_sync();
                 float tot = 0.f;
 #pragma unroll
-                for (int w = 0; w < DS_WARPS; ++w) tot += sh.red[threadIdx.x][w];
-                sh.scale[threadIdx.x] = rsqrtf(tot / (float)P.K + 1e-6f);
+                for (int w = 0; w < DS_WARPS; ++w) tot += sh.red[0][w];
+                const float scale = rsqrtf(tot / (float)P.K + 1e-6f);
+#pragma unroll
+                for (int n = 0; n < DS_RMS_HOLD; ++n) {
+                    const int i4 = threadIdx.x + n * DS_CTHREADS;
+                    if (n * DS_CTHREADS < q4)   // the same for every thread: warps stay whole
+                        place(0, i4, make_float4(v[n].x * scale, v[n].y * scale, v[n].z * scale, v[n].w * scale), i4 < q4, true);
+                }
+            } else {
+                if (P.in_op == AQ_IN_RMSNORM) {
+                    for (int m = 0; m < M; ++m) {
+                        const float4* s4 = reinterpret_cast<const float4*>(P.src + (int64_t)m * P.K);
+                        float ss = 0.f;
+                        for (int i = threadIdx.x; i < q4; i += DS_CTHREADS) {
+                            const float4 v = __ldcg(s4 + i);
+                            ss = fmaf(v.x, v.x, ss); ss = fmaf(v.y, v.y, ss); ss = fmaf(v.z, v.z, ss); ss = fmaf(v.w, v.w, ss);
+                        }
+#pragma unroll
+                        for (int d = 16; d > 0; d >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, d);
+                        if (lane == 0) sh.red[m][warp] = ss;
+                    }
+                    ds_consumer_sync();
+                    if ((int)threadIdx.x < M) {
+                        float tot = 0.f;
+#pragma unroll
+                        for (int w = 0; w < DS_WARPS; ++w) tot += sh.red[threadIdx.x][w];
+                        sh.scale[threadIdx.x] = rsqrtf(tot / (float)P.K + 1e-6f);
+                    }
+                    ds_consumer_sync();
+                }
+                // one list of work: first the slabs this CTA reads, then its share of the record
+                const int per_slab = 64 * M;
+                const int n_a = n_slabs * per_slab;
+                const int n_b = (g1 - g0) * M;
+                const int n_all = n_a + n_b;
+                for (int it0 = 0; it0 < n_all; it0 += DS_CTHREADS) {
+                    const int it = it0 + threadIdx.x;
+                    int m = 0, i4 = 0;
+                    bool valid = false;
+                    if (it < n_a) {
+                        const int sl = it / per_slab, w = it - sl * per_slab;
+                        m = w >> 6;
+                        int oi = 0;
+                        while (oi + 1 < P.op_count && sl >= sh.seg_xoff[pb][oi + 1]) ++oi;
+                        i4 = (sh.seg_slab_lo[pb][oi] + sl - sh.seg_xoff[pb][oi]) * 64 + (w & 63);
+                        valid = i4 < q4;
+                    } else if (it < n_all) {
+                        const int w = it - n_a;
+                        m = w / (g1 - g0);
+                        i4 = g0 + w - m * (g1 - g0);
+                        valid = true;
+                    }
+                    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (valid) v = ds_form4(P, m, i4 * 4, P.in_op == AQ_IN_RMSNORM ? sh.scale[m] : 1.f);
+                    if (it0 + (int)(threadIdx.x - lane) < n_a) {
+                        place(m, i4, v, valid, false);           // n_a is a multiple of 32: the whole warp is inside the slab items
+                    } else if (valid) {
+                        float sum;
+                        const uint2 r = ds_round4<BF16>(v, &sum);
+                        *reinterpret_cast<uint2*>(rec_out + (int64_t)m * P.K + i4 * 4) = r;
+                    }
+                }
             }
-            __syncthreads();
         }
-        {
-            // slabs this CTA's warps read -> shared memory, laid out [slab][token][256]
-            const int n_slabs = sh.seg_xoff[pb][P.op_count];
-            const int items = n_slabs * M * 64;   // groups of 4 elements
-            for (int it = threadIdx.x; it < items; it += DS_THREADS) {
-                const int k4 = it & 63, sm_ = it >> 6, m = sm_ % M, sl = sm_ / M;
-                int oi = 0;
-                while (oi + 1 < P.op_count && sl >= sh.seg_xoff[pb][oi + 1]) ++oi;
-                const int k = (sh.seg_slab_lo[pb][oi] + sl - sh.seg_xoff[pb][oi]) * 256 + k4 * 4;
-                uint2 r = make_uint2(0u, 0u);
-                if (k < P.K) r = ds_form4<BF16>(P, m, k, P.in_op == AQ_IN_RMSNORM ? sh.scale[m] : 1.f);
-                *reinterpret_cast<uint2*>(sh.xs + (size_t)it * 4) = r;
-            }
-            // this CTA's share of the vector -> the caller's workspace
-            const int q4 = P.K / 4;
-            const int g0 = (int)(((int64_t)q4 * blockIdx.x) / gridDim.x), g1 = (int)(((int64_t)q4 * (blockIdx.x + 1)) / gridDim.x);
-            const int span = g1 - g0;
-            for (int it = threadIdx.x; it < span * M; it += DS_THREADS) {
-                const int m = it / span, k = (g0 + it - m * span) * 4;
-                const uint2 r = ds_form4<BF16>(P, m, k, P.in_op == AQ_IN_RMSNORM ? sh.scale[m] : 1.f);
-                *reinterpret_cast<uint2*>(reinterpret_cast<uint16_t*>(P.stage) + (int64_t)m * P.K + k) = r;
-            }
-        }
-        __syncthreads();
+        ds_consumer_sync();
 
         // -- consume this warp's units of the phase --
         int wa, wb;
-        ds_warp_run(P.units_total, blockIdx.x, gridDim.x, warp, wa, wb);
+        ds_warp_run(P.units_q, P.units_r, blockIdx.x, warp, wa, wb);
 #pragma unroll 1
         for (int oi = 0; oi < P.op_count; ++oi) {
             const int opx = P.op_first + oi;
@@ -416,29 +549,31 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArg
             const int u0 = max(wa, op.unit_off) - op.unit_off, u1 = min(wb, op.unit_off + op.n_units) - op.unit_off;
             if (u0 < u1 && !dead) {
                 int Pk = u0 / NT, R = u0 - Pk * NT;
-                const int xbase = sh.seg_xoff[pb][oi] - sh.seg_slab_lo[pb][oi];   // slab Pk sits at xs[(xbase + Pk) M 256]
-                ds_load_x_operand<MT, BF16>(xo, sh.xs + (xbase + Pk) * M * 256, M, lane);
+                const uint8_t* xseg = sh.xs + (size_t)(sh.seg_xoff[pb][oi] - sh.seg_slab_lo[pb][oi] + Pk) * slab_bytes;
+                ds_load_x_operand<MT, BF16>(xo, xseg, M, lane);
+                float* dst = op.dst;
+                const float* res = op.res;
+                const int N = op.N;
 #pragma unroll 1
                 for (int u = u0; u < u1; ++u) {
-                    const uint32_t slot = cseq % DS_SLOTS, parity = (cseq / DS_SLOTS) & 1u;
-                    const uint32_t bar = ds_smem(&sh.bar[warp][slot]);
-                    dead = __any_sync(0xffffffffu, !ds_mbar_wait(bar, parity));
+                    dead = __any_sync(0xffffffffu, !ds_mbar_wait(ds_smem(&sh.full[warp][cslot]), cparity));
                     if (dead) {
                         if (lane == 0) { atomicCAS(&g_decode_status, 0, 2); sh.abort_flag = 1; }
                         break;
                     }
-                    const uint8_t* unit = &sh.ring[warp][slot][0];
+                    const uint8_t* unit = &sh.ring[warp][cslot][0];
                     float acc[4] = {0.f, 0.f, 0.f, 0.f};
                     if (bits == 2) unit_mac<2, MT, BF16>(unit, xo, lane, acc);
                     else if (bits == 3) unit_mac<3, MT, BF16>(unit, xo, lane, acc);
                     else unit_mac<4, MT, BF16>(unit, xo, lane, acc);
-                    ++cseq;
                     __syncwarp();        // every lane has read its part of the slot
-                    issue_next();        // refill it
-                    unit_commit<MT>(acc, op.dst, op.N, R * 16, op.N, M, lane, Pk == 0 ? op.res : nullptr);
+                    if (lane == 0) ds_mbar_arrive(ds_smem(&sh.empty[warp][cslot]));
+                    if (++cslot == DS_SLOTS) { cslot = 0; cparity ^= 1u; }
+                    unit_commit<MT>(acc, dst, N, R * 16, N, M, lane, Pk == 0 ? res : nullptr);
                     if (++R == NT) {
                         R = 0; ++Pk;
-                        if (u + 1 < u1) ds_load_x_operand<MT, BF16>(xo, sh.xs + (xbase + Pk) * M * 256, M, lane);
+                        xseg += slab_bytes;
+                        if (u + 1 < u1) ds_load_x_operand<MT, BF16>(xo, xseg, M, lane);
                     }
                 }
             }
@@ -456,14 +591,8 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArg
         }
     }
 
-    // copies still in flight into this CTA's shared memory must land before it exits
-    if (*reinterpret_cast<volatile int*>(&sh.abort_flag)) {
-        for (uint32_t s = cseq; s < iseq; ++s) {
-            const uint32_t bar = ds_smem(&sh.bar[warp][s % DS_SLOTS]);
-            ds_mbar_wait(bar, (s / DS_SLOTS) & 1u);
-        }
-        __nanosleep(100000);   // ... and a descriptor record that may still be on its way
-    }
+    // after a failed wait copies may still be on their way into this CTA's shared memory: give them time
+    if (*reinterpret_cast<volatile int*>(&sh.abort_flag)) __nanosleep(500000);
 }
 
 // ---- host: plan, cache, launch -----------------------------------------------------
@@ -542,18 +671,21 @@ bool build_decode_tables(const aq_stack_t* p, const StackPlan& plan, int M, int 
             }
             if ((int)deps.size() > DS_MAX_DEPS) return false;
             P.units_total = (int32_t)off;
+            P.units_q = (int32_t)(off / n_cta);
+            P.units_r = (int32_t)(off % n_cta);
             P.n_deps = (int)deps.size();
             for (size_t j = 0; j < deps.size(); ++j) P.deps[j] = (int16_t)deps[j];
             // every CTA's staged slabs must fit the shared-memory buffer
             for (int c = 0; c < n_cta; ++c) {
-                const int64_t ca = off * c / n_cta, cb = off * (c + 1) / n_cta;
+                const int64_t ca = (int64_t)P.units_q * c + std::min<int64_t>(c, P.units_r);
+                const int64_t cb = ca + P.units_q + (c < P.units_r ? 1 : 0);
                 int64_t slabs = 0;
                 for (int i = 0; i < P.op_count; ++i) {
                     const int64_t o0 = P.ops[i].unit_off, n = P.ops[i].n_units;
                     const int64_t u0 = std::max(ca, o0) - o0, u1 = std::min(cb, o0 + n) - o0;
                     if (u0 < u1) slabs += (u1 - 1) / P.ops[i].NT - u0 / P.ops[i].NT + 1;
                 }
-                if (slabs * M * 512 > DS_XS_BYTES) return false;
+                if (slabs * ds_slab_bytes(M) > DS_XS_BYTES) return false;
             }
             for (int i = first; i < last; ++i) writer[p->ops[i].dst] = i;
             phases.push_back(P);
@@ -635,7 +767,8 @@ int launch_decode_stack(const aq_stack_t* p, const StackPlan& plan, int M, aq_dt
     cudaError_t e = cudaMemsetAsync(a.cnt, 0, dp->cnt_bytes, s);
     if (e == cudaSuccess) {
         const bool bf = (dt == AQ_BF16);
-        if (M <= 2) e = bf ? launch_ds<2, true>(a, grid, s) : launch_ds<2, false>(a, grid, s);
+        if (M == 1) e = bf ? launch_ds<1, true>(a, grid, s) : launch_ds<1, false>(a, grid, s);
+        else if (M == 2) e = bf ? launch_ds<2, true>(a, grid, s) : launch_ds<2, false>(a, grid, s);
         else if (M <= 4) e = bf ? launch_ds<4, true>(a, grid, s) : launch_ds<4, false>(a, grid, s);
         else e = bf ? launch_ds<8, true>(a, grid, s) : launch_ds<8, false>(a, grid, s);
     }

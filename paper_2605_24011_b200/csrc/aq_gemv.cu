@@ -7,15 +7,7 @@
 // ring in shared memory, so several KB per warp are always in flight and no
 // block-wide barrier exists.
 //
-// Arithmetic: with w = d q + m per block,
-//     sum_k x w = d * sum (BIAS + q) x  +  (m - BIAS d) * sum x
-// The first sum runs on the tensor cores (mma.sync m16n8k16, fp32
-// accumulate): the A operand is built two codes per LOP3 by OR-ing the code
-// bits into the mantissa of the half-precision constant BIAS (1024 for fp16,
-// 128 for bf16), the B operand holds x.  The 8 columns of the instruction are
-// (block, token) pairs: with MT tokens per call, 8/MT blocks accumulate side
-// by side and the per-block scale is applied to the 4 accumulators only once
-// per group of 8/MT blocks.
+// The arithmetic of one unit is in aq_gemv_core.cuh.
 #include <type_traits>
 
 #include "aq_internal.h"
@@ -75,7 +67,9 @@ __global__ void __launch_bounds__(GEMV_WARPS * 32, 2) gemv_kernel(const GemvArgs
     }
 
     XOperand<MT> xo;
-    int64_t curP = -1;
+    int64_t P = u0 / a.NT;
+    int R = (int)(u0 - P * a.NT);
+    load_x_operand<MT, BF16>(xo, a.x, a.K, a.M, P, lane);
     int slot = 0;
     for (int64_t u = u0; u < u1; ++u) {
         cp_async_wait<GEMV_STAGES - 2>();
@@ -86,13 +80,14 @@ __global__ void __launch_bounds__(GEMV_WARPS * 32, 2) gemv_kernel(const GemvArgs
             if (un < u1) issue(un, ns);
             cp_async_commit();
         }
-        const int64_t P = u / a.NT;
-        const int R = (int)(u - P * a.NT);
-        if (P != curP) { load_x_operand<MT, BF16>(xo, a.x, a.K, a.M, P, lane); curP = P; }
         float acc[4] = {0.f, 0.f, 0.f, 0.f};
         unit_mac<BITS, MT, BF16>(ring + slot * UB, xo, lane, acc);
         unit_commit<MT>(acc, a.acc, a.ldacc, R * 16, a.N, a.M, lane);
         if (++slot == GEMV_STAGES) slot = 0;
+        if (++R == a.NT) {
+            R = 0; ++P;
+            if (u + 1 < u1) load_x_operand<MT, BF16>(xo, a.x, a.K, a.M, P, lane);
+        }
     }
     cp_async_wait<0>();
 }
@@ -119,7 +114,8 @@ static cudaError_t launch_one(const GemvArgs& a, cudaStream_t s) {
 
 template <int BITS, bool BF16>
 static cudaError_t launch_mt(const GemvArgs& a, cudaStream_t s) {
-    if (a.M <= 2) return launch_one<BITS, 2, BF16>(a, s);
+    if (a.M == 1) return launch_one<BITS, 1, BF16>(a, s);
+    if (a.M == 2) return launch_one<BITS, 2, BF16>(a, s);
     if (a.M <= 4) return launch_one<BITS, 4, BF16>(a, s);
     return launch_one<BITS, 8, BF16>(a, s);
 }

@@ -10,18 +10,11 @@ namespace aq {
 
 template <int BITS>
 __device__ __forceinline__ void place_code(uint32_t* words, int j, int hi, int c, uint32_t q) {
-    if constexpr (BITS == 4) {
-        words[(j >> 1) * 4 + (j & 1) * 2 + hi] |= q << (4 * ((c >> 1) + 4 * (c & 1)));
-    } else if constexpr (BITS == 2) {
-        words[(j >> 1) * 2 + hi] |= q << (16 * (c & 1) + 2 * ((c >> 1) + 4 * (j & 1)));
-    } else {
-        const int P = 4 * j + (c >> 1), half = c & 1;
-        if (P < 15) {
-            words[hi * 3 + P / 5] |= q << (16 * half + 3 * (P % 5));
-        } else {
 #pragma unroll
-            for (int tb = 0; tb < 3; ++tb) words[hi * 3 + tb] |= ((q >> tb) & 1u) << (16 * half + 15);
-        }
+    for (int tb = 0; tb < BITS; ++tb) {
+        int widx, bitpos;
+        slot_bit_home(BITS, j, hi, c, tb, widx, bitpos);
+        words[widx] |= ((q >> tb) & 1u) << bitpos;
     }
 }
 
