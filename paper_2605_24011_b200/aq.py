@@ -10,7 +10,7 @@ import ctypes as C
 import os
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libaq.so")
+LIB_PATH = os.environ.get("AQ_LIBRARY") or os.path.join(_HERE, "libaq.so")   # AQ_LIBRARY: another build of the same library
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(

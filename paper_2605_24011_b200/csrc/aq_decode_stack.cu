@@ -48,7 +48,8 @@ constexpr int DS_CTHREADS = DS_WARPS * 32;  // consumer threads
 constexpr int DS_THREADS = DS_CTHREADS + 32;   // + the copy warp
 constexpr int DS_SLOTS = 5;                 // ring depth per warp (units)
 constexpr int DS_SLOT_BYTES = 2560;         // the largest unit (4-bit: 2 fragments of 1280 B)
-constexpr int DS_XS_BYTES = 6 * 4128;       // staged input: six one-token slabs (see ds_slab_bytes)
+constexpr int DS_MAX_SLOTS = 6;             // staged slabs per phase per CTA (one token; fewer with more tokens)
+constexpr int DS_XS_BYTES = DS_MAX_SLOTS * 4128;   // staged input (see ds_slab_bytes)
 constexpr int DS_MAX_PHASE_OPS = 8;
 constexpr int DS_MAX_DEPS = 12;
 constexpr int DS_RMS_HOLD = 4;              // float4 per thread kept in registers by the one-token RMS path
@@ -67,10 +68,10 @@ struct DsOp {
     const float* res;      // float32 [M][N] added once (by the k-slab-0 units), or null
     int32_t N;             // true rows
     int32_t NT;            // 16-row tiles
-    int32_t n_units;       // KP * NT
-    int32_t unit_off;      // offset of this op's units inside its phase
+    int32_t n_units;       // KP * NT = units_q * (number of CTAs) + units_r
     int32_t bits;
-    int32_t pad_;
+    int32_t units_q;
+    int32_t units_r_rot;   // units_r | rot << 16: CTA c takes the run of slot (c + rot) mod (number of CTAs)
 };
 
 struct DsPhase {
@@ -84,16 +85,34 @@ struct DsPhase {
     int32_t units_total;
     int32_t n_deps;
     int16_t deps[DS_MAX_DEPS];   // ops that must be complete before this phase reads its inputs
-    int32_t units_q, units_r;    // units_total = units_q * (number of CTAs) + units_r
+    int32_t pad_[2];
     DsOp ops[DS_MAX_PHASE_OPS];
 };
 static_assert(sizeof(DsOp) == 48, "DsOp layout");
 static_assert(sizeof(DsPhase) % 16 == 0, "a phase record is fetched with one bulk copy");
 
+// What the copy stream needs to know of an op / a phase, small enough to keep the
+// whole program's worth in shared memory (a cursor then advances in tens of cycles).
+struct DsMiniOp {
+    const uint8_t* frags;
+    uint32_t q_bits;       // units_q | bits << 28
+    uint32_t r_rot;        // units_r | rot << 16
+};
+struct DsMiniPhase {
+    int32_t op_first;      // index into the mini-op table
+    int32_t op_count;
+    int32_t pad_[2];
+};
+static_assert(sizeof(DsMiniOp) == 16 && sizeof(DsMiniPhase) == 16, "mini tables are copied as 16-byte items");
+constexpr int DS_MINI_BYTES = 8192;
+
 struct DsArgs {
     const DsPhase* phases;
+    const DsMiniPhase* mini_phases;   // n_phases entries, followed by
+    const DsMiniOp* mini_ops;         // n_mini_ops entries (contiguous: one copy brings both)
     uint32_t* cnt;         // per-op arrival counters, zero at launch
     int n_phases;
+    int n_mini_ops;
     int M;
 };
 
@@ -159,51 +178,51 @@ __device__ __forceinline__ void ds_consumer_sync() { asm volatile("bar.sync 1, %
 struct DsCursor {
     int ph;                // phase (n_phases: past the end)
     int oi;                // op inside the phase
-    int wa, wb;            // the warp's run inside the phase's concatenated units
     int u, u_end;          // position inside the current op
     const uint8_t* base;   // the op's fragments
     int ub;                // bytes per unit
 };
 
-// The run of units CTA `cta` owns in a phase of q * (number of CTAs) + r units:
-// the first r CTAs take q + 1 units, the others q.
-__device__ __forceinline__ void ds_cta_run(int q, int r, int cta, int& a, int& b) {
-    a = q * cta + min(cta, r);
-    b = a + q + (cta < r ? 1 : 0);
+// Every op's units are dealt on their own: with n = q G + r units and G CTAs, slot
+// s takes q + 1 units if s < r, else q; CTA c takes slot (c + rot) mod G, where rot
+// moves on from op to op so that the odd units do not always land on the same CTAs.
+__device__ __forceinline__ void ds_cta_run(int q, int r_rot, int& a, int& b) {
+    const int r = r_rot & 0xFFFF, rot = r_rot >> 16;
+    int s = (int)blockIdx.x + rot;
+    if (s >= (int)gridDim.x) s -= (int)gridDim.x;
+    a = q * s + min(s, r);
+    b = a + q + (s < r ? 1 : 0);
 }
-// ... and the run of one of its warps.
-__device__ __forceinline__ void ds_warp_run(int q, int r, int cta, int warp, int& wa, int& wb) {
+// ... and the run of one of its consumer warps (the warps too take turns with the short shares).
+__device__ __forceinline__ void ds_warp_run(int q, int r_rot, int warp, int& wa, int& wb) {
     int a, b;
-    ds_cta_run(q, r, cta, a, b);
+    ds_cta_run(q, r_rot, a, b);
     const int n = b - a;
-    wa = a + (n * warp) / DS_WARPS;
-    wb = a + (n * (warp + 1)) / DS_WARPS;
+    int w = warp + ((r_rot >> 16) * 7) % DS_WARPS;
+    if (w >= DS_WARPS) w -= DS_WARPS;
+    wa = a + (n * w) / DS_WARPS;
+    wb = a + (n * (w + 1)) / DS_WARPS;
 }
 
 // Moves the cursor to the next op (from (ph, oi) on) in which the warp owns units.
-__device__ __forceinline__ void ds_seek(DsCursor& c, const DsArgs& a, int warp, bool new_phase) {
-    while (c.ph < a.n_phases) {
-        const DsPhase* P = a.phases + c.ph;
-        if (new_phase) {
-            ds_warp_run(__ldg(&P->units_q), __ldg(&P->units_r), blockIdx.x, warp, c.wa, c.wb);
-            c.oi = 0;
-            new_phase = false;
-        }
-        const int oc = __ldg(&P->op_count);
-        while (c.oi < oc) {
-            const DsOp* op = P->ops + c.oi;
-            const int off = __ldg(&op->unit_off), n = __ldg(&op->n_units);
-            const int u0 = max(c.wa, off) - off, u1 = min(c.wb, off + n) - off;
+// mp / mo: the mini tables (in shared memory when they fit, else in global memory).
+__device__ __forceinline__ void ds_seek(DsCursor& c, const DsMiniPhase* mp, const DsMiniOp* mo, int n_phases, int warp) {
+    while (c.ph < n_phases) {
+        const DsMiniPhase P = mp[c.ph];
+        while (c.oi < P.op_count) {
+            const DsMiniOp op = mo[P.op_first + c.oi];
+            int u0, u1;
+            ds_warp_run((int)(op.q_bits & 0x0FFFFFFFu), (int)op.r_rot, warp, u0, u1);
             if (u0 < u1) {
                 c.u = u0; c.u_end = u1;
-                c.ub = 2 * frag_bytes(__ldg(&op->bits));
-                c.base = reinterpret_cast<const uint8_t*>(__ldg(reinterpret_cast<const unsigned long long*>(&op->frags)));
+                c.ub = 2 * frag_bytes((int)(op.q_bits >> 28));
+                c.base = op.frags;
                 return;
             }
             ++c.oi;
         }
         ++c.ph;
-        new_phase = true;
+        c.oi = 0;
     }
 }
 
@@ -242,14 +261,17 @@ __device__ __forceinline__ float4 ds_form4(const DsPhase& P, int m, int k, float
 struct DsShared {
     alignas(128) uint8_t ring[DS_WARPS][DS_SLOTS][DS_SLOT_BYTES];
     alignas(128) uint8_t xs[DS_XS_BYTES];   // staged input slabs
+    alignas(16) uint8_t mini[DS_MINI_BYTES];   // [DsMiniPhase x n_phases][DsMiniOp x n_mini_ops] when they fit
     alignas(16) DsPhase rec[2];             // descriptors of the current and the next phase
     alignas(8) uint64_t full[DS_WARPS][DS_SLOTS];    // copy landed
     alignas(8) uint64_t empty[DS_WARPS][DS_SLOTS];   // consumer has read the slot
     alignas(8) uint64_t rec_bar[2];
     float red[AQ_DECODE_MAX_M][DS_WARPS];
     float scale[AQ_DECODE_MAX_M];
-    int seg_slab_lo[2][DS_MAX_PHASE_OPS];   // per op of the phase: first pair-slab staged for this CTA
-    int seg_xoff[2][DS_MAX_PHASE_OPS + 1];  // ... and where its slabs start in xs (in slabs); [op_count] = total
+    int seg_slab_lo[2][DS_MAX_PHASE_OPS];   // per op of the phase: first pair-slab this CTA reads for it
+    int seg_slot_lo[2][DS_MAX_PHASE_OPS];   // ... and the slot in xs where that slab is staged (the next slabs follow)
+    int slab_of_slot[2][DS_MAX_SLOTS];      // the slabs staged for this phase, ascending
+    int n_slots[2];
     int done[32];                           // warps of this CTA that finished op (index & 31)
     int abort_flag;
 };
@@ -316,8 +338,16 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArg
     // one-token slabs keep zeros everywhere but in the chunks the stagers rewrite every phase
     for (int i = threadIdx.x; i < DS_XS_BYTES / 16; i += DS_THREADS)
         reinterpret_cast<uint4*>(sh.xs)[i] = make_uint4(0, 0, 0, 0);
+    // the copy stream's tables: into shared memory when they fit
+    const int mini_items = a.n_phases + a.n_mini_ops;
+    const bool mini_in_smem = mini_items * 16 <= DS_MINI_BYTES;
+    if (mini_in_smem)
+        for (int i = threadIdx.x; i < mini_items; i += DS_THREADS)
+            reinterpret_cast<uint4*>(sh.mini)[i] = __ldg(reinterpret_cast<const uint4*>(a.mini_phases) + i);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     __syncthreads();
+    const DsMiniPhase* mp = mini_in_smem ? reinterpret_cast<const DsMiniPhase*>(sh.mini) : a.mini_phases;
+    const DsMiniOp* mo = mini_in_smem ? reinterpret_cast<const DsMiniOp*>(sh.mini + (size_t)a.n_phases * 16) : a.mini_ops;
 
     uint64_t pol, pol_keep;
     asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
@@ -326,8 +356,8 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArg
     if (warp == DS_WARPS) {
         // ================= the copy warp: lane w keeps consumer warp w's ring full =================
         DsCursor c;
-        c.ph = a.n_phases; c.oi = 0; c.wa = c.wb = 0; c.u = c.u_end = 0; c.base = nullptr; c.ub = 0;
-        if (lane < DS_WARPS) { c.ph = 0; ds_seek(c, a, lane, true); }
+        c.ph = a.n_phases; c.oi = 0; c.u = c.u_end = 0; c.base = nullptr; c.ub = 0;
+        if (lane < DS_WARPS) { c.ph = 0; ds_seek(c, mp, mo, a.n_phases, lane); }
         uint32_t iseq = 0;   // copies issued for this consumer
         uint64_t t_progress = ds_now_ns();
         uint32_t idle = 0;
@@ -343,12 +373,13 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArg
                     ds_expect_tx(bar, (uint32_t)c.ub);
                     ds_bulk_load(ds_smem(&sh.ring[lane][slot][0]), c.base + (int64_t)c.u * c.ub, (uint32_t)c.ub, bar, pol);
                     ++iseq;
-                    if (++c.u == c.u_end) { ++c.oi; ds_seek(c, a, lane, false); }
+                    if (++c.u == c.u_end) { ++c.oi; ds_seek(c, mp, mo, a.n_phases, lane); }
                     moved = true;
                 }
             }
             if (!__any_sync(0xffffffffu, active)) break;
             if (__any_sync(0xffffffffu, moved)) { idle = 0; continue; }
+            __nanosleep(200);   // a consumer needs about a microsecond per unit: no need to spin on its barriers
             if ((++idle & 255u) == 0) {   // nothing to do for a while: stop if the CTA gave up, or after the time limit
                 if (*reinterpret_cast<volatile int*>(&sh.abort_flag)) break;
                 const uint64_t t = ds_now_ns();
@@ -386,22 +417,31 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArg
         if (*reinterpret_cast<volatile int*>(&sh.abort_flag) == 0) {
             // -- which slabs of the input this CTA's warps will read (independent of the data) --
             if (threadIdx.x == DS_CTHREADS - 1) {
-                int ca, cb;
-                ds_cta_run(P.units_q, P.units_r, blockIdx.x, ca, cb);
-                int tot = 0;
+                int lo[DS_MAX_PHASE_OPS], hi[DS_MAX_PHASE_OPS];
                 for (int oi = 0; oi < P.op_count; ++oi) {
-                    const int off = P.ops[oi].unit_off, n = P.ops[oi].n_units, NT = P.ops[oi].NT;
-                    const int u0 = max(ca, off) - off, u1 = min(cb, off + n) - off;
-                    sh.seg_xoff[pb][oi] = tot;
-                    if (u0 < u1) {
-                        const int lo = u0 / NT, hi = (u1 - 1) / NT;
-                        sh.seg_slab_lo[pb][oi] = lo;
-                        tot += hi - lo + 1;
-                    } else {
-                        sh.seg_slab_lo[pb][oi] = 0;
-                    }
+                    int u0, u1;
+                    ds_cta_run(P.ops[oi].units_q, P.ops[oi].units_r_rot, u0, u1);
+                    lo[oi] = (u0 < u1) ? u0 / P.ops[oi].NT : 0;
+                    hi[oi] = (u0 < u1) ? (u1 - 1) / P.ops[oi].NT : -1;
+                    sh.seg_slab_lo[pb][oi] = lo[oi];
                 }
-                sh.seg_xoff[pb][P.op_count] = tot;
+                // ascending list of the distinct slabs: repeatedly take the smallest one above the last
+                int n = 0, last = -1;
+                for (;;) {
+                    int nxt = 0x7fffffff;
+                    for (int oi = 0; oi < P.op_count; ++oi) {
+                        if (hi[oi] > last) nxt = min(nxt, max(lo[oi], last + 1));
+                    }
+                    if (nxt == 0x7fffffff || n == DS_MAX_SLOTS) break;
+                    sh.slab_of_slot[pb][n++] = nxt;
+                    last = nxt;
+                }
+                sh.n_slots[pb] = n;
+                for (int oi = 0; oi < P.op_count; ++oi) {
+                    int sl = 0;
+                    while (sl < n && sh.slab_of_slot[pb][sl] != lo[oi]) ++sl;
+                    sh.seg_slot_lo[pb][oi] = sl;
+                }
             }
             // -- wait for the writers of what this phase reads --
             if ((int)threadIdx.x < P.n_deps) {
@@ -425,12 +465,18 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArg
 
         // -- form the rounded input vector: slabs this CTA reads -> shared memory, its share -> workspace --
         {
-            const int n_slabs = sh.seg_xoff[pb][P.op_count];
+            const int n_slots = sh.n_slots[pb];
             const int q4 = P.K >> 2;                                  // groups of 4 elements per token
             const int g0 = (int)(((int64_t)q4 * blockIdx.x) / gridDim.x), g1 = (int)(((int64_t)q4 * (blockIdx.x + 1)) / gridDim.x);
             uint16_t* rec_out = reinterpret_cast<uint16_t*>(P.stage);
-            // stores group i4 (elements 4 i4 ..) of token m where it is needed; whole warps call this together
-            auto place = [&](int m, int i4, float4 v, bool valid, bool with_record) {
+            // the staged copy of slab `slab`, or null when this CTA does not read it
+            auto slot_of = [&](int slab) -> uint8_t* {
+                for (int sl = 0; sl < n_slots; ++sl)
+                    if (sh.slab_of_slot[pb][sl] == slab) return sh.xs + (size_t)sl * slab_bytes;
+                return nullptr;
+            };
+            // stores group i4 (elements 4 i4 ..) of token m into slab copy `sl`; whole warps call this together
+            auto place = [&](uint8_t* sl, int m, int i4, float4 v, bool rec) {
                 float sum;
                 const uint2 r = ds_round4<BF16>(v, &sum);   // v is zero past the end of the row: padding stages zeros
                 if constexpr (MT == 1) {   // block sums: 8 consecutive groups = 8 consecutive lanes
@@ -438,29 +484,28 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArg
                     sum += __shfl_xor_sync(0xffffffffu, sum, 2);
                     sum += __shfl_xor_sync(0xffffffffu, sum, 4);
                 }
-                const int k = i4 * 4, slab = k >> 8, kl = k & 255;
-                for (int oi = 0; oi < P.op_count; ++oi) {
-                    const int lo = sh.seg_slab_lo[pb][oi], xo0 = sh.seg_xoff[pb][oi], n = sh.seg_xoff[pb][oi + 1] - xo0;
-                    if (slab >= lo && slab < lo + n) {
-                        uint8_t* sl = sh.xs + (size_t)(xo0 + slab - lo) * slab_bytes;
-                        ds_store4<MT>(sl, M, m, kl, r);
-                        if constexpr (MT == 1) {
-                            if ((lane & 7) == 0) *reinterpret_cast<float*>(sl + 4096 + (kl >> 5) * 4) = sum;
-                        }
+                const int kl = (i4 * 4) & 255;
+                if (sl) {
+                    ds_store4<MT>(sl, M, m, kl, r);
+                    if constexpr (MT == 1) {
+                        if ((lane & 7) == 0) *reinterpret_cast<float*>(sl + 4096 + (kl >> 5) * 4) = sum;
                     }
                 }
-                if (with_record && valid && i4 >= g0 && i4 < g1) *reinterpret_cast<uint2*>(rec_out + (int64_t)m * P.K + k) = r;
+                if (rec) *reinterpret_cast<uint2*>(rec_out + (int64_t)m * P.K + i4 * 4) = r;
             };
             if (P.in_op == AQ_IN_RMSNORM && MT == 1 && q4 <= DS_RMS_HOLD * DS_CTHREADS) {
-                // one token, row held in registers: one trip to L2
+                // one token, row held in registers: one trip to L2, destinations worked out while it is under way
                 float4 v[DS_RMS_HOLD];
-                float ss = 0.f;
+                uint8_t* dest[DS_RMS_HOLD];
 #pragma unroll
                 for (int n = 0; n < DS_RMS_HOLD; ++n) {
                     const int i4 = threadIdx.x + n * DS_CTHREADS;
                     v[n] = make_float4(0.f, 0.f, 0.f, 0.f);
                     if (i4 < q4) v[n] = __ldcg(reinterpret_cast<const float4*>(P.src) + i4);
                 }
+#pragma unroll
+                for (int n = 0; n < DS_RMS_HOLD; ++n) dest[n] = slot_of((threadIdx.x + n * DS_CTHREADS) >> 6);
+                float ss = 0.f;
 #pragma unroll
                 for (int n = 0; n < DS_RMS_HOLD; ++n) {
                     ss = fmaf(v[n].x, v[n].x, ss); ss = fmaf(v[n].y, v[n].y, ss);
@@ -478,7 +523,8 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArg
                 for (int n = 0; n < DS_RMS_HOLD; ++n) {
                     const int i4 = threadIdx.x + n * DS_CTHREADS;
                     if (n * DS_CTHREADS < q4)   // the same for every thread: warps stay whole
-                        place(0, i4, make_float4(v[n].x * scale, v[n].y * scale, v[n].z * scale, v[n].w * scale), i4 < q4, true);
+                        place(dest[n], 0, i4, make_float4(v[n].x * scale, v[n].y * scale, v[n].z * scale, v[n].w * scale),
+                              i4 >= g0 && i4 < g1);
                 }
             } else {
                 if (P.in_op == AQ_IN_RMSNORM) {
@@ -504,19 +550,19 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArg
                 }
                 // one list of work: first the slabs this CTA reads, then its share of the record
                 const int per_slab = 64 * M;
-                const int n_a = n_slabs * per_slab;
+                const int n_a = n_slots * per_slab;
                 const int n_b = (g1 - g0) * M;
                 const int n_all = n_a + n_b;
                 for (int it0 = 0; it0 < n_all; it0 += DS_CTHREADS) {
                     const int it = it0 + threadIdx.x;
                     int m = 0, i4 = 0;
                     bool valid = false;
+                    uint8_t* sl = nullptr;
                     if (it < n_a) {
-                        const int sl = it / per_slab, w = it - sl * per_slab;
+                        const int s_ = it / per_slab, w = it - s_ * per_slab;
                         m = w >> 6;
-                        int oi = 0;
-                        while (oi + 1 < P.op_count && sl >= sh.seg_xoff[pb][oi + 1]) ++oi;
-                        i4 = (sh.seg_slab_lo[pb][oi] + sl - sh.seg_xoff[pb][oi]) * 64 + (w & 63);
+                        i4 = sh.slab_of_slot[pb][s_] * 64 + (w & 63);
+                        sl = sh.xs + (size_t)s_ * slab_bytes;
                         valid = i4 < q4;
                     } else if (it < n_all) {
                         const int w = it - n_a;
@@ -527,7 +573,7 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArg
                     float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
                     if (valid) v = ds_form4(P, m, i4 * 4, P.in_op == AQ_IN_RMSNORM ? sh.scale[m] : 1.f);
                     if (it0 + (int)(threadIdx.x - lane) < n_a) {
-                        place(m, i4, v, valid, false);           // n_a is a multiple of 32: the whole warp is inside the slab items
+                        place(sl, m, i4, v, false);              // n_a is a multiple of 32: the whole warp is inside the slab items
                     } else if (valid) {
                         float sum;
                         const uint2 r = ds_round4<BF16>(v, &sum);
@@ -539,17 +585,16 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArg
         ds_consumer_sync();
 
         // -- consume this warp's units of the phase --
-        int wa, wb;
-        ds_warp_run(P.units_q, P.units_r, blockIdx.x, warp, wa, wb);
 #pragma unroll 1
         for (int oi = 0; oi < P.op_count; ++oi) {
             const int opx = P.op_first + oi;
             const DsOp& op = P.ops[oi];
             const int NT = op.NT, bits = op.bits;
-            const int u0 = max(wa, op.unit_off) - op.unit_off, u1 = min(wb, op.unit_off + op.n_units) - op.unit_off;
+            int u0, u1;
+            ds_warp_run(op.units_q, op.units_r_rot, warp, u0, u1);
             if (u0 < u1 && !dead) {
                 int Pk = u0 / NT, R = u0 - Pk * NT;
-                const uint8_t* xseg = sh.xs + (size_t)(sh.seg_xoff[pb][oi] - sh.seg_slab_lo[pb][oi] + Pk) * slab_bytes;
+                const uint8_t* xseg = sh.xs + (size_t)(sh.seg_slot_lo[pb][oi] + Pk - sh.seg_slab_lo[pb][oi]) * slab_bytes;
                 ds_load_x_operand<MT, BF16>(xo, xseg, M, lane);
                 float* dst = op.dst;
                 const float* res = op.res;
@@ -578,14 +623,14 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArg
                 }
             }
             // arrive: the CTA's last warp to finish the op publishes it
+            // (the warps' commits are ordered before the release below through the acq_rel counter in shared memory)
             __syncwarp();
             if (lane == 0) {
-                if (u0 < u1) __threadfence();
-                const int old = atomicAdd(&sh.done[opx & 31], 1);
+                int old;
+                asm volatile("atom.acq_rel.cta.shared::cta.add.u32 %0, [%1], 1;" : "=r"(old) : "r"(ds_smem(&sh.done[opx & 31])) : "memory");
                 if (old == DS_WARPS - 1) {
                     sh.done[opx & 31] = 0;
-                    __threadfence();
-                    atomicAdd(a.cnt + opx, 1u);
+                    asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(a.cnt + opx) : "memory");
                 }
             }
         }
@@ -601,8 +646,9 @@ namespace {
 struct DecodePlan {
     std::vector<uint8_t> key;
     std::vector<aq_handle_t> handles;
-    uint8_t* dev = nullptr;       // [phase records][arrival counters]
-    size_t phases_bytes = 0, cnt_bytes = 0;
+    uint8_t* dev = nullptr;       // [phase records][mini phases, mini ops][arrival counters]
+    size_t phases_bytes = 0, mini_bytes = 0, cnt_bytes = 0;
+    int n_mini_ops = 0;
     int n_phases = 0;
     int device = 0;
     uint64_t stamp = 0;
@@ -633,6 +679,7 @@ bool build_decode_tables(const aq_stack_t* p, const StackPlan& plan, int M, int 
     phases.clear();
     std::vector<int> writer(p->n_bufs, -1);
     std::vector<char> waited(p->n_ops, 0);
+    int rot = 0;   // where the next op's odd units start
     const int n_ph = (int)plan.phase_first.size();
     for (int ph = 0; ph < n_ph; ++ph) {
         const int pfirst = plan.phase_first[ph];
@@ -665,27 +712,30 @@ bool build_decode_tables(const aq_stack_t* p, const StackPlan& plan, int M, int 
                 d.res = (o.out_op == AQ_OUT_ADD) ? reinterpret_cast<const float*>(ws + plan.buf_off[o.res]) : nullptr;
                 if (o.out_op == AQ_OUT_ADD) need(o.res);
                 const int64_t nu = (int64_t)h->KP * h->NT;
-                if (off + nu > (int64_t)1 << 26) return false;
-                d.N = (int32_t)h->N; d.NT = h->NT; d.n_units = (int32_t)nu; d.unit_off = (int32_t)off; d.bits = h->bits;
+                if (off + nu > (int64_t)1 << 26 || n_cta > 32767) return false;
+                d.N = (int32_t)h->N; d.NT = h->NT; d.n_units = (int32_t)nu; d.bits = h->bits;
+                d.units_q = (int32_t)(nu / n_cta);
+                d.units_r_rot = (int32_t)(nu % n_cta) | (rot << 16);
+                rot = (int)((rot + nu % n_cta) % n_cta);
                 off += nu;
             }
             if ((int)deps.size() > DS_MAX_DEPS) return false;
             P.units_total = (int32_t)off;
-            P.units_q = (int32_t)(off / n_cta);
-            P.units_r = (int32_t)(off % n_cta);
             P.n_deps = (int)deps.size();
             for (size_t j = 0; j < deps.size(); ++j) P.deps[j] = (int16_t)deps[j];
             // every CTA's staged slabs must fit the shared-memory buffer
             for (int c = 0; c < n_cta; ++c) {
-                const int64_t ca = (int64_t)P.units_q * c + std::min<int64_t>(c, P.units_r);
-                const int64_t cb = ca + P.units_q + (c < P.units_r ? 1 : 0);
-                int64_t slabs = 0;
+                std::vector<int64_t> need;
                 for (int i = 0; i < P.op_count; ++i) {
-                    const int64_t o0 = P.ops[i].unit_off, n = P.ops[i].n_units;
-                    const int64_t u0 = std::max(ca, o0) - o0, u1 = std::min(cb, o0 + n) - o0;
-                    if (u0 < u1) slabs += (u1 - 1) / P.ops[i].NT - u0 / P.ops[i].NT + 1;
+                    const int64_t q = P.ops[i].units_q, r = P.ops[i].units_r_rot & 0xFFFF, ro = P.ops[i].units_r_rot >> 16;
+                    const int64_t sl = (c + ro) % n_cta;
+                    const int64_t u0 = q * sl + std::min(sl, r), u1 = u0 + q + (sl < r ? 1 : 0);
+                    if (u0 < u1)
+                        for (int64_t x = u0 / P.ops[i].NT; x <= (u1 - 1) / P.ops[i].NT; ++x) need.push_back(x);
                 }
-                if (slabs * ds_slab_bytes(M) > DS_XS_BYTES) return false;
+                std::sort(need.begin(), need.end());
+                const int64_t slabs = std::unique(need.begin(), need.end()) - need.begin();
+                if (slabs > DS_MAX_SLOTS || slabs * ds_slab_bytes(M) > DS_XS_BYTES) return false;
             }
             for (int i = first; i < last; ++i) writer[p->ops[i].dst] = i;
             phases.push_back(P);
@@ -743,10 +793,29 @@ int launch_decode_stack(const aq_stack_t* p, const StackPlan& plan, int M, aq_dt
         dp->device = dev;
         for (int i = 0; i < p->n_ops; ++i) dp->handles.push_back(p->ops[i].w);
         dp->phases_bytes = (phases.size() * sizeof(DsPhase) + 255) / 256 * 256;
+        std::vector<uint8_t> mini(phases.size() * sizeof(DsMiniPhase));
+        for (size_t i = 0; i < phases.size(); ++i) {
+            DsMiniPhase mph;
+            memset(&mph, 0, sizeof(mph));
+            mph.op_first = dp->n_mini_ops; mph.op_count = phases[i].op_count;
+            memcpy(mini.data() + i * sizeof(DsMiniPhase), &mph, sizeof(mph));
+            dp->n_mini_ops += phases[i].op_count;
+        }
+        for (size_t i = 0; i < phases.size(); ++i)
+            for (int j = 0; j < phases[i].op_count; ++j) {
+                DsMiniOp mop;
+                mop.frags = phases[i].ops[j].frags;
+                mop.q_bits = (uint32_t)phases[i].ops[j].units_q | ((uint32_t)phases[i].ops[j].bits << 28);
+                mop.r_rot = (uint32_t)phases[i].ops[j].units_r_rot;
+                const uint8_t* b = reinterpret_cast<const uint8_t*>(&mop);
+                mini.insert(mini.end(), b, b + sizeof(mop));
+            }
+        dp->mini_bytes = (mini.size() + 255) / 256 * 256;
         dp->cnt_bytes = ((size_t)p->n_ops * sizeof(uint32_t) + 255) / 256 * 256;
         dp->n_phases = (int)phases.size();
-        cudaError_t e = cudaMalloc(&dp->dev, dp->phases_bytes + dp->cnt_bytes);
+        cudaError_t e = cudaMalloc(&dp->dev, dp->phases_bytes + dp->mini_bytes + dp->cnt_bytes);
         if (e == cudaSuccess) e = cudaMemcpy(dp->dev, phases.data(), phases.size() * sizeof(DsPhase), cudaMemcpyHostToDevice);
+        if (e == cudaSuccess) e = cudaMemcpy(dp->dev + dp->phases_bytes, mini.data(), mini.size(), cudaMemcpyHostToDevice);
         if (e != cudaSuccess) { cudaGetLastError(); drop_plan(dp); *err = e; return -1; }
         if (g_plans.size() >= MAX_PLANS) {
             size_t oldest = 0;
@@ -761,7 +830,10 @@ int launch_decode_stack(const aq_stack_t* p, const StackPlan& plan, int M, aq_dt
 
     DsArgs a;
     a.phases = reinterpret_cast<const DsPhase*>(dp->dev);
-    a.cnt = reinterpret_cast<uint32_t*>(dp->dev + dp->phases_bytes);
+    a.mini_phases = reinterpret_cast<const DsMiniPhase*>(dp->dev + dp->phases_bytes);
+    a.mini_ops = reinterpret_cast<const DsMiniOp*>(dp->dev + dp->phases_bytes + (size_t)dp->n_phases * sizeof(DsMiniPhase));
+    a.n_mini_ops = dp->n_mini_ops;
+    a.cnt = reinterpret_cast<uint32_t*>(dp->dev + dp->phases_bytes + dp->mini_bytes);
     a.n_phases = dp->n_phases;
     a.M = M;
     cudaError_t e = cudaMemsetAsync(a.cnt, 0, dp->cnt_bytes, s);
