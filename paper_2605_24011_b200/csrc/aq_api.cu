@@ -187,12 +187,12 @@ static aq_status_t linear_common(aq_handle_t h, const void* x_dev, void* y_dev, 
         e = launch_gemv(h, x_dev, xdt, M, h->acc, ld, s);
         if (e == cudaSuccess) e = launch_finalize(h->acc, h->acc, ld, y_dev, ydt, M, h->N, s);
     } else if (ydt == AQ_F32) {
-        e = launch_gemm(h, x_dev, xdt, M, (float*)y_dev, h->N, false, s);
+        e = launch_gemm(h, x_dev, xdt, M, (float*)y_dev, h->N, nullptr, s);
     } else {
         float* tmp = nullptr;
         e = cudaMallocAsync(&tmp, (size_t)M * h->N * sizeof(float), s);
         if (e != cudaSuccess) { cudaGetLastError(); return AQ_ERR_ALLOC; }
-        e = launch_gemm(h, x_dev, xdt, M, tmp, h->N, false, s);
+        e = launch_gemm(h, x_dev, xdt, M, tmp, h->N, nullptr, s);
         if (e == cudaSuccess) e = launch_finalize(tmp, nullptr, h->N, y_dev, ydt, M, h->N, s);
         cudaFreeAsync(tmp, s);
     }

@@ -1,17 +1,22 @@
 // Prefill path (M > 8): dequantise-to-half + tensor-core GEMM on the packed
-// weights, out[m][n] (+)= sum_k x[m][k] w_hat[n][k]  (Appendix D: dequantise
-// on the fly inside the low-bit kernel; Eq. 1 for the decode).
+// weights, out[m][n] = (res[m][n]) + sum_k x[m][k] w_hat[n][k]  (Appendix D:
+// dequantise on the fly inside the low-bit kernel; Eq. 1 for the decode).
 //
 // Bound: tensor cores (dense contraction, 2 M flops per weight).  tcgen05
-// UMMA with the accumulator in TMEM:
-//   A (M side, 128)  = weight rows, dequantised by four warps from the packed
-//                      fragments into the K-major 128-byte-swizzled shared
-//                      memory layout the instruction reads,
+// UMMA with the accumulators in TMEM:
+//   A (M side, 128)   = weight rows, dequantised by eight warps from the packed
+//                       fragments into the K-major 128-byte-swizzled shared
+//                       memory layout the instruction reads,
 //   B (N side, <=256) = tokens, fetched by TMA with the same swizzle,
-//   D[128 lanes][tokens] fp32 in TMEM, read back with tcgen05.ld.
-// Warp roles: 0 = TMA / bulk-copy producer (+ TMEM allocation), 1..4 =
-// dequantise then epilogue, 5 = MMA issue.  Every mbarrier wait is bounded;
-// when one runs out the CTA raises a status word, drains and returns.
+//   D[128 lanes][tokens] fp32 in TMEM: two accumulators of up to 256 tokens, so
+//                       a weight is dequantised once per 512 tokens.
+// One persistent CTA per SM.  The work -- (row tile, token super-tile, 128-k
+// slab) triples, weighted by their accumulators -- is cut into equal contiguous
+// runs, one per CTA; a run that covers a tile's whole K stores its sums, any
+// other run adds them with red.add (the launcher zeroes the output first).
+// Warp roles: 0..7 = dequantise then epilogue, 8 = TMA / bulk-copy producer
+// (+ TMEM allocation), 9 = MMA issue.  Every mbarrier wait is bounded; when one
+// runs out the CTA raises a status word, drains and returns.
 #include <cuda.h>
 
 #include "aq_internal.h"
@@ -20,27 +25,66 @@
 namespace aq {
 
 constexpr int GM_ROWS = 128;       // weight rows per CTA tile (UMMA M)
-constexpr int GM_KSTAGE = 64;      // k per pipeline stage (one 128-byte swizzle atom of 16-bit elements)
-constexpr int GM_STAGES = 4;       // A/B ring depth
-constexpr int GM_PSTAGES = 2;      // packed-fragment ring depth (one k-slab of 128 per slot)
-constexpr int GM_THREADS = 192;
-constexpr int GM_MAX_TN = 256;     // tokens per CTA tile (UMMA N)
+constexpr int GM_KSTAGE = 64;      // k per A stage (one 128-byte swizzle atom of 16-bit elements)
+constexpr int GM_ASTAGES = 4;      // dequantised-weight ring (16 KB each)
+constexpr int GM_BSLOTS = 4;       // token ring: 256 tokens x 64 k = 32 KB each (one accumulator's share of a stage)
+constexpr int GM_PSTAGES = 2;      // packed-fragment ring (one k-slab of 128 per slot)
+constexpr int GM_DQ_WARPS = 8;
+constexpr int GM_THREADS = (GM_DQ_WARPS + 2) * 32;
+constexpr int GM_MAX_TN = 256;     // tokens per accumulator (UMMA N)
+constexpr int GM_B_BYTES = GM_MAX_TN * 128;
+constexpr int GM_A_BYTES = GM_ROWS * GM_KSTAGE * 2;
 constexpr uint32_t GM_SPIN_LIMIT = 40u * 1000u * 1000u;
 
 __device__ int g_gemm_status = 0;  // nonzero: a bounded wait ran out (code = which)
 
 struct GemmArgs {
     const uint8_t* frags;
-    float* out;
+    float* out;            // float32 [M][ldo]
+    const float* res;      // float32 [M][ldo] added once, or null
     int64_t ldo;
     int64_t N;
     int M;
-    int NT;          // 16-row tiles
-    int n_slabs;     // k-slabs of 128 (2 * KP)
-    int splits;
-    int tn;          // token tile = TMA box rows = UMMA N
-    int use_red;     // accumulate with red.add instead of plain stores
+    int NT;                // 16-row tiles
+    int n_slabs;           // 128-k slabs (K padded to 256)
+    int R;                 // row tiles of 128
+    int n_st;              // token super-tiles
+    int n2;                // the first n2 of them hold two accumulators, the others one
+    int st_tokens;         // tokens per super-tile (512 when M > 256)
+    int tn;                // TMA box rows: 256 when M > 256, else M rounded up to 16
 };
+
+// One contiguous piece of a CTA's run: slabs [s0, s1) of tile (rt, st).
+struct GemmSeg {
+    int rt, st, na, s0, s1;
+    int w0, w1;            // tokens (rounded up to 16) of the two accumulators
+};
+
+// Work is measured in slab-accumulators: a slab of a tile with two accumulators
+// counts 2.  Tiles are ordered super-tile-major, so the two-accumulator tiles come
+// first; run boundaries are even, hence whole slabs everywhere.
+__device__ __forceinline__ bool gemm_next_seg(long long& pos, long long hi, const GemmArgs& a, GemmSeg& sg) {
+    if (pos >= hi) return false;
+    const long long c2 = 2LL * a.n_slabs, reg2 = c2 * a.n2 * a.R;
+    long long t, end;
+    if (pos < reg2) {
+        t = pos / c2;
+        end = min(hi, (t + 1) * c2);
+        sg.na = 2; sg.s0 = (int)((pos - t * c2) >> 1); sg.s1 = (int)((end - t * c2) >> 1);
+    } else {
+        const long long t1 = (pos - reg2) / a.n_slabs, base = reg2 + t1 * a.n_slabs;
+        t = (long long)a.n2 * a.R + t1;
+        end = min(hi, base + a.n_slabs);
+        sg.na = 1; sg.s0 = (int)(pos - base); sg.s1 = (int)(end - base);
+    }
+    pos = end;
+    sg.st = (int)(t / a.R);
+    sg.rt = (int)(t - (long long)sg.st * a.R);
+    const int rem = a.M - sg.st * a.st_tokens;
+    if (sg.na == 2) { sg.w0 = GM_MAX_TN; sg.w1 = min(GM_MAX_TN, (rem - GM_MAX_TN + 15) & ~15); }
+    else { sg.w0 = min(a.tn, (rem + 15) & ~15); sg.w1 = 0; }
+    return true;
+}
 
 // ---- PTX wrappers -----------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -132,44 +176,54 @@ __device__ __forceinline__ uint32_t pack2(float a, float b) {
     }
 }
 
+// Two dequantised weights (k-adjacent, one row) as the 32-bit A-tile element.
+// p holds the two codes OR-ed into the mantissa of the half-precision constant
+// 128.0 (bf16) or 1024.0 (fp16) in each half.
+//   bf16: widen each half to fp32 (a shift / a mask), one FMA with the scale and
+//         with (min - 128 scale), round the pair to bf16;
+//   fp16: subtract 1024 (exact), one half2 FMA with scale and min.
+template <bool BF16>
+__device__ __forceinline__ uint32_t dequant_pair(uint32_t p, float d, float mb, __half2 d2, __half2 m2) {
+    if constexpr (BF16) {
+        const float f0 = __uint_as_float(p << 16), f1 = __uint_as_float(p & 0xffff0000u);
+        return pack2<true>(fmaf(f0, d, mb), fmaf(f1, d, mb));
+    } else {
+        const __half2 q = __hsub2(*reinterpret_cast<const __half2*>(&p), __float2half2_rn(1024.f));
+        const __half2 w = __hfma2(q, d2, m2);
+        return *reinterpret_cast<const uint32_t*>(&w);
+    }
+}
+
 template <int BITS, bool BF16>
 __global__ void __launch_bounds__(GM_THREADS, 1) gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
     constexpr int FB = frag_bytes(BITS);
-    constexpr int A_BYTES = GM_ROWS * GM_KSTAGE * 2;          // 16 KB
     constexpr int P_BYTES = 8 * FB;                           // packed fragments of one slab
+    constexpr uint32_t MAGIC = BF16 ? 0x43004300u : 0x64006400u;
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    const int tn = a.tn;
-    const int B_BYTES = tn * 128;
     uint8_t* sA = smem;
-    uint8_t* sB = sA + GM_STAGES * A_BYTES;
-    uint8_t* sP = sB + GM_STAGES * GM_MAX_TN * 128;
+    uint8_t* sB = sA + GM_ASTAGES * GM_A_BYTES;
+    uint8_t* sP = sB + GM_BSLOTS * GM_B_BYTES;
     uint64_t* bars = reinterpret_cast<uint64_t*>(sP + GM_PSTAGES * P_BYTES);
-    // bars: full[NS], empty[NS], pfull[NP], pempty[NP], accum
-    const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * GM_STAGES;
-    const uint32_t bar_pfull = bar_empty + 8 * GM_STAGES, bar_pempty = bar_pfull + 8 * GM_PSTAGES;
+    const uint32_t bar_afull = smem_u32(bars), bar_aempty = bar_afull + 8 * GM_ASTAGES;
+    const uint32_t bar_bfull = bar_aempty + 8 * GM_ASTAGES, bar_bempty = bar_bfull + 8 * GM_BSLOTS;
+    const uint32_t bar_pfull = bar_bempty + 8 * GM_BSLOTS, bar_pempty = bar_pfull + 8 * GM_PSTAGES;
     const uint32_t bar_accum = bar_pempty + 8 * GM_PSTAGES;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * GM_STAGES + 2 * GM_PSTAGES + 1);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * GM_ASTAGES + 2 * GM_BSLOTS + 2 * GM_PSTAGES + 1);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int n_tile = blockIdx.x, tok_tile = blockIdx.y, split = blockIdx.z;
-    const int slab0 = (int)(((int64_t)a.n_slabs * split) / a.splits);
-    const int slab1 = (int)(((int64_t)a.n_slabs * (split + 1)) / a.splits);
-    const int n_it = (slab1 - slab0) * 2;                     // k-stages of 64
-    const int rt0 = n_tile * 8;                               // first 16-row tile
-    const int n_rt = min(8, a.NT - rt0);                      // valid 16-row tiles in this CTA
-    uint32_t tmem_cols = 32;
-    while ((int)tmem_cols < tn) tmem_cols <<= 1;
+    const uint32_t tmem_cols = (a.n2 > 0) ? 512u : (a.tn <= 32 ? 32u : a.tn <= 64 ? 64u : a.tn <= 128 ? 128u : 256u);
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < GM_STAGES; ++s) { mbar_init(bar_full + 8 * s, 5); mbar_init(bar_empty + 8 * s, 1); }
-        for (int s = 0; s < GM_PSTAGES; ++s) { mbar_init(bar_pfull + 8 * s, 1); mbar_init(bar_pempty + 8 * s, 4); }
+        for (int s = 0; s < GM_ASTAGES; ++s) { mbar_init(bar_afull + 8 * s, GM_DQ_WARPS); mbar_init(bar_aempty + 8 * s, 1); }
+        for (int s = 0; s < GM_BSLOTS; ++s) { mbar_init(bar_bfull + 8 * s, 1); mbar_init(bar_bempty + 8 * s, 1); }
+        for (int s = 0; s < GM_PSTAGES; ++s) { mbar_init(bar_pfull + 8 * s, 1); mbar_init(bar_pempty + 8 * s, GM_DQ_WARPS); }
         mbar_init(bar_accum, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 0) {
+    if (warp == GM_DQ_WARPS) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(tmem_cols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
@@ -178,142 +232,184 @@ __global__ void __launch_bounds__(GM_THREADS, 1) gemm_kernel(const __grid_consta
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    if (n_it > 0) {
-        if (warp == 0) {
-            // ---------------- producer: packed fragments (bulk copies) + token tiles (TMA) --------------
-            if (lane == 0) {
-                bool ok = true;
-                for (int it = 0; it < n_it && ok; ++it) {
-                    if ((it & 1) == 0) {
-                        const int pi = it >> 1, ps = pi % GM_PSTAGES;
-                        ok = mbar_wait(bar_pempty + 8 * ps, ((pi / GM_PSTAGES) & 1) ^ 1, abort_flag, 1);
-                        if (!ok) break;
-                        const int slab = slab0 + pi;
-                        mbar_expect_tx(bar_pfull + 8 * ps, (uint32_t)(n_rt * FB));
-                        for (int ft = 0; ft < n_rt; ++ft) {
-                            const int64_t f = (((int64_t)(slab >> 1) * a.NT + rt0 + ft) * 2 + (slab & 1));
-                            bulk_load(smem_u32(sP + ps * P_BYTES + ft * FB), a.frags + f * FB, FB, bar_pfull + 8 * ps);
+    // this CTA's run, in slab-accumulators (even bounds)
+    const long long total = (long long)a.n_slabs * a.R * (2LL * a.n2 + (a.n_st - a.n2));
+    const long long run_lo = ((total * blockIdx.x) / gridDim.x) & ~1LL;
+    const long long run_hi = (blockIdx.x + 1 == gridDim.x) ? total : (((total * (blockIdx.x + 1)) / gridDim.x) & ~1LL);
+    GemmSeg sg;
+    long long pos = run_lo;
+
+    if (warp == GM_DQ_WARPS) {
+        // ---------------- producer: packed fragments (bulk copies) + token tiles (TMA) --------------
+        if (lane == 0) {
+            uint32_t pi = 0, bi = 0;
+            bool ok = true;
+            while (ok && gemm_next_seg(pos, run_hi, a, sg)) {
+                const int rt0 = sg.rt * 8, n_rt = min(8, a.NT - rt0);
+                for (int s = sg.s0; s < sg.s1 && ok; ++s) {
+                    const uint32_t ps = pi % GM_PSTAGES;
+                    ok = mbar_wait(bar_pempty + 8 * ps, ((pi / GM_PSTAGES) & 1) ^ 1, abort_flag, 1);
+                    if (!ok) break;
+                    mbar_expect_tx(bar_pfull + 8 * ps, (uint32_t)(n_rt * FB));
+                    for (int ft = 0; ft < n_rt; ++ft) {
+                        const int64_t f = (((int64_t)(s >> 1) * a.NT + rt0 + ft) * 2 + (s & 1));
+                        bulk_load(smem_u32(sP + ps * P_BYTES + ft * FB), a.frags + f * FB, FB, bar_pfull + 8 * ps);
+                    }
+                    ++pi;
+                    for (int h = 0; h < 2 && ok; ++h) {
+                        for (int j = 0; j < sg.na; ++j) {
+                            const uint32_t bs = bi % GM_BSLOTS;
+                            ok = mbar_wait(bar_bempty + 8 * bs, ((bi / GM_BSLOTS) & 1) ^ 1, abort_flag, 2);
+                            if (!ok) break;
+                            mbar_expect_tx(bar_bfull + 8 * bs, (uint32_t)(a.tn * 128));
+                            tma_load_2d(smem_u32(sB + bs * GM_B_BYTES), &tmap_x, (2 * s + h) * GM_KSTAGE,
+                                        sg.st * a.st_tokens + j * GM_MAX_TN, bar_bfull + 8 * bs);
+                            ++bi;
                         }
                     }
-                    const int s = it % GM_STAGES;
-                    ok = mbar_wait(bar_empty + 8 * s, ((it / GM_STAGES) & 1) ^ 1, abort_flag, 2);
-                    if (!ok) break;
-                    mbar_expect_tx(bar_full + 8 * s, (uint32_t)B_BYTES);
-                    tma_load_2d(smem_u32(sB + s * GM_MAX_TN * 128), &tmap_x, (slab0 * 2 + it) * GM_KSTAGE, tok_tile * tn,
-                                bar_full + 8 * s);
                 }
             }
-        } else if (warp == 5) {
-            // ---------------- MMA issue ----------------------------------------------------------------
-            if (lane == 0) {
-                const uint32_t idesc = (1u << 4) | ((BF16 ? 1u : 0u) << 7) | ((BF16 ? 1u : 0u) << 10) |
-                                       ((uint32_t)(tn >> 3) << 17) | ((uint32_t)(GM_ROWS >> 4) << 24);
-                bool ok = true;
-                for (int it = 0; it < n_it; ++it) {
-                    const int s = it % GM_STAGES;
-                    ok = mbar_wait(bar_full + 8 * s, (it / GM_STAGES) & 1, abort_flag, 3);
+        }
+    } else if (warp == GM_DQ_WARPS + 1) {
+        // ---------------- MMA issue ----------------------------------------------------------------
+        if (lane == 0) {
+            uint32_t ai = 0, bi = 0;
+            bool ok = true;
+            while (ok && gemm_next_seg(pos, run_hi, a, sg)) {
+                uint32_t idesc[2];
+                for (int j = 0; j < 2; ++j) {
+                    const uint32_t w = (j == 0) ? sg.w0 : sg.w1;
+                    idesc[j] = (1u << 4) | ((BF16 ? 1u : 0u) << 7) | ((BF16 ? 1u : 0u) << 10) | ((w >> 3) << 17) |
+                               ((uint32_t)(GM_ROWS >> 4) << 24);
+                }
+                for (int it = 2 * sg.s0; it < 2 * sg.s1 && ok; ++it) {
+                    const uint32_t as = ai % GM_ASTAGES;
+                    ok = mbar_wait(bar_afull + 8 * as, (ai / GM_ASTAGES) & 1, abort_flag, 3);
                     if (!ok) break;
-                    tc_fence_after();
-                    const uint64_t ad = make_smem_desc(smem_u32(sA + s * A_BYTES));
-                    const uint64_t bd = make_smem_desc(smem_u32(sB + s * GM_MAX_TN * 128));
+                    const uint64_t ad = make_smem_desc(smem_u32(sA + as * GM_A_BYTES));
+                    for (int j = 0; j < sg.na; ++j) {
+                        const uint32_t bs = bi % GM_BSLOTS;
+                        ok = mbar_wait(bar_bfull + 8 * bs, (bi / GM_BSLOTS) & 1, abort_flag, 4);
+                        if (!ok) break;
+                        tc_fence_after();
+                        const uint64_t bd = make_smem_desc(smem_u32(sB + bs * GM_B_BYTES));
 #pragma unroll
-                    for (int k = 0; k < GM_KSTAGE / 16; ++k)
-                        umma_f16(tmem_base, ad + 2 * k, bd + 2 * k, idesc, (it > 0 || k > 0) ? 1u : 0u);
-                    umma_commit(bar_empty + 8 * s);
+                        for (int k = 0; k < GM_KSTAGE / 16; ++k)
+                            umma_f16(tmem_base + (uint32_t)(j * GM_MAX_TN), ad + 2 * k, bd + 2 * k, idesc[j],
+                                     (it > 2 * sg.s0 || k > 0) ? 1u : 0u);
+                        umma_commit(bar_bempty + 8 * bs);
+                        ++bi;
+                    }
+                    if (!ok) break;
+                    umma_commit(bar_aempty + 8 * as);
+                    ++ai;
                 }
                 if (ok) umma_commit(bar_accum);
             }
-        } else {
-            // ---------------- dequantise (warps 1..4), then epilogue ------------------------------------
-            const int dw = warp - 1, g = lane >> 2, t = lane & 3;
-            bool ok = true;
-            for (int pi = 0; pi < (n_it >> 1) && ok; ++pi) {
-                const int ps = pi % GM_PSTAGES;
-                ok = mbar_wait(bar_pfull + 8 * ps, (pi / GM_PSTAGES) & 1, abort_flag, 4);
+        }
+    } else {
+        // ---------------- dequantise (warps 0..7), then epilogue -----------------------------------
+        const int dw = warp, g = lane >> 2, t = lane & 3;
+        uint32_t pi = 0, ai = 0, segc = 0;
+        bool ok = true;
+        while (ok && gemm_next_seg(pos, run_hi, a, sg)) {
+            const int rt0 = sg.rt * 8, n_rt = min(8, a.NT - rt0);
+            for (int s = sg.s0; s < sg.s1 && ok; ++s) {
+                const uint32_t ps = pi % GM_PSTAGES;
+                ok = mbar_wait(bar_pfull + 8 * ps, (pi / GM_PSTAGES) & 1, abort_flag, 5);
                 if (!ok) break;
-                LaneCodes<BITS> lc[2];
-                uint32_t dmw[2][2][4];   // [fragment][row half][block]: half2 (scale, min)
-#pragma unroll
-                for (int q = 0; q < 2; ++q) {
-                    const int ft = 2 * dw + q;
-                    const uint8_t* fb = sP + ps * P_BYTES + ft * FB;
-                    if (ft < n_rt) {
-                        load_lane_codes<BITS>(lc[q], fb, lane);
+                ++pi;
+                LaneCodes<BITS> lc;
+                uint32_t dmw[2][4];   // [row half][block]: half2 (scale, min)
+                {
+                    const uint8_t* fb = sP + ps * P_BYTES + dw * FB;
+                    if (dw < n_rt) {
+                        load_lane_codes<BITS>(lc, fb, lane);
                         const uint4 s0 = *reinterpret_cast<const uint4*>(fb + g * 16);
                         const uint4 s1 = *reinterpret_cast<const uint4*>(fb + (g + 8) * 16);
-                        dmw[q][0][0] = s0.x; dmw[q][0][1] = s0.y; dmw[q][0][2] = s0.z; dmw[q][0][3] = s0.w;
-                        dmw[q][1][0] = s1.x; dmw[q][1][1] = s1.y; dmw[q][1][2] = s1.z; dmw[q][1][3] = s1.w;
+                        dmw[0][0] = s0.x; dmw[0][1] = s0.y; dmw[0][2] = s0.z; dmw[0][3] = s0.w;
+                        dmw[1][0] = s1.x; dmw[1][1] = s1.y; dmw[1][2] = s1.z; dmw[1][3] = s1.w;
                     } else {
 #pragma unroll
-                        for (int i = 0; i < 2 * BITS; ++i) lc[q].w[i] = 0;
+                        for (int i = 0; i < 2 * BITS; ++i) lc.w[i] = 0;
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) { dmw[q][0][i] = 0; dmw[q][1][i] = 0; }
+                        for (int i = 0; i < 4; ++i) { dmw[0][i] = 0; dmw[1][i] = 0; }
                     }
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_pempty + 8 * ps);   // packed bytes are in registers now
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
-                    const int it = 2 * pi + h, s = it % GM_STAGES;
-                    ok = mbar_wait(bar_empty + 8 * s, ((it / GM_STAGES) & 1) ^ 1, abort_flag, 5);
+                    const uint32_t as = ai % GM_ASTAGES;
+                    ok = mbar_wait(bar_aempty + 8 * as, ((ai / GM_ASTAGES) & 1) ^ 1, abort_flag, 6);
                     if (!ok) break;
-                    uint8_t* At = sA + s * A_BYTES;
+                    ++ai;
+                    uint8_t* At = sA + as * GM_A_BYTES;
 #pragma unroll
-                    for (int q = 0; q < 2; ++q) {
+                    for (int jj = 0; jj < 2; ++jj) {
+                        const int j = 2 * h + jj;
 #pragma unroll
-                        for (int jj = 0; jj < 2; ++jj) {
-                            const int j = 2 * h + jj;
+                        for (int hi = 0; hi < 2; ++hi) {
+                            const __half2 dm = *reinterpret_cast<const __half2*>(&dmw[hi][j]);
+                            const float d = __low2float(dm);
+                            const float mb = fmaf(-128.f, d, __high2float(dm));
+                            const __half2 d2 = __low2half2(dm), m2 = __high2half2(dm);
+                            uint32_t o[4];
 #pragma unroll
-                            for (int hi = 0; hi < 2; ++hi) {
-                                const __half2 dm = *reinterpret_cast<const __half2*>(&dmw[q][hi][j]);
-                                const float d = __low2float(dm), m = __high2float(dm);
-                                uint32_t o[4];
-#pragma unroll
-                                for (int i = 0; i < 4; ++i) {
-                                    const uint32_t p = code_pair<BITS>(lc[q], j, hi, i, 0u);
-                                    o[i] = pack2<BF16>(fmaf(d, (float)(p & 0xffffu), m), fmaf(d, (float)(p >> 16), m));
-                                }
-                                const int row = (2 * dw + q) * 16 + g + 8 * hi;
-                                const int chunk = (jj * 4 + t) ^ (row & 7);
-                                *reinterpret_cast<uint4*>(At + (row >> 3) * 1024 + (row & 7) * 128 + chunk * 16) =
-                                    make_uint4(o[0], o[1], o[2], o[3]);
-                            }
+                            for (int i = 0; i < 4; ++i) o[i] = dequant_pair<BF16>(code_pair<BITS>(lc, j, hi, i, MAGIC), d, mb, d2, m2);
+                            const int row = dw * 16 + g + 8 * hi;
+                            const int chunk = (jj * 4 + t) ^ (row & 7);
+                            *reinterpret_cast<uint4*>(At + (row >> 3) * 1024 + (row & 7) * 128 + chunk * 16) =
+                                make_uint4(o[0], o[1], o[2], o[3]);
                         }
                     }
                     fence_async_smem();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(bar_full + 8 * s);
+                    if (lane == 0) mbar_arrive(bar_afull + 8 * as);
                 }
             }
-            // epilogue: TMEM lane quarter (warp % 4) -> out[token][row]
-            if (ok) ok = mbar_wait(bar_accum, 0, abort_flag, 6);
+            // epilogue: TMEM lane quarter (warp % 4) x this warp group's columns -> out[token][row]
+            if (ok) ok = mbar_wait(bar_accum, segc & 1, abort_flag, 7);
+            ++segc;
             if (ok) {
                 tc_fence_after();
-                const int lq = warp & 3;
-                const int64_t n = (int64_t)n_tile * GM_ROWS + lq * 32 + lane;
-                for (int c0 = 0; c0 < tn; c0 += 32) {
+                const int lq = dw & 3, grp = dw >> 2;
+                int c_lo, c_hi, acc;
+                if (sg.na == 2) { acc = grp; c_lo = 0; c_hi = grp ? sg.w1 : sg.w0; }
+                else {
+                    const int half = ((sg.w0 / 2 + 31) / 32) * 32;
+                    acc = 0; c_lo = grp ? min(half, sg.w0) : 0; c_hi = grp ? sg.w0 : min(half, sg.w0);
+                }
+                const bool whole = (sg.s0 == 0 && sg.s1 == a.n_slabs);
+                const bool add_res = (a.res != nullptr && sg.s0 == 0);
+                const int64_t n = (int64_t)sg.rt * GM_ROWS + lq * 32 + lane;
+                const int tok0 = sg.st * a.st_tokens + acc * GM_MAX_TN;
+                for (int c0 = c_lo; c0 < c_hi; c0 += 32) {
                     uint32_t v[32];
-                    tmem_ld32(tmem_base + ((uint32_t)(lq * 32) << 16) + (uint32_t)c0, v);
+                    tmem_ld32(tmem_base + ((uint32_t)(lq * 32) << 16) + (uint32_t)(acc * GM_MAX_TN + c0), v);
                     tmem_ld_wait();
                     if (n < a.N) {
 #pragma unroll
                         for (int j = 0; j < 32; ++j) {
-                            const int tok = tok_tile * tn + c0 + j;
-                            if (c0 + j < tn && tok < a.M) {
-                                float* o = a.out + (int64_t)tok * a.ldo + n;
-                                if (a.use_red) atomicAdd(o, __uint_as_float(v[j]));
-                                else *o = __uint_as_float(v[j]);
+                            const int tok = tok0 + c0 + j;
+                            if (c0 + j < c_hi && tok < a.M) {
+                                const int64_t o = (int64_t)tok * a.ldo + n;
+                                float val = __uint_as_float(v[j]);
+                                if (add_res) val += __ldg(a.res + o);
+                                if (whole) a.out[o] = val;
+                                else atomicAdd(a.out + o, val);
                             }
                         }
                     }
                 }
+                tc_fence_before();   // the next run's first MMA may overwrite the accumulators
             }
         }
     }
     tc_fence_before();
     __syncthreads();
     if (*abort_flag) __nanosleep(200000);   // let copies in flight land before the CTA's shared memory goes away
-    if (warp == 0) {
+    if (warp == GM_DQ_WARPS) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
     }
@@ -337,9 +433,9 @@ static EncodeTiledFn encode_fn() {
 }
 
 template <int BITS, bool BF16>
-static cudaError_t launch_one(const CUtensorMap& tm, const GemmArgs& a, dim3 grid, cudaStream_t s) {
+static cudaError_t launch_one(const CUtensorMap& tm, const GemmArgs& a, int grid, cudaStream_t s) {
     constexpr int FB = frag_bytes(BITS);
-    constexpr int SMEM = 1024 + GM_STAGES * (GM_ROWS * GM_KSTAGE * 2 + GM_MAX_TN * 128) + GM_PSTAGES * 8 * FB + 256;
+    constexpr int SMEM = 1024 + GM_ASTAGES * GM_A_BYTES + GM_BSLOTS * GM_B_BYTES + GM_PSTAGES * 8 * FB + 256;
     auto kern = gemm_kernel<BITS, BF16>;
     static bool configured = false;
     if (!configured) {
@@ -353,21 +449,33 @@ static cudaError_t launch_one(const CUtensorMap& tm, const GemmArgs& a, dim3 gri
 }
 
 cudaError_t launch_gemm(const aq_handle_s* h, const void* x, aq_dtype_t xdt, int M, float* out, int64_t ldo,
-                        bool accumulate, cudaStream_t s) {
+                        const float* res, cudaStream_t s) {
     EncodeTiledFn enc = encode_fn();
     if (!enc) return cudaErrorNotSupported;
     GemmArgs a;
-    a.frags = h->frags; a.out = out; a.ldo = ldo; a.N = h->N; a.M = M; a.NT = h->NT; a.n_slabs = h->KP * 2;
-    a.tn = (M >= GM_MAX_TN) ? GM_MAX_TN : ((M + 15) / 16) * 16;
-    const int n_tiles = (h->NT + 7) / 8;
-    const int tok_tiles = (M + a.tn - 1) / a.tn;
-    // split K until the grid covers the SMs (at most one slab-pair per split)
-    int splits = 1;
-    const int target = sm_count();
-    while (n_tiles * tok_tiles * splits < target && splits * 2 <= a.n_slabs / 2) splits *= 2;
-    a.splits = splits;
-    a.use_red = (accumulate || splits > 1) ? 1 : 0;
-    if (splits > 1 && !accumulate) {
+    a.frags = h->frags; a.out = out; a.res = res; a.ldo = ldo; a.N = h->N; a.M = M; a.NT = h->NT;
+    a.n_slabs = h->KP * 2;
+    a.R = (h->NT + 7) / 8;
+    if (M > GM_MAX_TN) {
+        a.tn = GM_MAX_TN; a.st_tokens = 2 * GM_MAX_TN;
+        a.n_st = (M + a.st_tokens - 1) / a.st_tokens;
+        a.n2 = (M - a.st_tokens * (a.n_st - 1) > GM_MAX_TN) ? a.n_st : a.n_st - 1;
+    } else {
+        a.tn = ((M + 15) / 16) * 16; a.st_tokens = a.tn; a.n_st = 1; a.n2 = 0;
+    }
+    const long long total = (long long)a.n_slabs * a.R * (2LL * a.n2 + (a.n_st - a.n2));
+    int grid = sm_count();
+    if (total / 2 < grid) grid = (int)(total / 2);
+    // runs that do not end on tile boundaries add into the output: it must start from zero
+    bool all_whole = true;
+    {
+        const long long c2 = 2LL * a.n_slabs, reg2 = c2 * a.n2 * a.R;
+        for (int c = 1; c < grid && all_whole; ++c) {
+            const long long b = ((total * c) / grid) & ~1LL;
+            all_whole = (b <= reg2) ? (b % c2 == 0) : ((b - reg2) % a.n_slabs == 0);
+        }
+    }
+    if (!all_whole) {
         cudaError_t e = cudaMemset2DAsync(out, (size_t)ldo * sizeof(float), 0, (size_t)h->N * sizeof(float), (size_t)M, s);
         if (e != cudaSuccess) return e;
     }
@@ -381,7 +489,6 @@ cudaError_t launch_gemm(const aq_handle_s* h, const void* x, aq_dtype_t xdt, int
                            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
-    const dim3 grid((unsigned)n_tiles, (unsigned)tok_tiles, (unsigned)splits);
     const bool bf = (xdt == AQ_BF16);
     switch (h->bits) {
         case 2: return bf ? launch_one<2, true>(tm, a, grid, s) : launch_one<2, false>(tm, a, grid, s);

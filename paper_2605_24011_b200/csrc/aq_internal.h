@@ -43,9 +43,10 @@ cudaError_t launch_gemv(const aq_handle_s* h, const void* x, aq_dtype_t xdt, int
 cudaError_t launch_finalize(const float* acc_in, float* acc_zero, int64_t ldacc, void* y, aq_dtype_t ydt,
                             int M, int64_t N, cudaStream_t s);
 
-// prefill path: out[m][n] (+)= sum_k x[m][k] w[n][k]; out fp32 [M][ldo]
+// prefill path: out[m][n] = (res ? res[m][n] : 0) + sum_k x[m][k] w[n][k]; out, res fp32 [M][ldo];
+// out need not be initialised (the launcher zeroes it when tiles are split over CTAs)
 cudaError_t launch_gemm(const aq_handle_s* h, const void* x, aq_dtype_t xdt, int M, float* out,
-                        int64_t ldo, bool accumulate, cudaStream_t s);
+                        int64_t ldo, const float* res, cudaStream_t s);
 
 // Where a program's buffers and staged inputs sit in the caller's workspace (aq_stack.cu).
 struct StackPlan {

@@ -153,12 +153,16 @@ static cudaError_t run_stack(const aq_stack_t* p, const StackPlan& plan, const T
         while (j < p->n_ops && same_input(p->ops[j], f)) {
             const aq_stack_op_t& o = p->ops[j];
             const int64_t N = p->buf_width[o.dst];
-            if (o.out_op == AQ_OUT_ADD) {
-                e = cudaMemcpyAsync(buf(o.dst), buf(o.res), (size_t)M * N * sizeof(float), cudaMemcpyDeviceToDevice, s);
-                if (e != cudaSuccess) return e;
+            const float* res = (o.out_op == AQ_OUT_ADD) ? buf(o.res) : nullptr;
+            if (decode) {
+                if (res) {
+                    e = cudaMemcpyAsync(buf(o.dst), res, (size_t)M * N * sizeof(float), cudaMemcpyDeviceToDevice, s);
+                    if (e != cudaSuccess) return e;
+                }
+                e = launch_gemv(o.w, stage, dt, M, buf(o.dst), N, s);
+            } else {
+                e = launch_gemm(o.w, stage, dt, M, buf(o.dst), N, res, s);
             }
-            if (decode) e = launch_gemv(o.w, stage, dt, M, buf(o.dst), N, s);
-            else e = launch_gemm(o.w, stage, dt, M, buf(o.dst), N, o.out_op == AQ_OUT_ADD, s);
             if (e != cudaSuccess) return e;
             o.w->last_stream = s;
             ++j;
