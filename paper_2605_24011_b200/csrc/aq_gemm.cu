@@ -14,10 +14,14 @@
 // slab) triples, weighted by their accumulators -- is cut into equal contiguous
 // runs, one per CTA; a run that covers a tile's whole K stores its sums, any
 // other run adds them with red.add (the launcher zeroes the output first).
-// Warp roles: 0..7 = dequantise then epilogue, 8 = TMA / bulk-copy producer
-// (+ TMEM allocation), 9 = MMA issue.  Every mbarrier wait is bounded; when one
+// Warp roles: 0..7 = dequantise then epilogue, 8 = token-tile TMA producer
+// (+ TMEM allocation), 9 = MMA issue, 10 = packed-fragment bulk-copy producer.
+// Epilogue: TMEM -> registers -> 32 x 32 fp32 chunks in shared memory (the idle
+// A ring) -> TMA tensor store, or TMA reduce-add when the tile is split.  Every mbarrier wait is bounded; when one
 // runs out the CTA raises a status word, drains and returns.
 #include <cuda.h>
+
+#include <cstring>
 
 #include "aq_internal.h"
 #include "aq_layout.cuh"
@@ -28,9 +32,9 @@ constexpr int GM_ROWS = 128;       // weight rows per CTA tile (UMMA M)
 constexpr int GM_KSTAGE = 64;      // k per A stage (one 128-byte swizzle atom of 16-bit elements)
 constexpr int GM_ASTAGES = 4;      // dequantised-weight ring (16 KB each)
 constexpr int GM_BSLOTS = 4;       // token ring: 256 tokens x 64 k = 32 KB each (one accumulator's share of a stage)
-constexpr int GM_PSTAGES = 2;      // packed-fragment ring (one k-slab of 128 per slot)
+constexpr int GM_PSTAGES = 3;      // packed-fragment ring (one k-slab of 128 per slot)
 constexpr int GM_DQ_WARPS = 8;
-constexpr int GM_THREADS = (GM_DQ_WARPS + 2) * 32;
+constexpr int GM_THREADS = (GM_DQ_WARPS + 3) * 32;
 constexpr int GM_MAX_TN = 256;     // tokens per accumulator (UMMA N)
 constexpr int GM_B_BYTES = GM_MAX_TN * 128;
 constexpr int GM_A_BYTES = GM_ROWS * GM_KSTAGE * 2;
@@ -52,6 +56,7 @@ struct GemmArgs {
     int n2;                // the first n2 of them hold two accumulators, the others one
     int st_tokens;         // tokens per super-tile (512 when M > 256)
     int tn;                // TMA box rows: 256 when M > 256, else M rounded up to 16
+    int tma_out;           // 1: the epilogue writes through the output tensor map (needs ldo % 4 == 0)
 };
 
 // One contiguous piece of a CTA's run: slabs [s0, s1) of tile (rt, st).
@@ -131,6 +136,17 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
 
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, uint32_t src, int c0, int c1) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(tm), "r"(src), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* tm, uint32_t src, int c0, int c1) {
+    asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(tm), "r"(src), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+template <int N> __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
@@ -195,7 +211,7 @@ __device__ __forceinline__ uint32_t dequant_pair(uint32_t p, float d, float mb, 
 }
 
 template <int BITS, bool BF16>
-__global__ void __launch_bounds__(GM_THREADS, 1) gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
+__global__ void __launch_bounds__(GM_THREADS, 1) gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_out, const GemmArgs a) {
     constexpr int FB = frag_bytes(BITS);
     constexpr int P_BYTES = 8 * FB;                           // packed fragments of one slab
     constexpr uint32_t MAGIC = BF16 ? 0x43004300u : 0x64006400u;
@@ -240,13 +256,32 @@ __global__ void __launch_bounds__(GM_THREADS, 1) gemm_kernel(const __grid_consta
     long long pos = run_lo;
 
     if (warp == GM_DQ_WARPS) {
-        // ---------------- producer: packed fragments (bulk copies) + token tiles (TMA) --------------
+        // ---------------- producer: token tiles (TMA) ---------------------------------------------
         if (lane == 0) {
-            uint32_t pi = 0, bi = 0;
+            uint32_t bi = 0;
+            bool ok = true;
+            while (ok && gemm_next_seg(pos, run_hi, a, sg)) {
+                for (int it = 2 * sg.s0; it < 2 * sg.s1 && ok; ++it) {
+                    for (int j = 0; j < sg.na; ++j) {
+                        const uint32_t bs = bi % GM_BSLOTS;
+                        ok = mbar_wait(bar_bempty + 8 * bs, ((bi / GM_BSLOTS) & 1) ^ 1, abort_flag, 2);
+                        if (!ok) break;
+                        mbar_expect_tx(bar_bfull + 8 * bs, (uint32_t)(a.tn * 128));
+                        tma_load_2d(smem_u32(sB + bs * GM_B_BYTES), &tmap_x, it * GM_KSTAGE,
+                                    sg.st * a.st_tokens + j * GM_MAX_TN, bar_bfull + 8 * bs);
+                        ++bi;
+                    }
+                }
+            }
+        }
+    } else if (warp == GM_DQ_WARPS + 2) {
+        // ---------------- producer: packed fragments (bulk copies) ----------------------------------
+        if (lane == 0) {
+            uint32_t pi = 0;
             bool ok = true;
             while (ok && gemm_next_seg(pos, run_hi, a, sg)) {
                 const int rt0 = sg.rt * 8, n_rt = min(8, a.NT - rt0);
-                for (int s = sg.s0; s < sg.s1 && ok; ++s) {
+                for (int s = sg.s0; s < sg.s1; ++s) {
                     const uint32_t ps = pi % GM_PSTAGES;
                     ok = mbar_wait(bar_pempty + 8 * ps, ((pi / GM_PSTAGES) & 1) ^ 1, abort_flag, 1);
                     if (!ok) break;
@@ -256,17 +291,6 @@ __global__ void __launch_bounds__(GM_THREADS, 1) gemm_kernel(const __grid_consta
                         bulk_load(smem_u32(sP + ps * P_BYTES + ft * FB), a.frags + f * FB, FB, bar_pfull + 8 * ps);
                     }
                     ++pi;
-                    for (int h = 0; h < 2 && ok; ++h) {
-                        for (int j = 0; j < sg.na; ++j) {
-                            const uint32_t bs = bi % GM_BSLOTS;
-                            ok = mbar_wait(bar_bempty + 8 * bs, ((bi / GM_BSLOTS) & 1) ^ 1, abort_flag, 2);
-                            if (!ok) break;
-                            mbar_expect_tx(bar_bfull + 8 * bs, (uint32_t)(a.tn * 128));
-                            tma_load_2d(smem_u32(sB + bs * GM_B_BYTES), &tmap_x, (2 * s + h) * GM_KSTAGE,
-                                        sg.st * a.st_tokens + j * GM_MAX_TN, bar_bfull + 8 * bs);
-                            ++bi;
-                        }
-                    }
                 }
             }
         }
@@ -312,7 +336,7 @@ __global__ void __launch_bounds__(GM_THREADS, 1) gemm_kernel(const __grid_consta
         const int dw = warp, g = lane >> 2, t = lane & 3;
         uint32_t pi = 0, ai = 0, segc = 0;
         bool ok = true;
-        while (ok && gemm_next_seg(pos, run_hi, a, sg)) {
+        while (gemm_next_seg(pos, run_hi, a, sg)) {   // (every warp walks every run, also after a failed wait: see the barrier below)
             const int rt0 = sg.rt * 8, n_rt = min(8, a.NT - rt0);
             for (int s = sg.s0; s < sg.s1 && ok; ++s) {
                 const uint32_t ps = pi % GM_PSTAGES;
@@ -382,30 +406,66 @@ __global__ void __launch_bounds__(GM_THREADS, 1) gemm_kernel(const __grid_consta
                 }
                 const bool whole = (sg.s0 == 0 && sg.s1 == a.n_slabs);
                 const bool add_res = (a.res != nullptr && sg.s0 == 0);
-                const int64_t n = (int64_t)sg.rt * GM_ROWS + lq * 32 + lane;
+                const int n0 = sg.rt * GM_ROWS + lq * 32;
+                const int64_t n = (int64_t)n0 + lane;
                 const int tok0 = sg.st * a.st_tokens + acc * GM_MAX_TN;
-                for (int c0 = c_lo; c0 < c_hi; c0 += 32) {
-                    uint32_t v[32];
-                    tmem_ld32(tmem_base + ((uint32_t)(lq * 32) << 16) + (uint32_t)(acc * GM_MAX_TN + c0), v);
-                    tmem_ld_wait();
-                    if (n < a.N) {
+                if (a.tma_out) {
+                    // the A ring is idle now (every MMA of the run has completed): two 4 KB chunks per warp
+                    float* stg = reinterpret_cast<float*>(sA + dw * 8192);
+                    int buf = 0;
+                    for (int c0 = c_lo; c0 < c_hi; c0 += 32, buf ^= 1) {
+                        uint32_t v[32];
+                        tmem_ld32(tmem_base + ((uint32_t)(lq * 32) << 16) + (uint32_t)(acc * GM_MAX_TN + c0), v);
+                        tmem_ld_wait();
+                        if (lane == 0) bulk_wait_read<1>();   // the copy that last read this chunk has left shared memory
+                        __syncwarp();
+                        float* chunk = stg + buf * 1024;      // [32 tokens][32 rows]
 #pragma unroll
                         for (int j = 0; j < 32; ++j) {
-                            const int tok = tok0 + c0 + j;
-                            if (c0 + j < c_hi && tok < a.M) {
-                                const int64_t o = (int64_t)tok * a.ldo + n;
-                                float val = __uint_as_float(v[j]);
-                                if (add_res) val += __ldg(a.res + o);
-                                if (whole) a.out[o] = val;
-                                else atomicAdd(a.out + o, val);
+                            float val = __uint_as_float(v[j]);
+                            if (add_res) {
+                                const int tok = tok0 + c0 + j;
+                                if (tok < a.M && n < a.N) val += __ldg(a.res + (int64_t)tok * a.ldo + n);
+                            }
+                            chunk[j * 32 + lane] = val;
+                        }
+                        fence_async_smem();
+                        __syncwarp();
+                        if (lane == 0) {   // rows / tokens past the end of the tensor are clipped by the copy
+                            if (whole) tma_store_2d(&tmap_out, smem_u32(chunk), n0, tok0 + c0);
+                            else tma_reduce_add_2d(&tmap_out, smem_u32(chunk), n0, tok0 + c0);
+                            bulk_commit();
+                        }
+                    }
+                    if (lane == 0) bulk_wait_read<0>();       // the A ring is written again right after
+                    __syncwarp();
+                } else {
+                    for (int c0 = c_lo; c0 < c_hi; c0 += 32) {
+                        uint32_t v[32];
+                        tmem_ld32(tmem_base + ((uint32_t)(lq * 32) << 16) + (uint32_t)(acc * GM_MAX_TN + c0), v);
+                        tmem_ld_wait();
+                        if (n < a.N) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) {
+                                const int tok = tok0 + c0 + j;
+                                if (c0 + j < c_hi && tok < a.M) {
+                                    const int64_t o = (int64_t)tok * a.ldo + n;
+                                    float val = __uint_as_float(v[j]);
+                                    if (add_res) val += __ldg(a.res + o);
+                                    if (whole) a.out[o] = val;
+                                    else atomicAdd(a.out + o, val);
+                                }
                             }
                         }
                     }
                 }
                 tc_fence_before();   // the next run's first MMA may overwrite the accumulators
             }
+            // the chunks staged above live in the A ring: nobody refills it before everybody has left the epilogue
+            asm volatile("bar.sync 1, %0;" ::"n"(GM_DQ_WARPS * 32) : "memory");
         }
     }
+    if (warp < GM_DQ_WARPS && lane == 0) bulk_wait_all<0>();   // this thread's output copies are complete
     tc_fence_before();
     __syncthreads();
     if (*abort_flag) __nanosleep(200000);   // let copies in flight land before the CTA's shared memory goes away
@@ -433,7 +493,7 @@ static EncodeTiledFn encode_fn() {
 }
 
 template <int BITS, bool BF16>
-static cudaError_t launch_one(const CUtensorMap& tm, const GemmArgs& a, int grid, cudaStream_t s) {
+static cudaError_t launch_one(const CUtensorMap& tm, const CUtensorMap& tmo, const GemmArgs& a, int grid, cudaStream_t s) {
     constexpr int FB = frag_bytes(BITS);
     constexpr int SMEM = 1024 + GM_ASTAGES * GM_A_BYTES + GM_BSLOTS * GM_B_BYTES + GM_PSTAGES * 8 * FB + 256;
     auto kern = gemm_kernel<BITS, BF16>;
@@ -443,7 +503,7 @@ static cudaError_t launch_one(const CUtensorMap& tm, const GemmArgs& a, int grid
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    kern<<<grid, GM_THREADS, SMEM, s>>>(tm, a);
+    kern<<<grid, GM_THREADS, SMEM, s>>>(tm, tmo, a);
     count_launch();
     return cudaGetLastError();
 }
@@ -489,11 +549,23 @@ cudaError_t launch_gemm(const aq_handle_s* h, const void* x, aq_dtype_t xdt, int
                            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+    // the output as a tensor [M][N] of float32 for the epilogue's 32 x 32 copies (row pitch must be 16-byte aligned)
+    CUtensorMap tmo;
+    memset(&tmo, 0, sizeof(tmo));
+    a.tma_out = 0;
+    if (ldo % 4 == 0 && (reinterpret_cast<uintptr_t>(out) & 15u) == 0) {
+        const cuuint64_t odims[2] = {(cuuint64_t)h->N, (cuuint64_t)M};
+        const cuuint64_t ostrides[1] = {(cuuint64_t)ldo * 4};
+        const cuuint32_t obox[2] = {32, 32};
+        if (enc(&tmo, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, out, odims, ostrides, obox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS)
+            a.tma_out = 1;
+    }
     const bool bf = (xdt == AQ_BF16);
     switch (h->bits) {
-        case 2: return bf ? launch_one<2, true>(tm, a, grid, s) : launch_one<2, false>(tm, a, grid, s);
-        case 3: return bf ? launch_one<3, true>(tm, a, grid, s) : launch_one<3, false>(tm, a, grid, s);
-        default: return bf ? launch_one<4, true>(tm, a, grid, s) : launch_one<4, false>(tm, a, grid, s);
+        case 2: return bf ? launch_one<2, true>(tm, tmo, a, grid, s) : launch_one<2, false>(tm, tmo, a, grid, s);
+        case 3: return bf ? launch_one<3, true>(tm, tmo, a, grid, s) : launch_one<3, false>(tm, tmo, a, grid, s);
+        default: return bf ? launch_one<4, true>(tm, tmo, a, grid, s) : launch_one<4, false>(tm, tmo, a, grid, s);
     }
 }
 
