@@ -404,8 +404,9 @@ __global__ void __launch_bounds__(GM_THREADS, 1) gemm_kernel(const __grid_consta
                     const int half = ((sg.w0 / 2 + 31) / 32) * 32;
                     acc = 0; c_lo = grp ? min(half, sg.w0) : 0; c_hi = grp ? sg.w0 : min(half, sg.w0);
                 }
-                const bool whole = (sg.s0 == 0 && sg.s1 == a.n_slabs);
-                const bool add_res = (a.res != nullptr && sg.s0 == 0);
+                // with a residual the launcher has copied it into out: every run then adds on top of it
+                const bool whole = (sg.s0 == 0 && sg.s1 == a.n_slabs) && (a.res == nullptr || !a.tma_out);
+                const bool add_res = (a.res != nullptr && sg.s0 == 0 && !a.tma_out);
                 const int n0 = sg.rt * GM_ROWS + lq * 32;
                 const int64_t n = (int64_t)n0 + lane;
                 const int tok0 = sg.st * a.st_tokens + acc * GM_MAX_TN;
@@ -421,14 +422,7 @@ __global__ void __launch_bounds__(GM_THREADS, 1) gemm_kernel(const __grid_consta
                         __syncwarp();
                         float* chunk = stg + buf * 1024;      // [32 tokens][32 rows]
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            float val = __uint_as_float(v[j]);
-                            if (add_res) {
-                                const int tok = tok0 + c0 + j;
-                                if (tok < a.M && n < a.N) val += __ldg(a.res + (int64_t)tok * a.ldo + n);
-                            }
-                            chunk[j * 32 + lane] = val;
-                        }
+                        for (int j = 0; j < 32; ++j) chunk[j * 32 + lane] = __uint_as_float(v[j]);
                         fence_async_smem();
                         __syncwarp();
                         if (lane == 0) {   // rows / tokens past the end of the tensor are clipped by the copy
@@ -526,19 +520,6 @@ cudaError_t launch_gemm(const aq_handle_s* h, const void* x, aq_dtype_t xdt, int
     const long long total = (long long)a.n_slabs * a.R * (2LL * a.n2 + (a.n_st - a.n2));
     int grid = sm_count();
     if (total / 2 < grid) grid = (int)(total / 2);
-    // runs that do not end on tile boundaries add into the output: it must start from zero
-    bool all_whole = true;
-    {
-        const long long c2 = 2LL * a.n_slabs, reg2 = c2 * a.n2 * a.R;
-        for (int c = 1; c < grid && all_whole; ++c) {
-            const long long b = ((total * c) / grid) & ~1LL;
-            all_whole = (b <= reg2) ? (b % c2 == 0) : ((b - reg2) % a.n_slabs == 0);
-        }
-    }
-    if (!all_whole) {
-        cudaError_t e = cudaMemset2DAsync(out, (size_t)ldo * sizeof(float), 0, (size_t)h->N * sizeof(float), (size_t)M, s);
-        if (e != cudaSuccess) return e;
-    }
     CUtensorMap tm;
     const cuuint64_t dims[2] = {(cuuint64_t)h->K, (cuuint64_t)M};
     const cuuint64_t strides[1] = {(cuuint64_t)h->K * 2};
@@ -560,6 +541,24 @@ cudaError_t launch_gemm(const aq_handle_s* h, const void* x, aq_dtype_t xdt, int
         if (enc(&tmo, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, out, odims, ostrides, obox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                 CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS)
             a.tma_out = 1;
+    }
+    // What out holds before the kernel: the residual when there is one (every run then adds to it);
+    // else zeros when some run does not cover a whole tile; else nothing.
+    if (res && a.tma_out) {
+        cudaError_t e = cudaMemcpy2DAsync(out, (size_t)ldo * sizeof(float), res, (size_t)ldo * sizeof(float),
+                                          (size_t)h->N * sizeof(float), (size_t)M, cudaMemcpyDeviceToDevice, s);
+        if (e != cudaSuccess) return e;
+    } else {
+        bool all_whole = true;
+        const long long c2 = 2LL * a.n_slabs, reg2 = c2 * a.n2 * a.R;
+        for (int c = 1; c < grid && all_whole; ++c) {
+            const long long b = ((total * c) / grid) & ~1LL;
+            all_whole = (b <= reg2) ? (b % c2 == 0) : ((b - reg2) % a.n_slabs == 0);
+        }
+        if (!all_whole) {
+            cudaError_t e = cudaMemset2DAsync(out, (size_t)ldo * sizeof(float), 0, (size_t)h->N * sizeof(float), (size_t)M, s);
+            if (e != cudaSuccess) return e;
+        }
     }
     const bool bf = (xdt == AQ_BF16);
     switch (h->bits) {

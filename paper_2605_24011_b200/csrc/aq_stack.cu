@@ -9,6 +9,7 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
+#include <algorithm>
 #include <vector>
 
 #include "aq_internal.h"
@@ -82,35 +83,57 @@ __global__ void narrow_kernel(const float* __restrict__ x, T* __restrict__ out, 
     if (i < n) out[i] = from_f32<T>(x[i]);
 }
 
-// One CTA per token row: x[m][k] = round(transform(src[m][k])).
+// Rounds four values and stores them as one 8-byte word.
+template <typename T>
+__device__ __forceinline__ void store_round4(T* o, const float4& v) {
+    const T a = from_f32<T>(v.x), b = from_f32<T>(v.y), c = from_f32<T>(v.z), d = from_f32<T>(v.w);
+    uint2 r;
+    r.x = (uint32_t)*reinterpret_cast<const uint16_t*>(&a) | ((uint32_t)*reinterpret_cast<const uint16_t*>(&b) << 16);
+    r.y = (uint32_t)*reinterpret_cast<const uint16_t*>(&c) | ((uint32_t)*reinterpret_cast<const uint16_t*>(&d) << 16);
+    *reinterpret_cast<uint2*>(o) = r;
+}
+
+// x[m][k] = round(transform(src[m][k])); K is a multiple of 32, rows are 16-byte aligned.
+// RMS scaling: one CTA per token row.  The other two forms have no row-wide term and
+// run as a flat grid over groups of four elements (blockIdx.y = 0).
 template <typename T>
 __global__ void __launch_bounds__(256) stage_kernel(const float* __restrict__ src, const float* __restrict__ src2,
-                                                    int in_op, int64_t K, T* __restrict__ x) {
-    const int64_t m = blockIdx.x;
-    const float* s = src + m * K;
-    T* o = x + m * K;
-    float scale = 1.f;
-    if (in_op == AQ_IN_RMSNORM) {
-        __shared__ float red[8];
-        float ss = 0.f;
-        for (int64_t k = threadIdx.x; k < K; k += 256) ss = fmaf(s[k], s[k], ss);
-#pragma unroll
-        for (int d = 16; d > 0; d >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, d);
-        if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
-        __syncthreads();
-        float tot = 0.f;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) tot += red[i];
-        scale = rsqrtf(tot / (float)K + 1e-6f);
-    }
-    if (in_op == AQ_IN_SILU_MUL) {
-        const float* s2 = src2 + m * K;
-        for (int64_t k = threadIdx.x; k < K; k += 256) {
-            const float g = s[k];
-            o[k] = from_f32<T>(g / (1.f + expf(-g)) * s2[k]);
+                                                    int in_op, int64_t K, int64_t total4, T* __restrict__ x) {
+    if (in_op != AQ_IN_RMSNORM) {
+        const float4* s4 = reinterpret_cast<const float4*>(src);
+        const float4* t4 = reinterpret_cast<const float4*>(src2);
+        for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < total4; i += (int64_t)gridDim.x * 256) {
+            float4 v = s4[i];
+            if (in_op == AQ_IN_SILU_MUL) {
+                const float4 u = t4[i];
+                v.x = v.x / (1.f + expf(-v.x)) * u.x; v.y = v.y / (1.f + expf(-v.y)) * u.y;
+                v.z = v.z / (1.f + expf(-v.z)) * u.z; v.w = v.w / (1.f + expf(-v.w)) * u.w;
+            }
+            store_round4<T>(x + 4 * i, v);
         }
-    } else {
-        for (int64_t k = threadIdx.x; k < K; k += 256) o[k] = from_f32<T>(s[k] * scale);
+        return;
+    }
+    const int64_t m = blockIdx.x;
+    const float4* s4 = reinterpret_cast<const float4*>(src + m * K);
+    T* o = x + m * K;
+    const int64_t q4 = K >> 2;
+    __shared__ float red[8];
+    float ss = 0.f;
+    for (int64_t k = threadIdx.x; k < q4; k += 256) {
+        const float4 v = s4[k];
+        ss = fmaf(v.x, v.x, ss); ss = fmaf(v.y, v.y, ss); ss = fmaf(v.z, v.z, ss); ss = fmaf(v.w, v.w, ss);
+    }
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, d);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    float tot = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) tot += red[i];
+    const float scale = rsqrtf(tot / (float)K + 1e-6f);
+    for (int64_t k = threadIdx.x; k < q4; k += 256) {
+        const float4 v = s4[k];
+        store_round4<T>(o + 4 * k, make_float4(v.x * scale, v.y * scale, v.z * scale, v.w * scale));
     }
 }
 
@@ -147,7 +170,11 @@ static cudaError_t run_stack(const aq_stack_t* p, const StackPlan& plan, const T
         const aq_stack_op_t& f = p->ops[i];
         const int64_t K = p->buf_width[f.src];
         T* stage = reinterpret_cast<T*>(ws + plan.in_off[i]);
-        stage_kernel<T><<<M, 256, 0, s>>>(buf(f.src), f.in_op == AQ_IN_SILU_MUL ? buf(f.src2) : nullptr, f.in_op, K, stage);
+        {
+            const int64_t total4 = (int64_t)M * K / 4;
+            const unsigned g = (f.in_op == AQ_IN_RMSNORM) ? (unsigned)M : (unsigned)std::min<int64_t>((total4 + 255) / 256, 4 * 148);
+            stage_kernel<T><<<g, 256, 0, s>>>(buf(f.src), f.in_op == AQ_IN_SILU_MUL ? buf(f.src2) : nullptr, f.in_op, K, total4, stage);
+        }
         count_launch();
         int j = i;
         while (j < p->n_ops && same_input(p->ops[j], f)) {
