@@ -42,26 +42,37 @@ constexpr uint32_t GM_SPIN_LIMIT = 40u * 1000u * 1000u;
 
 __device__ int g_gemm_status = 0;  // nonzero: a bounded wait ran out (code = which)
 
-struct GemmArgs {
+constexpr int GM_MAX_OPS = 4;      // matrices that share one input (q|k|v, gate|up) run as one launch
+
+struct GemmOp {
     const uint8_t* frags;
     float* out;            // float32 [M][ldo]
     const float* res;      // float32 [M][ldo] added once, or null
     int64_t ldo;
-    int64_t N;
-    int M;
+    int N;
     int NT;                // 16-row tiles
-    int n_slabs;           // 128-k slabs (K padded to 256)
     int R;                 // row tiles of 128
+    int bits;
+};
+
+struct GemmArgs {
+    GemmOp op[GM_MAX_OPS];
+    int n_ops;
+    int Rtot;              // row tiles of 128 over all ops
+    int M;
+    int n_slabs;           // 128-k slabs (K padded to 256)
     int n_st;              // token super-tiles
     int n2;                // the first n2 of them hold two accumulators, the others one
     int st_tokens;         // tokens per super-tile (512 when M > 256)
     int tn;                // TMA box rows: 256 when M > 256, else M rounded up to 16
-    int tma_out;           // 1: the epilogue writes through the output tensor map (needs ldo % 4 == 0)
+    int tma_out;           // 1: the epilogue writes through the output tensor maps (needs ldo % 4 == 0)
 };
+
+struct GemmOutMaps { CUtensorMap m[GM_MAX_OPS]; };
 
 // One contiguous piece of a CTA's run: slabs [s0, s1) of tile (rt, st).
 struct GemmSeg {
-    int rt, st, na, s0, s1;
+    int op, rt, st, na, s0, s1;   // rt: row tile inside matrix op
     int w0, w1;            // tokens (rounded up to 16) of the two accumulators
 };
 
@@ -70,7 +81,7 @@ struct GemmSeg {
 // first; run boundaries are even, hence whole slabs everywhere.
 __device__ __forceinline__ bool gemm_next_seg(long long& pos, long long hi, const GemmArgs& a, GemmSeg& sg) {
     if (pos >= hi) return false;
-    const long long c2 = 2LL * a.n_slabs, reg2 = c2 * a.n2 * a.R;
+    const long long c2 = 2LL * a.n_slabs, reg2 = c2 * a.n2 * a.Rtot;
     long long t, end;
     if (pos < reg2) {
         t = pos / c2;
@@ -78,13 +89,16 @@ __device__ __forceinline__ bool gemm_next_seg(long long& pos, long long hi, cons
         sg.na = 2; sg.s0 = (int)((pos - t * c2) >> 1); sg.s1 = (int)((end - t * c2) >> 1);
     } else {
         const long long t1 = (pos - reg2) / a.n_slabs, base = reg2 + t1 * a.n_slabs;
-        t = (long long)a.n2 * a.R + t1;
+        t = (long long)a.n2 * a.Rtot + t1;
         end = min(hi, base + a.n_slabs);
         sg.na = 1; sg.s0 = (int)(pos - base); sg.s1 = (int)(end - base);
     }
     pos = end;
-    sg.st = (int)(t / a.R);
-    sg.rt = (int)(t - (long long)sg.st * a.R);
+    sg.st = (int)(t / a.Rtot);
+    int r = (int)(t - (long long)sg.st * a.Rtot);
+    sg.op = 0;
+    while (sg.op + 1 < a.n_ops && r >= a.op[sg.op].R) { r -= a.op[sg.op].R; ++sg.op; }
+    sg.rt = r;
     const int rem = a.M - sg.st * a.st_tokens;
     if (sg.na == 2) { sg.w0 = GM_MAX_TN; sg.w1 = min(GM_MAX_TN, (rem - GM_MAX_TN + 15) & ~15); }
     else { sg.w0 = min(a.tn, (rem + 15) & ~15); sg.w1 = 0; }
@@ -210,11 +224,67 @@ __device__ __forceinline__ uint32_t dequant_pair(uint32_t p, float d, float mb, 
     }
 }
 
+// One dequantise warp's share of a k-slab: its fragment (16 rows x 128 k) becomes
+// rows 16 dw .. 16 dw + 15 of two A stages.  `have` is false for row tiles past the
+// end of the matrix (zeros are written).  Returns false when a wait ran out.
 template <int BITS, bool BF16>
-__global__ void __launch_bounds__(GM_THREADS, 1) gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_out, const GemmArgs a) {
+__device__ __forceinline__ bool dequant_slab(const uint8_t* slab, bool have, int dw, int lane, uint8_t* sA, uint32_t bar_pempty_slot,
+                                             uint32_t bar_aempty, uint32_t bar_afull, uint32_t& ai, volatile int* abort_flag) {
     constexpr int FB = frag_bytes(BITS);
-    constexpr int P_BYTES = 8 * FB;                           // packed fragments of one slab
     constexpr uint32_t MAGIC = BF16 ? 0x43004300u : 0x64006400u;
+    const int g = lane >> 2, t = lane & 3;
+    LaneCodes<BITS> lc;
+    uint32_t dmw[2][4];   // [row half][block]: half2 (scale, min)
+    {
+        const uint8_t* fb = slab + dw * FB;
+        if (have) {
+            load_lane_codes<BITS>(lc, fb, lane);
+            const uint4 s0 = *reinterpret_cast<const uint4*>(fb + g * 16);
+            const uint4 s1 = *reinterpret_cast<const uint4*>(fb + (g + 8) * 16);
+            dmw[0][0] = s0.x; dmw[0][1] = s0.y; dmw[0][2] = s0.z; dmw[0][3] = s0.w;
+            dmw[1][0] = s1.x; dmw[1][1] = s1.y; dmw[1][2] = s1.z; dmw[1][3] = s1.w;
+        } else {
+#pragma unroll
+            for (int i = 0; i < 2 * BITS; ++i) lc.w[i] = 0;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { dmw[0][i] = 0; dmw[1][i] = 0; }
+        }
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar_pempty_slot);   // packed bytes are in registers now
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const uint32_t as = ai % GM_ASTAGES;
+        if (!mbar_wait(bar_aempty + 8 * as, ((ai / GM_ASTAGES) & 1) ^ 1, abort_flag, 6)) return false;
+        ++ai;
+        uint8_t* At = sA + as * GM_A_BYTES;
+#pragma unroll
+        for (int jj = 0; jj < 2; ++jj) {
+            const int j = 2 * h + jj;
+#pragma unroll
+            for (int hi = 0; hi < 2; ++hi) {
+                const __half2 dm = *reinterpret_cast<const __half2*>(&dmw[hi][j]);
+                const float d = __low2float(dm);
+                const float mb = fmaf(-128.f, d, __high2float(dm));
+                const __half2 d2 = __low2half2(dm), m2 = __high2half2(dm);
+                uint32_t o[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) o[i] = dequant_pair<BF16>(code_pair<BITS>(lc, j, hi, i, MAGIC), d, mb, d2, m2);
+                const int row = dw * 16 + g + 8 * hi;
+                const int chunk = (jj * 4 + t) ^ (row & 7);
+                *reinterpret_cast<uint4*>(At + (row >> 3) * 1024 + (row & 7) * 128 + chunk * 16) = make_uint4(o[0], o[1], o[2], o[3]);
+            }
+        }
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_afull + 8 * as);
+    }
+    return true;
+}
+
+template <bool BF16>
+__global__ void __launch_bounds__(GM_THREADS, 1) gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ GemmOutMaps tmap_out, const GemmArgs a) {
+    constexpr int P_BYTES = 8 * frag_bytes(4);                // packed fragments of one slab (largest width)
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* sA = smem;
@@ -249,7 +319,7 @@ __global__ void __launch_bounds__(GM_THREADS, 1) gemm_kernel(const __grid_consta
     const uint32_t tmem_base = *tmem_slot;
 
     // this CTA's run, in slab-accumulators (even bounds)
-    const long long total = (long long)a.n_slabs * a.R * (2LL * a.n2 + (a.n_st - a.n2));
+    const long long total = (long long)a.n_slabs * a.Rtot * (2LL * a.n2 + (a.n_st - a.n2));
     const long long run_lo = ((total * blockIdx.x) / gridDim.x) & ~1LL;
     const long long run_hi = (blockIdx.x + 1 == gridDim.x) ? total : (((total * (blockIdx.x + 1)) / gridDim.x) & ~1LL);
     GemmSeg sg;
@@ -280,15 +350,17 @@ __global__ void __launch_bounds__(GM_THREADS, 1) gemm_kernel(const __grid_consta
             uint32_t pi = 0;
             bool ok = true;
             while (ok && gemm_next_seg(pos, run_hi, a, sg)) {
-                const int rt0 = sg.rt * 8, n_rt = min(8, a.NT - rt0);
+                const GemmOp& op = a.op[sg.op];
+                const int rt0 = sg.rt * 8, n_rt = min(8, op.NT - rt0);
+                const int FB = frag_bytes(op.bits);
                 for (int s = sg.s0; s < sg.s1; ++s) {
                     const uint32_t ps = pi % GM_PSTAGES;
                     ok = mbar_wait(bar_pempty + 8 * ps, ((pi / GM_PSTAGES) & 1) ^ 1, abort_flag, 1);
                     if (!ok) break;
                     mbar_expect_tx(bar_pfull + 8 * ps, (uint32_t)(n_rt * FB));
                     for (int ft = 0; ft < n_rt; ++ft) {
-                        const int64_t f = (((int64_t)(s >> 1) * a.NT + rt0 + ft) * 2 + (s & 1));
-                        bulk_load(smem_u32(sP + ps * P_BYTES + ft * FB), a.frags + f * FB, FB, bar_pfull + 8 * ps);
+                        const int64_t f = (((int64_t)(s >> 1) * op.NT + rt0 + ft) * 2 + (s & 1));
+                        bulk_load(smem_u32(sP + ps * P_BYTES + ft * FB), op.frags + f * FB, FB, bar_pfull + 8 * ps);
                     }
                     ++pi;
                 }
@@ -333,64 +405,21 @@ __global__ void __launch_bounds__(GM_THREADS, 1) gemm_kernel(const __grid_consta
         }
     } else {
         // ---------------- dequantise (warps 0..7), then epilogue -----------------------------------
-        const int dw = warp, g = lane >> 2, t = lane & 3;
+        const int dw = warp;
         uint32_t pi = 0, ai = 0, segc = 0;
         bool ok = true;
         while (gemm_next_seg(pos, run_hi, a, sg)) {   // (every warp walks every run, also after a failed wait: see the barrier below)
-            const int rt0 = sg.rt * 8, n_rt = min(8, a.NT - rt0);
+            const GemmOp& op = a.op[sg.op];
+            const int n_rt = min(8, op.NT - sg.rt * 8);
             for (int s = sg.s0; s < sg.s1 && ok; ++s) {
                 const uint32_t ps = pi % GM_PSTAGES;
                 ok = mbar_wait(bar_pfull + 8 * ps, (pi / GM_PSTAGES) & 1, abort_flag, 5);
                 if (!ok) break;
                 ++pi;
-                LaneCodes<BITS> lc;
-                uint32_t dmw[2][4];   // [row half][block]: half2 (scale, min)
-                {
-                    const uint8_t* fb = sP + ps * P_BYTES + dw * FB;
-                    if (dw < n_rt) {
-                        load_lane_codes<BITS>(lc, fb, lane);
-                        const uint4 s0 = *reinterpret_cast<const uint4*>(fb + g * 16);
-                        const uint4 s1 = *reinterpret_cast<const uint4*>(fb + (g + 8) * 16);
-                        dmw[0][0] = s0.x; dmw[0][1] = s0.y; dmw[0][2] = s0.z; dmw[0][3] = s0.w;
-                        dmw[1][0] = s1.x; dmw[1][1] = s1.y; dmw[1][2] = s1.z; dmw[1][3] = s1.w;
-                    } else {
-#pragma unroll
-                        for (int i = 0; i < 2 * BITS; ++i) lc.w[i] = 0;
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) { dmw[0][i] = 0; dmw[1][i] = 0; }
-                    }
-                }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar_pempty + 8 * ps);   // packed bytes are in registers now
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const uint32_t as = ai % GM_ASTAGES;
-                    ok = mbar_wait(bar_aempty + 8 * as, ((ai / GM_ASTAGES) & 1) ^ 1, abort_flag, 6);
-                    if (!ok) break;
-                    ++ai;
-                    uint8_t* At = sA + as * GM_A_BYTES;
-#pragma unroll
-                    for (int jj = 0; jj < 2; ++jj) {
-                        const int j = 2 * h + jj;
-#pragma unroll
-                        for (int hi = 0; hi < 2; ++hi) {
-                            const __half2 dm = *reinterpret_cast<const __half2*>(&dmw[hi][j]);
-                            const float d = __low2float(dm);
-                            const float mb = fmaf(-128.f, d, __high2float(dm));
-                            const __half2 d2 = __low2half2(dm), m2 = __high2half2(dm);
-                            uint32_t o[4];
-#pragma unroll
-                            for (int i = 0; i < 4; ++i) o[i] = dequant_pair<BF16>(code_pair<BITS>(lc, j, hi, i, MAGIC), d, mb, d2, m2);
-                            const int row = dw * 16 + g + 8 * hi;
-                            const int chunk = (jj * 4 + t) ^ (row & 7);
-                            *reinterpret_cast<uint4*>(At + (row >> 3) * 1024 + (row & 7) * 128 + chunk * 16) =
-                                make_uint4(o[0], o[1], o[2], o[3]);
-                        }
-                    }
-                    fence_async_smem();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar_afull + 8 * as);
-                }
+                const uint8_t* slab = sP + ps * P_BYTES;
+                if (op.bits == 2) ok = dequant_slab<2, BF16>(slab, dw < n_rt, dw, lane, sA, bar_pempty + 8 * ps, bar_aempty, bar_afull, ai, abort_flag);
+                else if (op.bits == 3) ok = dequant_slab<3, BF16>(slab, dw < n_rt, dw, lane, sA, bar_pempty + 8 * ps, bar_aempty, bar_afull, ai, abort_flag);
+                else ok = dequant_slab<4, BF16>(slab, dw < n_rt, dw, lane, sA, bar_pempty + 8 * ps, bar_aempty, bar_afull, ai, abort_flag);
             }
             // epilogue: TMEM lane quarter (warp % 4) x this warp group's columns -> out[token][row]
             if (ok) ok = mbar_wait(bar_accum, segc & 1, abort_flag, 7);
@@ -405,8 +434,9 @@ __global__ void __launch_bounds__(GM_THREADS, 1) gemm_kernel(const __grid_consta
                     acc = 0; c_lo = grp ? min(half, sg.w0) : 0; c_hi = grp ? sg.w0 : min(half, sg.w0);
                 }
                 // with a residual the launcher has copied it into out: every run then adds on top of it
-                const bool whole = (sg.s0 == 0 && sg.s1 == a.n_slabs) && (a.res == nullptr || !a.tma_out);
-                const bool add_res = (a.res != nullptr && sg.s0 == 0 && !a.tma_out);
+                const bool whole = (sg.s0 == 0 && sg.s1 == a.n_slabs) && (op.res == nullptr || !a.tma_out);
+                const bool add_res = (op.res != nullptr && sg.s0 == 0 && !a.tma_out);
+                const CUtensorMap* tmo = &tmap_out.m[sg.op];
                 const int n0 = sg.rt * GM_ROWS + lq * 32;
                 const int64_t n = (int64_t)n0 + lane;
                 const int tok0 = sg.st * a.st_tokens + acc * GM_MAX_TN;
@@ -426,8 +456,8 @@ __global__ void __launch_bounds__(GM_THREADS, 1) gemm_kernel(const __grid_consta
                         fence_async_smem();
                         __syncwarp();
                         if (lane == 0) {   // rows / tokens past the end of the tensor are clipped by the copy
-                            if (whole) tma_store_2d(&tmap_out, smem_u32(chunk), n0, tok0 + c0);
-                            else tma_reduce_add_2d(&tmap_out, smem_u32(chunk), n0, tok0 + c0);
+                            if (whole) tma_store_2d(tmo, smem_u32(chunk), n0, tok0 + c0);
+                            else tma_reduce_add_2d(tmo, smem_u32(chunk), n0, tok0 + c0);
                             bulk_commit();
                         }
                     }
@@ -438,16 +468,16 @@ __global__ void __launch_bounds__(GM_THREADS, 1) gemm_kernel(const __grid_consta
                         uint32_t v[32];
                         tmem_ld32(tmem_base + ((uint32_t)(lq * 32) << 16) + (uint32_t)(acc * GM_MAX_TN + c0), v);
                         tmem_ld_wait();
-                        if (n < a.N) {
+                        if (n < op.N) {
 #pragma unroll
                             for (int j = 0; j < 32; ++j) {
                                 const int tok = tok0 + c0 + j;
                                 if (c0 + j < c_hi && tok < a.M) {
-                                    const int64_t o = (int64_t)tok * a.ldo + n;
+                                    const int64_t o = (int64_t)tok * op.ldo + n;
                                     float val = __uint_as_float(v[j]);
-                                    if (add_res) val += __ldg(a.res + o);
-                                    if (whole) a.out[o] = val;
-                                    else atomicAdd(a.out + o, val);
+                                    if (add_res) val += __ldg(op.res + o);
+                                    if (whole) op.out[o] = val;
+                                    else atomicAdd(op.out + o, val);
                                 }
                             }
                         }
@@ -486,11 +516,10 @@ static EncodeTiledFn encode_fn() {
     return fn;
 }
 
-template <int BITS, bool BF16>
-static cudaError_t launch_one(const CUtensorMap& tm, const CUtensorMap& tmo, const GemmArgs& a, int grid, cudaStream_t s) {
-    constexpr int FB = frag_bytes(BITS);
-    constexpr int SMEM = 1024 + GM_ASTAGES * GM_A_BYTES + GM_BSLOTS * GM_B_BYTES + GM_PSTAGES * 8 * FB + 256;
-    auto kern = gemm_kernel<BITS, BF16>;
+template <bool BF16>
+static cudaError_t launch_one(const CUtensorMap& tm, const GemmOutMaps& tmo, const GemmArgs& a, int grid, cudaStream_t s) {
+    constexpr int SMEM = 1024 + GM_ASTAGES * GM_A_BYTES + GM_BSLOTS * GM_B_BYTES + GM_PSTAGES * 8 * frag_bytes(4) + 256;
+    auto kern = gemm_kernel<BF16>;
     static bool configured = false;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
@@ -502,14 +531,21 @@ static cudaError_t launch_one(const CUtensorMap& tm, const CUtensorMap& tmo, con
     return cudaGetLastError();
 }
 
-cudaError_t launch_gemm(const aq_handle_s* h, const void* x, aq_dtype_t xdt, int M, float* out, int64_t ldo,
-                        const float* res, cudaStream_t s) {
+// n (<= GM_MAX_OPS) matrices with the same K against one x: out[i] = (res[i]) + x W_i^T.
+cudaError_t launch_gemm_group(const aq_handle_s* const* hs, int n, const void* x, aq_dtype_t xdt, int M, float* const* outs,
+                              const int64_t* ldos, const float* const* ress, cudaStream_t s) {
     EncodeTiledFn enc = encode_fn();
-    if (!enc) return cudaErrorNotSupported;
+    if (!enc || n < 1 || n > GM_MAX_OPS) return cudaErrorNotSupported;
     GemmArgs a;
-    a.frags = h->frags; a.out = out; a.res = res; a.ldo = ldo; a.N = h->N; a.M = M; a.NT = h->NT;
-    a.n_slabs = h->KP * 2;
-    a.R = (h->NT + 7) / 8;
+    memset(&a, 0, sizeof(a));
+    a.n_ops = n; a.M = M; a.n_slabs = hs[0]->KP * 2;
+    for (int i = 0; i < n; ++i) {
+        if (hs[i]->K != hs[0]->K) return cudaErrorInvalidValue;
+        GemmOp& o = a.op[i];
+        o.frags = hs[i]->frags; o.out = outs[i]; o.res = ress ? ress[i] : nullptr; o.ldo = ldos[i];
+        o.N = (int)hs[i]->N; o.NT = hs[i]->NT; o.R = (hs[i]->NT + 7) / 8; o.bits = hs[i]->bits;
+        a.Rtot += o.R;
+    }
     if (M > GM_MAX_TN) {
         a.tn = GM_MAX_TN; a.st_tokens = 2 * GM_MAX_TN;
         a.n_st = (M + a.st_tokens - 1) / a.st_tokens;
@@ -517,12 +553,12 @@ cudaError_t launch_gemm(const aq_handle_s* h, const void* x, aq_dtype_t xdt, int
     } else {
         a.tn = ((M + 15) / 16) * 16; a.st_tokens = a.tn; a.n_st = 1; a.n2 = 0;
     }
-    const long long total = (long long)a.n_slabs * a.R * (2LL * a.n2 + (a.n_st - a.n2));
+    const long long total = (long long)a.n_slabs * a.Rtot * (2LL * a.n2 + (a.n_st - a.n2));
     int grid = sm_count();
     if (total / 2 < grid) grid = (int)(total / 2);
     CUtensorMap tm;
-    const cuuint64_t dims[2] = {(cuuint64_t)h->K, (cuuint64_t)M};
-    const cuuint64_t strides[1] = {(cuuint64_t)h->K * 2};
+    const cuuint64_t dims[2] = {(cuuint64_t)hs[0]->K, (cuuint64_t)M};
+    const cuuint64_t strides[1] = {(cuuint64_t)hs[0]->K * 2};
     const cuuint32_t box[2] = {(cuuint32_t)GM_KSTAGE, (cuuint32_t)a.tn};
     const cuuint32_t estr[2] = {1, 1};
     const CUresult r = enc(&tm, xdt == AQ_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2,
@@ -530,42 +566,46 @@ cudaError_t launch_gemm(const aq_handle_s* h, const void* x, aq_dtype_t xdt, int
                            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
-    // the output as a tensor [M][N] of float32 for the epilogue's 32 x 32 copies (row pitch must be 16-byte aligned)
-    CUtensorMap tmo;
+    // the outputs as tensors [M][N] of float32 for the epilogue's 32 x 32 copies (row pitch must be 16-byte aligned)
+    GemmOutMaps tmo;
     memset(&tmo, 0, sizeof(tmo));
-    a.tma_out = 0;
-    if (ldo % 4 == 0 && (reinterpret_cast<uintptr_t>(out) & 15u) == 0) {
-        const cuuint64_t odims[2] = {(cuuint64_t)h->N, (cuuint64_t)M};
-        const cuuint64_t ostrides[1] = {(cuuint64_t)ldo * 4};
+    a.tma_out = 1;
+    for (int i = 0; i < n && a.tma_out; ++i) {
+        const GemmOp& o = a.op[i];
+        if (o.ldo % 4 != 0 || (reinterpret_cast<uintptr_t>(o.out) & 15u) != 0) { a.tma_out = 0; break; }
+        const cuuint64_t odims[2] = {(cuuint64_t)o.N, (cuuint64_t)M};
+        const cuuint64_t ostrides[1] = {(cuuint64_t)o.ldo * 4};
         const cuuint32_t obox[2] = {32, 32};
-        if (enc(&tmo, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, out, odims, ostrides, obox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS)
-            a.tma_out = 1;
+        if (enc(&tmo.m[i], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, o.out, odims, ostrides, obox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            a.tma_out = 0;
     }
-    // What out holds before the kernel: the residual when there is one (every run then adds to it);
+    // What an output holds before the kernel: the residual when there is one (every run then adds to it);
     // else zeros when some run does not cover a whole tile; else nothing.
-    if (res && a.tma_out) {
-        cudaError_t e = cudaMemcpy2DAsync(out, (size_t)ldo * sizeof(float), res, (size_t)ldo * sizeof(float),
-                                          (size_t)h->N * sizeof(float), (size_t)M, cudaMemcpyDeviceToDevice, s);
-        if (e != cudaSuccess) return e;
-    } else {
-        bool all_whole = true;
-        const long long c2 = 2LL * a.n_slabs, reg2 = c2 * a.n2 * a.R;
+    bool all_whole = true;
+    {
+        const long long c2 = 2LL * a.n_slabs, reg2 = c2 * a.n2 * a.Rtot;
         for (int c = 1; c < grid && all_whole; ++c) {
             const long long b = ((total * c) / grid) & ~1LL;
             all_whole = (b <= reg2) ? (b % c2 == 0) : ((b - reg2) % a.n_slabs == 0);
         }
-        if (!all_whole) {
-            cudaError_t e = cudaMemset2DAsync(out, (size_t)ldo * sizeof(float), 0, (size_t)h->N * sizeof(float), (size_t)M, s);
-            if (e != cudaSuccess) return e;
-        }
     }
-    const bool bf = (xdt == AQ_BF16);
-    switch (h->bits) {
-        case 2: return bf ? launch_one<2, true>(tm, tmo, a, grid, s) : launch_one<2, false>(tm, tmo, a, grid, s);
-        case 3: return bf ? launch_one<3, true>(tm, tmo, a, grid, s) : launch_one<3, false>(tm, tmo, a, grid, s);
-        default: return bf ? launch_one<4, true>(tm, tmo, a, grid, s) : launch_one<4, false>(tm, tmo, a, grid, s);
+    for (int i = 0; i < n; ++i) {
+        const GemmOp& o = a.op[i];
+        cudaError_t e = cudaSuccess;
+        if (o.res && a.tma_out)
+            e = cudaMemcpy2DAsync(o.out, (size_t)o.ldo * sizeof(float), o.res, (size_t)o.ldo * sizeof(float),
+                                  (size_t)o.N * sizeof(float), (size_t)M, cudaMemcpyDeviceToDevice, s);
+        else if (!all_whole)
+            e = cudaMemset2DAsync(o.out, (size_t)o.ldo * sizeof(float), 0, (size_t)o.N * sizeof(float), (size_t)M, s);
+        if (e != cudaSuccess) return e;
     }
+    return (xdt == AQ_BF16) ? launch_one<true>(tm, tmo, a, grid, s) : launch_one<false>(tm, tmo, a, grid, s);
+}
+
+cudaError_t launch_gemm(const aq_handle_s* h, const void* x, aq_dtype_t xdt, int M, float* out, int64_t ldo,
+                        const float* res, cudaStream_t s) {
+    return launch_gemm_group(&h, 1, x, xdt, M, &out, &ldo, &res, s);
 }
 
 int read_gemm_status(bool clear) {

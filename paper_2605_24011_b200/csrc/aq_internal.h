@@ -47,6 +47,10 @@ cudaError_t launch_finalize(const float* acc_in, float* acc_zero, int64_t ldacc,
 // out need not be initialised (the launcher zeroes it when tiles are split over CTAs)
 cudaError_t launch_gemm(const aq_handle_s* h, const void* x, aq_dtype_t xdt, int M, float* out,
                         int64_t ldo, const float* res, cudaStream_t s);
+// the same for up to AQ_GEMM_MAX_GROUP matrices of one K that read the same x, as one launch
+#define AQ_GEMM_MAX_GROUP 4
+cudaError_t launch_gemm_group(const aq_handle_s* const* hs, int n, const void* x, aq_dtype_t xdt, int M,
+                              float* const* outs, const int64_t* ldos, const float* const* ress, cudaStream_t s);
 
 // Where a program's buffers and staged inputs sit in the caller's workspace (aq_stack.cu).
 struct StackPlan {

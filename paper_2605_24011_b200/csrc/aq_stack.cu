@@ -178,21 +178,33 @@ static cudaError_t run_stack(const aq_stack_t* p, const StackPlan& plan, const T
         count_launch();
         int j = i;
         while (j < p->n_ops && same_input(p->ops[j], f)) {
-            const aq_stack_op_t& o = p->ops[j];
-            const int64_t N = p->buf_width[o.dst];
-            const float* res = (o.out_op == AQ_OUT_ADD) ? buf(o.res) : nullptr;
             if (decode) {
-                if (res) {
-                    e = cudaMemcpyAsync(buf(o.dst), res, (size_t)M * N * sizeof(float), cudaMemcpyDeviceToDevice, s);
+                const aq_stack_op_t& o = p->ops[j];
+                const int64_t N = p->buf_width[o.dst];
+                if (o.out_op == AQ_OUT_ADD) {
+                    e = cudaMemcpyAsync(buf(o.dst), buf(o.res), (size_t)M * N * sizeof(float), cudaMemcpyDeviceToDevice, s);
                     if (e != cudaSuccess) return e;
                 }
                 e = launch_gemv(o.w, stage, dt, M, buf(o.dst), N, s);
-            } else {
-                e = launch_gemm(o.w, stage, dt, M, buf(o.dst), N, res, s);
+                if (e != cudaSuccess) return e;
+                o.w->last_stream = s;
+                ++j;
+            } else {   // the matrices of a phase read the same x: up to AQ_GEMM_MAX_GROUP of them per launch
+                const aq_handle_s* hs[AQ_GEMM_MAX_GROUP];
+                float* outs[AQ_GEMM_MAX_GROUP];
+                const float* ress[AQ_GEMM_MAX_GROUP];
+                int64_t ldos[AQ_GEMM_MAX_GROUP];
+                int n = 0;
+                while (n < AQ_GEMM_MAX_GROUP && j < p->n_ops && same_input(p->ops[j], f)) {
+                    const aq_stack_op_t& o = p->ops[j];
+                    hs[n] = o.w; outs[n] = buf(o.dst); ldos[n] = p->buf_width[o.dst];
+                    ress[n] = (o.out_op == AQ_OUT_ADD) ? buf(o.res) : nullptr;
+                    o.w->last_stream = s;
+                    ++n; ++j;
+                }
+                e = launch_gemm_group(hs, n, stage, dt, M, outs, ldos, ress, s);
+                if (e != cudaSuccess) return e;
             }
-            if (e != cudaSuccess) return e;
-            o.w->last_stream = s;
-            ++j;
         }
         i = j;
     }
