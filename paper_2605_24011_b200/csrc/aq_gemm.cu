@@ -532,8 +532,9 @@ static cudaError_t launch_one(const CUtensorMap& tm, const GemmOutMaps& tmo, con
 }
 
 // n (<= GM_MAX_OPS) matrices with the same K against one x: out[i] = (res[i]) + x W_i^T.
+// outs_ready: the caller has already put the residual (or zeros) into every output.
 cudaError_t launch_gemm_group(const aq_handle_s* const* hs, int n, const void* x, aq_dtype_t xdt, int M, float* const* outs,
-                              const int64_t* ldos, const float* const* ress, cudaStream_t s) {
+                              const int64_t* ldos, const float* const* ress, bool outs_ready, cudaStream_t s) {
     EncodeTiledFn enc = encode_fn();
     if (!enc || n < 1 || n > GM_MAX_OPS) return cudaErrorNotSupported;
     GemmArgs a;
@@ -590,7 +591,8 @@ cudaError_t launch_gemm_group(const aq_handle_s* const* hs, int n, const void* x
             all_whole = (b <= reg2) ? (b % c2 == 0) : ((b - reg2) % a.n_slabs == 0);
         }
     }
-    for (int i = 0; i < n; ++i) {
+    if (outs_ready && !a.tma_out) return cudaErrorInvalidValue;   // (the caller checks gemm_outputs_can_be_preset first)
+    for (int i = 0; i < n && !outs_ready; ++i) {
         const GemmOp& o = a.op[i];
         cudaError_t e = cudaSuccess;
         if (o.res && a.tma_out)
@@ -605,7 +607,15 @@ cudaError_t launch_gemm_group(const aq_handle_s* const* hs, int n, const void* x
 
 cudaError_t launch_gemm(const aq_handle_s* h, const void* x, aq_dtype_t xdt, int M, float* out, int64_t ldo,
                         const float* res, cudaStream_t s) {
-    return launch_gemm_group(&h, 1, x, xdt, M, &out, &ldo, &res, s);
+    return launch_gemm_group(&h, 1, x, xdt, M, &out, &ldo, &res, false, s);
+}
+
+// True when launch_gemm_group accepts outputs preset by the caller (they are written through tensor maps).
+bool gemm_outputs_can_be_preset(float* const* outs, const int64_t* ldos, int n) {
+    if (!encode_fn()) return false;
+    for (int i = 0; i < n; ++i)
+        if (ldos[i] % 4 != 0 || (reinterpret_cast<uintptr_t>(outs[i]) & 15u) != 0) return false;
+    return true;
 }
 
 int read_gemm_status(bool clear) {

@@ -50,7 +50,9 @@ cudaError_t launch_gemm(const aq_handle_s* h, const void* x, aq_dtype_t xdt, int
 // the same for up to AQ_GEMM_MAX_GROUP matrices of one K that read the same x, as one launch
 #define AQ_GEMM_MAX_GROUP 4
 cudaError_t launch_gemm_group(const aq_handle_s* const* hs, int n, const void* x, aq_dtype_t xdt, int M,
-                              float* const* outs, const int64_t* ldos, const float* const* ress, cudaStream_t s);
+                              float* const* outs, const int64_t* ldos, const float* const* ress, bool outs_ready,
+                              cudaStream_t s);
+bool gemm_outputs_can_be_preset(float* const* outs, const int64_t* ldos, int n);
 
 // Where a program's buffers and staged inputs sit in the caller's workspace (aq_stack.cu).
 struct StackPlan {

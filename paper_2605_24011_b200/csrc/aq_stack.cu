@@ -96,9 +96,24 @@ __device__ __forceinline__ void store_round4(T* o, const float4& v) {
 // x[m][k] = round(transform(src[m][k])); K is a multiple of 32, rows are 16-byte aligned.
 // RMS scaling: one CTA per token row.  The other two forms have no row-wide term and
 // run as a flat grid over groups of four elements (blockIdx.y = 0).
+// Outputs the linears of a phase will add into: dst = src (the residual) or zero, n4 groups of four floats each.
+struct PresetList {
+    float4* dst[8];
+    const float4* src[8];
+    int64_t n4[8];
+    int n;
+};
+
 template <typename T>
 __global__ void __launch_bounds__(256) stage_kernel(const float* __restrict__ src, const float* __restrict__ src2,
-                                                    int in_op, int64_t K, int64_t total4, T* __restrict__ x) {
+                                                    int in_op, int64_t K, int64_t total4, T* __restrict__ x,
+                                                    const PresetList pre) {
+    for (int q = 0; q < pre.n; ++q) {
+        float4* d = pre.dst[q];
+        const float4* r = pre.src[q];
+        for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < pre.n4[q]; i += (int64_t)gridDim.x * 256)
+            d[i] = r ? r[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
     if (in_op != AQ_IN_RMSNORM) {
         const float4* s4 = reinterpret_cast<const float4*>(src);
         const float4* t4 = reinterpret_cast<const float4*>(src2);
@@ -170,10 +185,33 @@ static cudaError_t run_stack(const aq_stack_t* p, const StackPlan& plan, const T
         const aq_stack_op_t& f = p->ops[i];
         const int64_t K = p->buf_width[f.src];
         T* stage = reinterpret_cast<T*>(ws + plan.in_off[i]);
+        PresetList pre;
+        pre.n = 0;
+        bool preset = false;
+        if (!decode) {   // the phase's outputs start as residual / zero: written here, in the same launch as x
+            float* outs[8];
+            int64_t ldos[8];
+            int n = 0;
+            bool fits = true;
+            for (int q = i; q < p->n_ops && same_input(p->ops[q], f); ++q) {
+                if (n == 8) { fits = false; break; }
+                outs[n] = buf(p->ops[q].dst); ldos[n] = p->buf_width[p->ops[q].dst]; ++n;
+            }
+            if (fits && gemm_outputs_can_be_preset(outs, ldos, n)) {
+                preset = true;
+                for (int q = 0; q < n; ++q) {
+                    const aq_stack_op_t& o = p->ops[i + q];
+                    pre.dst[q] = reinterpret_cast<float4*>(outs[q]);
+                    pre.src[q] = (o.out_op == AQ_OUT_ADD) ? reinterpret_cast<const float4*>(buf(o.res)) : nullptr;
+                    pre.n4[q] = (int64_t)M * ldos[q] / 4;
+                }
+                pre.n = n;
+            }
+        }
         {
             const int64_t total4 = (int64_t)M * K / 4;
             const unsigned g = (f.in_op == AQ_IN_RMSNORM) ? (unsigned)M : (unsigned)std::min<int64_t>((total4 + 255) / 256, 4 * 148);
-            stage_kernel<T><<<g, 256, 0, s>>>(buf(f.src), f.in_op == AQ_IN_SILU_MUL ? buf(f.src2) : nullptr, f.in_op, K, total4, stage);
+            stage_kernel<T><<<g, 256, 0, s>>>(buf(f.src), f.in_op == AQ_IN_SILU_MUL ? buf(f.src2) : nullptr, f.in_op, K, total4, stage, pre);
         }
         count_launch();
         int j = i;
@@ -202,7 +240,7 @@ static cudaError_t run_stack(const aq_stack_t* p, const StackPlan& plan, const T
                     o.w->last_stream = s;
                     ++n; ++j;
                 }
-                e = launch_gemm_group(hs, n, stage, dt, M, outs, ldos, ress, s);
+                e = launch_gemm_group(hs, n, stage, dt, M, outs, ldos, ress, preset, s);
                 if (e != cudaSuccess) return e;
             }
         }
