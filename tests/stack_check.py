@@ -13,11 +13,13 @@ from oracle import aq_oracle as O
 from paper_2605_24011_b200 import aq
 
 
-def check_program(prog, names, ws, M, dtype, quantised, rows=None, cols_sample=None, rng=None):
+def check_program(prog, names, ws, M, dtype, quantised, rows=None, cols_sample=None, rng=None, cols_of=None):
     """quantised: dict (layer, name) -> (d, m, q) oracle codes of that matrix,
     or a callable (layer, name, row_idx) -> (d, m, q) restricted to rows.
     rows: token rows to check (default all).  cols_sample: number of output
-    columns to sample per op (default all).  Returns worst normalised error."""
+    columns to sample per op (default all); cols_of(layer, name) gives the output
+    columns to check instead (the rows of W that were kept at packing time).
+    Returns worst normalised error."""
     ulp = 2.0 ** -10 if dtype == torch.float16 else 2.0 ** -7
     tiny = 2.0 ** -24 if dtype == torch.float16 else 1e-37     # spacing of binary16 subnormals
     rows = list(range(M)) if rows is None else rows
@@ -44,7 +46,9 @@ def check_program(prog, names, ws, M, dtype, quantised, rows=None, cols_sample=N
 
         key = names[i]
         N = prog.buf_width[op["dst"]]
-        if cols_sample is not None and cols_sample < N:
+        if cols_of is not None:
+            cols = np.asarray(cols_of(key[0], key[1]))
+        elif cols_sample is not None and cols_sample < N:
             cols = np.sort(rng.choice(N, size=cols_sample, replace=False))
         else:
             cols = np.arange(N)
