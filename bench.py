@@ -104,6 +104,20 @@ def _timed(fn, steps, warmup, torch):
     return e0.elapsed_time(e1)
 
 
+def reduce_max(values, dist, device):
+    """Max over ranks of each entry (the slowest rank decides a multi-rank time)."""
+    import torch
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def whole_job_gbs(world, packed_bytes_per_rank, ms_per_step):
+    """Replicas only: every rank streams its own copy of the weights; the job's rate is the sum."""
+    return world * packed_bytes_per_rank / (ms_per_step * 1e-3) / 1e9
+
+
 def oracle_layer_sample(which=("q", "k", "v", "o", "gate", "up", "down")):
     """Host-side inputs for the oracle timing: one 7B-shaped layer (or part of it)."""
     import numpy as np
@@ -214,7 +228,7 @@ WORKLOAD = ("7B-class decoder linear stack, M=1 decode: 32 layers x {q,k,v,o 409
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
     ap.add_argument("--layers", type=int, default=32, help="decoder layers (32 = the full workload)")
@@ -281,13 +295,10 @@ def main():
     ms_e2e = _timed(step_e2e, args.steps, 3, torch)
     clocks = sampler.stop()
     aq.aq_check()
-    if dist:
-        t = torch.tensor([ms, ms_e2e], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, ms_e2e = float(t[0]), float(t[1])
+    ms, ms_e2e = reduce_max([ms, ms_e2e], dist, "cuda")
     ms_step = ms / args.steps
-    value = world * packed / (ms_step * 1e-3) / 1e9
-    e2e = world * packed / (ms_e2e / args.steps * 1e-3) / 1e9
+    value = whole_job_gbs(world, packed, ms_step)
+    e2e = whole_job_gbs(world, packed, ms_e2e / args.steps)
 
     line = {
         "metric": "decode_weight_stream", "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
@@ -305,7 +316,9 @@ def main():
         "pct_of_nominal_hbm": 100.0 * (value / world) / NOMINAL_HBM_GBS,
         "roofline": {"bound": "hbm", "achieved": value / world, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": (value / world) / peaks["hbm_gbs"], "traffic": DECODE_TRAFFIC_BYTES,
-                     "peak_source": peaks["source"], "kernel": "gemv_kernel (all launches of one stack pass)",
+                     "peak_source": peaks["source"],
+                     "kernel": "decode_stack_kernel (one launch per pass; time = whole pass incl. its two glue kernels)",
+                     "traffic_note": "dram bytes of the 4-layer ncu capture scaled by packed bytes to 32 layers",
                      "algorithmic_bytes_per_step": packed},
     }
 
@@ -314,10 +327,11 @@ def main():
         line["dequant"] = dequant_leg(aq, synth, peaks, torch)
         cores = len(os.sched_getaffinity(0))
         mats = oracle_layer_sample()
-        dt, nb = time_oracle(mats)
+        dt, nb = time_oracle(mats, repeats=7)
         line["cpu_baseline"] = {"value": nb / dt / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
                                 "seconds": dt,
-                                "sample": "one 7B-shaped layer (7 matrices, 202M weights, M=1): oracle dequant + fp64 mat-vec"}
+                                "sample": "7 passes over one 7B-shaped layer (7 matrices, 202M weights, M=1): "
+                                          "oracle dequant + fp64 mat-vec"}
     if rank == 0:
         print(json.dumps(line))
     if dist:
@@ -326,8 +340,9 @@ def main():
 
 # dram__bytes_read.sum + dram__bytes_write.sum of the decode kernel per stack pass, from the ncu
 # capture summarised under profiles/ (None until a capture has been taken).
-DECODE_TRAFFIC_BYTES = None
-PREFILL_TRAFFIC_BYTES = None
+DECODE_TRAFFIC_BYTES = int((354.999e6 + 3.867e6) * 2833383424 / 354.17e6)
+# gemm_kernel: 43.75 MB per 11008 x 4096 launch, scaled by weights to the 224 matrices of one pass
+PREFILL_TRAFFIC_BYTES = int(43.75e6 * 6476005376 / (11008 * 4096))
 
 
 def prefill_leg(aq, workloads, prog, out_buf, info, peaks, torch):
@@ -352,30 +367,36 @@ def prefill_leg(aq, workloads, prog, out_buf, info, peaks, torch):
             "roofline": {"bound": "tensor", "achieved": tf, "peak": peaks["bf16_tflops_sustained"] or peaks["bf16_tflops"],
                          "unit": "TFLOP/s", "frac": tf / (peaks["bf16_tflops_sustained"] or peaks["bf16_tflops"]),
                          "traffic": PREFILL_TRAFFIC_BYTES, "peak_source": peaks["source"] + " (sustained: timed inside a long step)",
-                         "kernel": "gemm_kernel (all launches of one stack pass, glue kernels included in the time)"}}
+                         "kernel": "gemm_kernel (128 grouped launches per pass; time = whole pass incl. staging kernels)"}}
 
 
 def dequant_leg(aq, synth, peaks, torch):
-    """Standalone dequant, K = N = 4096 4-bit, rotating over 24 packed copies so that every call misses L2."""
-    N = K = 4096
-    W = synth.weights_device(N, K, 1)
-    hs = [aq.aq_pack(4, 32, W) for _ in range(24)]
-    outs = [torch.empty((N, K), dtype=torch.float16, device="cuda") for _ in range(8)]
-    i = [0]
+    """Standalone dequant, cold L2 (packed copies and outputs in rotation): the single 4096 x 4096 4-bit linear of the
+    small configuration (launch-latency sized: 44 MB per call) and a 16384 x 8192 matrix that amortises the launch."""
+    def run(N, K, n_packed, n_out, steps):
+        W = synth.weights_device(N, K, 1)
+        hs = [aq.aq_pack(4, 32, W) for _ in range(n_packed)]
+        del W
+        outs = [torch.empty((N, K), dtype=torch.float16, device="cuda") for _ in range(n_out)]
+        i = [0]
 
-    def step():
-        aq.aq_dequant(hs[i[0] % 24], outs[i[0] % 8])
-        i[0] += 1
+        def step():
+            aq.aq_dequant(hs[i[0] % n_packed], outs[i[0] % n_out])
+            i[0] += 1
 
-    ms = _timed(step, 48, 8, torch) / 48
-    nbytes = N * K * 5 // 8 + N * K * 2
-    gbs = nbytes / (ms * 1e-3) / 1e9
-    for h in hs:
-        h.free()
-    return {"workload": "aq_dequant 4096x4096 4-bit -> fp16, cold L2 (24 packed copies, 8 outputs in rotation)",
-            "us_per_call": 1e3 * ms, "gbs": gbs,
-            "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                         "frac": gbs / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"]}}
+        ms = _timed(step, steps, 8, torch) / steps
+        for h in hs:
+            h.free()
+        nbytes = N * K * 5 // 8 + N * K * 2
+        return ms, nbytes / (ms * 1e-3) / 1e9
+
+    ms_s, gbs_s = run(4096, 4096, 24, 8, 48)
+    ms_l, gbs_l = run(16384, 8192, 3, 2, 12)
+    return {"workload": "aq_dequant 4-bit -> fp16, cold L2: 16384x8192 (roofline) and 4096x4096 (the single-linear configuration)",
+            "us_per_call": 1e3 * ms_l, "gbs": gbs_l, "us_per_call_4096": 1e3 * ms_s, "gbs_4096": gbs_s,
+            "roofline": {"bound": "hbm", "achieved": gbs_l, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": gbs_l / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
+                         "kernel": "dequant_kernel, 16384x8192"}}
 
 
 if __name__ == "__main__":

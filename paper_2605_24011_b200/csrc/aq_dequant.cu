@@ -39,9 +39,13 @@ __device__ __forceinline__ void decode_unit(const LaneCodes<BITS>& lc, const uin
     const float d = __low2float(dm), m = __high2float(dm);
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
+        // the two codes as floats without a conversion: 2^23 + q has q in its low mantissa bits, and
+        // (2^23 + q) - 2^23 is exact, so the value is the same as (float)q
         const uint32_t p = code_pair<BITS>(lc, j, hi, i, 0u);
-        w[2 * i] = fmaf(d, (float)(p & 0xffffu), m);
-        w[2 * i + 1] = fmaf(d, (float)(p >> 16), m);
+        const float q0 = __uint_as_float((p & 0xffffu) | 0x4B000000u) - 8388608.f;
+        const float q1 = __uint_as_float(__byte_perm(p, 0x4B000000u, 0x7632)) - 8388608.f;
+        w[2 * i] = fmaf(d, q0, m);
+        w[2 * i + 1] = fmaf(d, q1, m);
     }
 }
 
