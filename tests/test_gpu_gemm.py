@@ -63,6 +63,19 @@ def test_gemm_prefill_rows(aq, bits, M):
     _run(aq, bits, 512, 4096, M, "bf16", kind="vision_text", out_f32=False)
 
 
+@pytest.mark.parametrize("bits", (2, 3, 4))
+def test_gemm_row_count_not_a_multiple_of_four(aq, bits):
+    """The output row pitch is then not 16-byte aligned: the epilogue falls back from TMA to plain stores / atomics."""
+    _run(aq, bits, 250, 512, 40, "bf16")
+    _run(aq, bits, 1030, 1024, 300, "f16")
+
+
+@pytest.mark.parametrize("M", (1024, 1300, 4096))
+def test_gemm_many_tokens(aq, M):
+    """Several token super-tiles, the last one ragged; M = 4096 is the largest call the library takes."""
+    _run(aq, 3, 160, 512, M, "bf16")
+
+
 def test_gemm_m_consistency_with_decode(aq):
     """Rows of an M=64 tensor-core call agree with the M=1 streaming call on the same handle."""
     bits, N, K = 3, 256, 1024
