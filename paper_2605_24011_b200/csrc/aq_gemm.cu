@@ -317,6 +317,9 @@ __global__ void __launch_bounds__(GM_THREADS, 1) gemm_kernel(const __grid_consta
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // everything above touched only this CTA's own resources; from here on the predecessor's results are read
+    pdl_wait();
+    pdl_launch_dependents();
 
     // this CTA's run, in slab-accumulators (even bounds)
     const long long total = (long long)a.n_slabs * a.Rtot * (2LL * a.n2 + (a.n_st - a.n2));
@@ -526,9 +529,9 @@ static cudaError_t launch_one(const CUtensorMap& tm, const GemmOutMaps& tmo, con
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    kern<<<grid, GM_THREADS, SMEM, s>>>(tm, tmo, a);
+    cudaError_t e = launch_pdl(kern, dim3((unsigned)grid), dim3(GM_THREADS), SMEM, s, tm, tmo, a);
     count_launch();
-    return cudaGetLastError();
+    return e;
 }
 
 // n (<= GM_MAX_OPS) matrices with the same K against one x: out[i] = (res[i]) + x W_i^T.

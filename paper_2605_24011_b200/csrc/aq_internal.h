@@ -70,6 +70,25 @@ int launch_decode_stack(const aq_stack_t* p, const StackPlan& plan, int M, aq_dt
 void decode_stack_forget(aq_handle_t h);   // drops cached device tables that name h
 int read_decode_status(bool clear);        // nonzero: a bounded wait in the decode-stack kernel ran out
 
+// Programmatic dependent launch, used along the prefill path: a kernel launched with launch_pdl may become
+// resident while its predecessor on the stream still runs; it must execute pdl_wait() before it touches anything the
+// predecessor wrote, and a kernel lets its successor in early with pdl_launch_dependents().
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+static inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args... args) {
+    cudaLaunchConfig_t cfg;
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
+#endif
+
 int sm_count();
 void count_launch(int n = 1);       // process-wide count of this library's kernel launches
 int read_gemm_status(bool clear);   // nonzero: a bounded wait in the GEMM kernel ran out

@@ -108,6 +108,8 @@ template <typename T>
 __global__ void __launch_bounds__(256) stage_kernel(const float* __restrict__ src, const float* __restrict__ src2,
                                                     int in_op, int64_t K, int64_t total4, T* __restrict__ x,
                                                     const PresetList pre) {
+    pdl_wait();                 // the buffers read and preset here belong to the kernels before this one
+    pdl_launch_dependents();    // the linears of this phase may set themselves up meanwhile
     for (int q = 0; q < pre.n; ++q) {
         float4* d = pre.dst[q];
         const float4* r = pre.src[q];
@@ -211,7 +213,10 @@ static cudaError_t run_stack(const aq_stack_t* p, const StackPlan& plan, const T
         {
             const int64_t total4 = (int64_t)M * K / 4;
             const unsigned g = (f.in_op == AQ_IN_RMSNORM) ? (unsigned)M : (unsigned)std::min<int64_t>((total4 + 255) / 256, 4 * 148);
-            stage_kernel<T><<<g, 256, 0, s>>>(buf(f.src), f.in_op == AQ_IN_SILU_MUL ? buf(f.src2) : nullptr, f.in_op, K, total4, stage, pre);
+            const float* s2 = (f.in_op == AQ_IN_SILU_MUL) ? buf(f.src2) : nullptr;
+            if (decode) stage_kernel<T><<<g, 256, 0, s>>>(buf(f.src), s2, (int)f.in_op, K, total4, stage, pre);
+            else e = launch_pdl(stage_kernel<T>, dim3(g), dim3(256), 0, s, (const float*)buf(f.src), s2, (int)f.in_op, K, total4, stage, pre);
+            if (e != cudaSuccess) return e;
         }
         count_launch();
         int j = i;
