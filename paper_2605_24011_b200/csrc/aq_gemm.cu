@@ -21,6 +21,7 @@
 // runs out the CTA raises a status word, drains and returns.
 #include <cuda.h>
 
+#include <atomic>
 #include <cstring>
 
 #include "aq_internal.h"
@@ -41,6 +42,13 @@ constexpr int GM_A_BYTES = GM_ROWS * GM_KSTAGE * 2;
 constexpr uint32_t GM_SPIN_LIMIT = 40u * 1000u * 1000u;
 
 __device__ int g_gemm_status = 0;  // nonzero: a bounded wait ran out (code = which)
+
+// Split tiles without zeroing the output first: the run that holds a tile's last k-slab is the first thing its CTA
+// does; it STORES its sums and then writes the launch's epoch into the tile's flag; the other runs of the tile add
+// theirs once they see it.  Flags are never reset: every launch has its own epoch and takes the next of a few arrays.
+constexpr int GM_FLAG_SLOTS = 8;
+constexpr int GM_MAX_TILES = 8192;
+__device__ uint32_t g_tile_flags[GM_FLAG_SLOTS][GM_MAX_TILES];
 
 constexpr int GM_MAX_OPS = 4;      // matrices that share one input (q|k|v, gate|up) run as one launch
 
@@ -66,6 +74,9 @@ struct GemmArgs {
     int st_tokens;         // tokens per super-tile (512 when M > 256)
     int tn;                // TMA box rows: 256 when M > 256, else M rounded up to 16
     int tma_out;           // 1: the epilogue writes through the output tensor maps (needs ldo % 4 == 0)
+    int store_first;       // 1: split tiles of matrices without a residual use the store-then-add protocol above
+    int flag_slot;
+    uint32_t epoch;
 };
 
 struct GemmOutMaps { CUtensorMap m[GM_MAX_OPS]; };
@@ -73,6 +84,7 @@ struct GemmOutMaps { CUtensorMap m[GM_MAX_OPS]; };
 // One contiguous piece of a CTA's run: slabs [s0, s1) of tile (rt, st).
 struct GemmSeg {
     int op, rt, st, na, s0, s1;   // rt: row tile inside matrix op
+    int tile;                     // index of the tile in the launch
     int w0, w1;            // tokens (rounded up to 16) of the two accumulators
 };
 
@@ -94,6 +106,7 @@ __device__ __forceinline__ bool gemm_next_seg(long long& pos, long long hi, cons
         sg.na = 1; sg.s0 = (int)(pos - base); sg.s1 = (int)(end - base);
     }
     pos = end;
+    sg.tile = (int)t;
     sg.st = (int)(t / a.Rtot);
     int r = (int)(t - (long long)sg.st * a.Rtot);
     sg.op = 0;
@@ -161,6 +174,14 @@ __device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* tm, uint32_
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
 template <int N> __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t* p) {
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release_u32(uint32_t* p, uint32_t v) {
+    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
@@ -437,7 +458,24 @@ __global__ void __launch_bounds__(GM_THREADS, 1) gemm_kernel(const __grid_consta
                     acc = 0; c_lo = grp ? min(half, sg.w0) : 0; c_hi = grp ? sg.w0 : min(half, sg.w0);
                 }
                 // with a residual the launcher has copied it into out: every run then adds on top of it
-                const bool whole = (sg.s0 == 0 && sg.s1 == a.n_slabs) && (op.res == nullptr || !a.tma_out);
+                const bool first_mode = a.store_first && op.res == nullptr;
+                const bool entire = (sg.s0 == 0 && sg.s1 == a.n_slabs);
+                const bool whole = (entire && (op.res == nullptr || !a.tma_out)) || (first_mode && sg.s1 == a.n_slabs);
+                const bool raise_flag = first_mode && whole && !entire;
+                if (first_mode && !whole) {   // the tile's last-slab run has to have stored before anything is added
+                    const uint32_t* fl = &g_tile_flags[a.flag_slot][sg.tile];
+                    uint32_t seen = 0, spins = 0;
+                    if (lane == 0) {
+                        while ((seen = ld_acquire_u32(fl)) != a.epoch) {
+                            if (++spins > (1u << 22) || *abort_flag) break;
+                            __nanosleep(100);
+                        }
+                        if (seen != a.epoch) { *abort_flag = 1; atomicCAS(&g_gemm_status, 0, 8); }
+                    }
+                    seen = __shfl_sync(0xffffffffu, seen, 0);
+                    ok = (seen == a.epoch);
+                }
+                if (ok) {
                 const bool add_res = (op.res != nullptr && sg.s0 == 0 && !a.tma_out);
                 const CUtensorMap* tmo = &tmap_out.m[sg.op];
                 const int n0 = sg.rt * GM_ROWS + lq * 32;
@@ -464,7 +502,10 @@ __global__ void __launch_bounds__(GM_THREADS, 1) gemm_kernel(const __grid_consta
                             bulk_commit();
                         }
                     }
-                    if (lane == 0) bulk_wait_read<0>();       // the A ring is written again right after
+                    if (lane == 0) {
+                        if (raise_flag) bulk_wait_all<0>();   // the stores must have landed before the flag goes up
+                        else bulk_wait_read<0>();             // the A ring is written again right after
+                    }
                     __syncwarp();
                 } else {
                     for (int c0 = c_lo; c0 < c_hi; c0 += 32) {
@@ -486,10 +527,13 @@ __global__ void __launch_bounds__(GM_THREADS, 1) gemm_kernel(const __grid_consta
                         }
                     }
                 }
+                }
                 tc_fence_before();   // the next run's first MMA may overwrite the accumulators
             }
             // the chunks staged above live in the A ring: nobody refills it before everybody has left the epilogue
             asm volatile("bar.sync 1, %0;" ::"n"(GM_DQ_WARPS * 32) : "memory");
+            if (threadIdx.x == 0 && ok && a.store_first && a.op[sg.op].res == nullptr && sg.s1 == a.n_slabs && sg.s0 != 0)
+                st_release_u32(&g_tile_flags[a.flag_slot][sg.tile], a.epoch);
         }
     }
     if (warp < GM_DQ_WARPS && lane == 0) bulk_wait_all<0>();   // this thread's output copies are complete
@@ -533,6 +577,8 @@ static cudaError_t launch_one(const CUtensorMap& tm, const GemmOutMaps& tmo, con
     count_launch();
     return e;
 }
+
+bool gemm_stores_first(const aq_handle_s* const* hs, int n, int M);
 
 // n (<= GM_MAX_OPS) matrices with the same K against one x: out[i] = (res[i]) + x W_i^T.
 // outs_ready: the caller has already put the residual (or zeros) into every output.
@@ -595,13 +641,20 @@ cudaError_t launch_gemm_group(const aq_handle_s* const* hs, int n, const void* x
         }
     }
     if (outs_ready && !a.tma_out) return cudaErrorInvalidValue;   // (the caller checks gemm_outputs_can_be_preset first)
+    static std::atomic<uint32_t> epoch_counter{0};
+    a.store_first = (a.tma_out && gemm_stores_first(hs, n, M)) ? 1 : 0;
+    a.epoch = epoch_counter.fetch_add(1) + 1;
+    if (a.epoch == 0) a.epoch = epoch_counter.fetch_add(1) + 1;   // flags start out as zero: never use that value
+    a.flag_slot = (int)(a.epoch % GM_FLAG_SLOTS);
+    // What an output holds before the kernel: the residual when there is one (every run then adds to it); zeros
+    // when runs add without the store-first protocol; else nothing.  With outs_ready the caller has done this.
     for (int i = 0; i < n && !outs_ready; ++i) {
         const GemmOp& o = a.op[i];
         cudaError_t e = cudaSuccess;
         if (o.res && a.tma_out)
             e = cudaMemcpy2DAsync(o.out, (size_t)o.ldo * sizeof(float), o.res, (size_t)o.ldo * sizeof(float),
                                   (size_t)o.N * sizeof(float), (size_t)M, cudaMemcpyDeviceToDevice, s);
-        else if (!all_whole)
+        else if (!all_whole && !(a.store_first && !o.res))
             e = cudaMemset2DAsync(o.out, (size_t)o.ldo * sizeof(float), 0, (size_t)o.N * sizeof(float), (size_t)M, s);
         if (e != cudaSuccess) return e;
     }
@@ -611,6 +664,14 @@ cudaError_t launch_gemm_group(const aq_handle_s* const* hs, int n, const void* x
 cudaError_t launch_gemm(const aq_handle_s* h, const void* x, aq_dtype_t xdt, int M, float* out, int64_t ldo,
                         const float* res, cudaStream_t s) {
     return launch_gemm_group(&h, 1, x, xdt, M, &out, &ldo, &res, false, s);
+}
+
+// True when outputs without a residual need no zeroing before launch_gemm_group (split tiles store first).
+bool gemm_stores_first(const aq_handle_s* const* hs, int n, int M) {
+    long long R = 0;
+    for (int i = 0; i < n; ++i) R += (hs[i]->NT + 7) / 8;
+    const long long n_st = (M > GM_MAX_TN) ? (M + 2 * GM_MAX_TN - 1) / (2 * GM_MAX_TN) : 1;
+    return R * n_st <= GM_MAX_TILES;
 }
 
 // True when launch_gemm_group accepts outputs preset by the caller (they are written through tensor maps).

@@ -201,13 +201,22 @@ static cudaError_t run_stack(const aq_stack_t* p, const StackPlan& plan, const T
             }
             if (fits && gemm_outputs_can_be_preset(outs, ldos, n)) {
                 preset = true;
+                // launches are made of up to AQ_GEMM_MAX_GROUP matrices: zeros are needed where such a group
+                // cannot use the store-first protocol for its split tiles
                 for (int q = 0; q < n; ++q) {
                     const aq_stack_op_t& o = p->ops[i + q];
-                    pre.dst[q] = reinterpret_cast<float4*>(outs[q]);
-                    pre.src[q] = (o.out_op == AQ_OUT_ADD) ? reinterpret_cast<const float4*>(buf(o.res)) : nullptr;
-                    pre.n4[q] = (int64_t)M * ldos[q] / 4;
+                    const bool has_res = (o.out_op == AQ_OUT_ADD);
+                    if (!has_res) {
+                        const int g0 = q - q % AQ_GEMM_MAX_GROUP, gn = std::min(AQ_GEMM_MAX_GROUP, n - g0);
+                        const aq_handle_s* hs[AQ_GEMM_MAX_GROUP];
+                        for (int r = 0; r < gn; ++r) hs[r] = p->ops[i + g0 + r].w;
+                        if (gemm_stores_first(hs, gn, M)) continue;
+                    }
+                    pre.dst[pre.n] = reinterpret_cast<float4*>(outs[q]);
+                    pre.src[pre.n] = has_res ? reinterpret_cast<const float4*>(buf(o.res)) : nullptr;
+                    pre.n4[pre.n] = (int64_t)M * ldos[q] / 4;
+                    ++pre.n;
                 }
-                pre.n = n;
             }
         }
         {
