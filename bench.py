@@ -220,6 +220,111 @@ def run_micro(args):
     print(json.dumps(out))
 
 
+def run_configs(args):
+    """The five workload configurations, one timing each (CUDA events, cold weights where a case fits in L2)."""
+    import torch
+    from paper_2605_24011_b200 import aq, programs, synth, workloads
+    torch.cuda.set_device(0)
+    peaks = _peaks()
+    out = {"peaks": peaks}
+
+    def timed_us(fn, steps, warm=3):
+        return 1e3 * _timed(fn, steps, warm, torch) / steps
+
+    # 1: single linear 4096 x 4096, 4-bit, x fp16 [1][4096]: dequant + linear M = 1, cold (rotating copies) and L2-hot
+    W = synth.weights_device(4096, 4096, 0)
+    hs = [aq.aq_pack(4, 32, W) for _ in range(24)]
+    del W
+    x = workloads.activations_device(1, 4096, torch.float16, 1, 0)
+    y = torch.empty((1, 4096), dtype=torch.float16, device="cuda")
+    wf = [torch.empty((4096, 4096), dtype=torch.float16, device="cuda") for _ in range(8)]
+    i = [0]
+
+    def lin_cold():
+        aq.aq_linear(hs[i[0] % 24], x, y); i[0] += 1
+
+    def deq_cold():
+        aq.aq_dequant(hs[i[0] % 24], wf[i[0] % 8]); i[0] += 1
+
+    pb = 4096 * 4096 * 5 // 8
+    t_lc, t_lh = timed_us(lin_cold, 48), timed_us(lambda: aq.aq_linear(hs[0], x, y), 48)
+    t_dc, t_dh = timed_us(deq_cold, 48), timed_us(lambda: aq.aq_dequant(hs[0], wf[0]), 48)
+    out["config1"] = {"linear_M1_us_cold": t_lc, "linear_M1_gbs_cold": pb / t_lc / 1e3, "linear_M1_us_l2hot": t_lh,
+                      "linear_M1_gbs_l2hot": pb / t_lh / 1e3, "dequant_us_cold": t_dc,
+                      "dequant_gbs_cold": (pb + 2 * 4096 * 4096) / t_dc / 1e3, "dequant_us_l2hot": t_dh,
+                      "note": "one aq_linear call = streaming kernel + output cast (two launches)"}
+    for h in hs:
+        h.free()
+    del wf
+
+    # 2: LLaMA-2-7B MLP at 3-bit, M = 1 and M = 8 (weights 67.6 MB: L2-resident when repeated; 6 copies rotate)
+    H, I = 4096, 11008
+    sets = []
+    for c in range(6):
+        g = aq.aq_pack(3, 32, synth.weights_device(I, H, 20 + c))
+        u = aq.aq_pack(3, 32, synth.weights_device(I, H, 30 + c))
+        d = aq.aq_pack(3, 32, synth.weights_device(H, I, 40 + c))
+        sets.append(programs.mlp_program(g, u, d, H, I) + ((g, u, d),))
+    cfg2 = {}
+    for M in (1, 8):
+        ws = torch.empty(sets[0][0].workspace_bytes(M), dtype=torch.uint8, device="cuda")
+        x0 = workloads.activations_device(M, H, torch.float16, 2, M)
+        yo = torch.empty((M, H), dtype=torch.float16, device="cuda")
+
+        def mlp():
+            prog, ob = sets[i[0] % 6][0], sets[i[0] % 6][1]
+            aq.aq_stack_forward(prog, x0, yo, ob, M, ws); i[0] += 1
+
+        t = timed_us(mlp, 36, 12)
+        cfg2[f"M{M}_us"] = t
+        cfg2[f"M{M}_gbs"] = 3 * 22_544_384 / t / 1e3
+    out["config2"] = cfg2
+    for st in sets:
+        for h in st[3]:
+            h.free()
+    del sets
+
+    # 3 and 4: the 7B-class stack, M = 1 (fp16) and M = 512 (bf16)
+    prog, out_buf, names, _, info = workloads.llama7b_decode_stack(n_layers=32, seed=0)
+    for M, dt, key in ((1, torch.float16, "config3"), (8, torch.float16, "config3_M8"), (512, torch.bfloat16, "config4")):
+        ws = torch.empty(prog.workspace_bytes(M), dtype=torch.uint8, device="cuda")
+        x0 = workloads.activations_device(M, 4096, dt, 3, M, kind="vision_text" if M == 512 else "normal")
+        yo = torch.empty((M, 4096), dtype=dt, device="cuda")
+        t = timed_us(lambda: aq.aq_stack_forward(prog, x0, yo, out_buf, M, ws), 20 if M <= 8 else 5)
+        out[key] = {"us_per_pass": t, "gbs": info["packed_bytes"] / t / 1e3, "tflops": 2.0 * M * info["weights"] / t / 1e6,
+                    "mean_code_bits": info["mean_code_bits"]}
+        del ws
+    del prog
+
+    # 5: Gemma-2B-shaped backbone, prefill M = 768 (bf16); action expert, 10 steps at M = 50
+    prog, out_buf, names, _, info = workloads.gemma2b_stack(n_layers=18, seed=0)
+    M = 768
+    ws = torch.empty(prog.workspace_bytes(M), dtype=torch.uint8, device="cuda")
+    x0 = workloads.activations_device(M, 2048, torch.bfloat16, 5, 0)
+    yo = torch.empty((M, 2048), dtype=torch.bfloat16, device="cuda")
+    t = timed_us(lambda: aq.aq_stack_forward(prog, x0, yo, out_buf, M, ws), 5)
+    c5 = {"backbone_prefill_M768_us": t, "backbone_prefill_tflops": 2.0 * M * info["weights"] / t / 1e6,
+          "backbone_mean_code_bits": info["mean_code_bits"]}
+    del prog, ws
+    prog, out_buf, names, _, info = workloads.expert_stack(n_layers=18, seed=0)
+    M = 50
+    ws = torch.empty(prog.workspace_bytes(M), dtype=torch.uint8, device="cuda")
+    xs = [workloads.activations_device(M, 1024, torch.bfloat16, 6, st) for st in range(10)]
+    yo = torch.empty((M, 1024), dtype=torch.bfloat16, device="cuda")
+
+    def ten_steps():
+        for st in range(10):
+            aq.aq_stack_forward(prog, xs[st], yo, out_buf, M, ws)
+
+    t = timed_us(ten_steps, 5)
+    c5.update({"expert_10_steps_M50_us": t, "expert_us_per_step": t / 10, "expert_gbs": 10 * info["packed_bytes"] / t / 1e3,
+               "expert_tflops": 10 * 2.0 * M * info["weights"] / t / 1e6,
+               "expert_note": "194.6 MB of packed weights per step: partly L2-resident across the 10 steps"})
+    out["config5"] = c5
+    aq.aq_check()
+    print(json.dumps(out))
+
+
 WORKLOAD = ("7B-class decoder linear stack, M=1 decode: 32 layers x {q,k,v,o 4096x4096; gate,up 11008x4096; "
             "down 4096x11008}, per-matrix 2/3/4-bit (mean 2.5), blocks of 32 + fp16 scale/min, N(0,0.02) weights "
             "with 0.1% x20 outliers, x fp16 N(0,1)")
@@ -235,6 +340,8 @@ def main():
     ap.add_argument("--no-extras", action="store_true", help="skip prefill / dequant / oracle legs")
     ap.add_argument("--micro", choices=("decode_linear", "prefill_linear", "dequant", "decode_stack", "prefill_stack"),
                     help="time one kernel on a small case (the command ncu captures are taken from) instead of the benchmark")
+    ap.add_argument("--configs", action="store_true",
+                    help="time all five workload configurations once each and print one JSON object (not the benchmark line)")
     ap.add_argument("--bits", type=int, default=2)
     ap.add_argument("--M", type=int, default=None)
     ap.add_argument("--N", type=int, default=None)
@@ -245,6 +352,9 @@ def main():
         return
     if args.micro:
         run_micro(args)
+        return
+    if args.configs:
+        run_configs(args)
         return
 
     import numpy as np
