@@ -184,8 +184,12 @@ static aq_status_t linear_common(aq_handle_t h, const void* x_dev, void* y_dev, 
     cudaError_t e;
     if (M <= AQ_DECODE_MAX_M) {
         const int64_t ld = (int64_t)h->NT * 16;
-        e = launch_gemv(h, x_dev, xdt, M, h->acc, ld, s);
-        if (e == cudaSuccess) e = launch_finalize(h->acc, h->acc, ld, y_dev, ydt, M, h->N, s);
+        if ((int64_t)M * h->N <= 65536) {   // small outputs: the streaming kernel's last CTA casts them (one launch)
+            e = launch_gemv(h, x_dev, xdt, M, h->acc, ld, s, y_dev, ydt);
+        } else {
+            e = launch_gemv(h, x_dev, xdt, M, h->acc, ld, s);
+            if (e == cudaSuccess) e = launch_finalize(h->acc, h->acc, ld, y_dev, ydt, M, h->N, s);
+        }
     } else if (ydt == AQ_F32) {
         e = launch_gemm(h, x_dev, xdt, M, (float*)y_dev, h->N, nullptr, s);
     } else {

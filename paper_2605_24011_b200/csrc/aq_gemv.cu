@@ -29,6 +29,10 @@ struct GemvArgs {
     int64_t N;          // true N: rows >= N are padding and are not written
     int NT;
     int M;
+    // when y is given the last CTA to finish casts the sums into y[m][n] and zeroes them again (one launch per linear)
+    void* y;
+    int ydt;
+    unsigned int* ticket;   // zero between launches
 };
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint64_t pol) {
@@ -49,8 +53,7 @@ __global__ void __launch_bounds__(GEMV_WARPS * 32, 2) gemv_kernel(const GemvArgs
     const int64_t gw = (int64_t)blockIdx.x * GEMV_WARPS + warp;
     const int64_t nw = (int64_t)gridDim.x * GEMV_WARPS;
     const int64_t u0 = (a.n_units * gw) / nw, u1 = (a.n_units * (gw + 1)) / nw;
-    if (u0 >= u1) return;
-
+    if (u0 < u1) {
     uint64_t pol;
     asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
 
@@ -90,6 +93,27 @@ __global__ void __launch_bounds__(GEMV_WARPS * 32, 2) gemv_kernel(const GemvArgs
         }
     }
     cp_async_wait<0>();
+    }
+    if (a.y == nullptr) return;
+    // last-CTA epilogue: sums of all CTAs are complete once every CTA has taken a ticket after a fence
+    __shared__ int is_last;
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) is_last = (atomicAdd(a.ticket, 1u) == gridDim.x - 1) ? 1 : 0;
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    const int64_t total = (int64_t)a.M * a.N;
+    for (int64_t i = threadIdx.x; i < total; i += blockDim.x) {
+        const int64_t m = i / a.N, n = i - m * a.N;
+        float* p = a.acc + m * a.ldacc + n;
+        const float v = __ldcg(p);
+        *p = 0.f;
+        if (a.ydt == AQ_F32) reinterpret_cast<float*>(a.y)[i] = v;
+        else if (a.ydt == AQ_F16) reinterpret_cast<__half*>(a.y)[i] = __float2half_rn(v);
+        else reinterpret_cast<__nv_bfloat16*>(a.y)[i] = __float2bfloat16_rn(v);
+    }
+    if (threadIdx.x == 0) *a.ticket = 0u;
 }
 
 template <int BITS, int MT, bool BF16>
@@ -121,8 +145,9 @@ static cudaError_t launch_mt(const GemvArgs& a, cudaStream_t s) {
 }
 
 cudaError_t launch_gemv(const aq_handle_s* h, const void* x, aq_dtype_t xdt, int M, float* acc, int64_t ldacc,
-                        cudaStream_t s) {
+                        cudaStream_t s, void* y_fused, aq_dtype_t ydt) {
     GemvArgs a;
+    a.y = y_fused; a.ydt = (int)ydt; a.ticket = reinterpret_cast<unsigned int*>(h->flags) + 16;
     a.frags = h->frags; a.x = x; a.acc = acc; a.K = h->K; a.ldacc = ldacc;
     a.n_units = (int64_t)h->KP * h->NT; a.NT = h->NT; a.M = M; a.N = h->N;
     const bool bf = (xdt == AQ_BF16);

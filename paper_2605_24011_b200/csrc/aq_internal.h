@@ -36,9 +36,10 @@ cudaError_t launch_import(const aq_handle_s* h, const uint8_t* canon_dev, cudaSt
 cudaError_t launch_export(const aq_handle_s* h, uint8_t* canon_dev, cudaStream_t s);
 cudaError_t launch_dequant(const aq_handle_s* h, void* out, aq_dtype_t dt, cudaStream_t s);
 
-// decode path: accumulate x W^T into acc (fp32 [M][ldacc]); x is [M][K] of xdt
+// decode path: accumulate x W^T into acc (fp32 [M][ldacc]); x is [M][K] of xdt.  With y_fused the kernel's last CTA
+// also writes y[m][n] = cast(acc[m][n]) (row-major [M][N] of ydt) and leaves acc zero again: acc must be the handle's own
 cudaError_t launch_gemv(const aq_handle_s* h, const void* x, aq_dtype_t xdt, int M, float* acc,
-                        int64_t ldacc, cudaStream_t s);
+                        int64_t ldacc, cudaStream_t s, void* y_fused = nullptr, aq_dtype_t ydt = AQ_F32);
 // y[m][n] = cast(acc[m][n]) for n < N, then acc = 0
 cudaError_t launch_finalize(const float* acc_in, float* acc_zero, int64_t ldacc, void* y, aq_dtype_t ydt,
                             int M, int64_t N, cudaStream_t s);
