@@ -225,3 +225,151 @@ def rms_scale(h: np.ndarray, eps: float = 1e-6) -> np.ndarray:
     """Per-row scalar 1 / sqrt(mean(h^2) + eps) of a gain-free RMS norm, float64."""
     h = np.asarray(h, dtype=np.float64)
     return 1.0 / np.sqrt((h * h).mean(axis=-1, keepdims=True) + eps)
+
+
+# --------------------------------------------------------------------------
+# Intra-tensor scale optimisation [Section 3.3, Eq. 10 and Eq. 11]
+# --------------------------------------------------------------------------
+# Eq. 10: per block, minimise Phi_b = sum_i omega_i (w_i - w_hat_i)^2 with
+# omega_i = F_ii sqrt(sigma_b^2 + w_i^2), sigma_b^2 the block's mean squared weight and F the
+# diagonal Fisher scores (F = 1: the magnitude-weighted row of the ablation table).
+# Eq. 11 alternates nearest codes for a fixed scale with the closed-form scale for fixed codes.
+# The paper writes the symmetric decode s_b q_i; this container decodes scale * q + min
+# (Eq. 1 with a zero point), so the least-squares step here solves for the pair (scale, min):
+# the same stationarity condition with two unknowns.  Reading taken where the paper is silent:
+# start from the round-to-nearest parameters; stop when the normal equations are singular or the
+# scale is not positive; keep the round-to-nearest block when the optimised one, after rounding
+# its parameters to binary16, does not lower Phi_b.
+
+def _omega(Wb: np.ndarray, Fb) -> np.ndarray:
+    """Eq. 10 weights in float64; Wb [..., 32]."""
+    Wb = Wb.astype(np.float64)
+    sig2 = (Wb * Wb).mean(axis=-1, keepdims=True)
+    om = np.sqrt(sig2 + Wb * Wb)
+    return om if Fb is None else om * Fb.astype(np.float64)
+
+
+def block_phi(W: np.ndarray, d, m, q, F=None) -> np.ndarray:
+    """Phi_b of Eq. 10 in float64 for decoded values d q + m; returns [N][K/32]."""
+    N, K = W.shape
+    Wb = np.asarray(W, dtype=np.float64).reshape(N, K // BLOCK, BLOCK)
+    Fb = None if F is None else np.asarray(F).reshape(N, K // BLOCK, BLOCK)
+    what = (np.asarray(d, dtype=np.float64)[:, :, None] * np.asarray(q, dtype=np.float64).reshape(N, K // BLOCK, BLOCK)
+            + np.asarray(m, dtype=np.float64)[:, :, None])
+    return (_omega(Wb, Fb) * (Wb - what) ** 2).sum(axis=2)
+
+
+def scale_opt_ideal(W: np.ndarray, bits: int, F=None, rounds: int = 4):
+    """Eq. 11 in float64 from the round-to-nearest start.  Returns (s, m, q, trace): unrounded
+    parameters [N][K/32], codes [N][K] and Phi_b after every half step (q step, then
+    least-squares step), which Eq. 11 says never goes up."""
+    N, K = W.shape
+    L = float(code_max(bits))
+    Wb = np.asarray(W, dtype=np.float64).reshape(N, K // BLOCK, BLOCK)
+    Fb = None if F is None else np.asarray(F).reshape(N, K // BLOCK, BLOCK)
+    om = _omega(Wb, Fb)
+    mn, mx = Wb.min(axis=2), Wb.max(axis=2)
+    s = (mx - mn) / L
+    m = mn.copy()
+    live = s > 0
+    q = np.zeros_like(Wb)
+    trace = []
+    phi = lambda: (om * (Wb - (s[:, :, None] * q + m[:, :, None])) ** 2).sum(axis=2)
+    for _ in range(rounds):
+        with np.errstate(divide="ignore", invalid="ignore"):
+            t = np.where(live[:, :, None], (Wb - m[:, :, None]) / np.where(live, s, 1.0)[:, :, None], 0.0)
+        q = np.clip(np.floor(t + 0.5), 0, L)
+        trace.append(phi())
+        S0, S1, S2 = om.sum(axis=2), (om * q).sum(axis=2), (om * q * q).sum(axis=2)
+        Sw, Swq = (om * Wb).sum(axis=2), (om * Wb * q).sum(axis=2)
+        det = S0 * S2 - S1 * S1
+        with np.errstate(divide="ignore", invalid="ignore"):
+            s_new = (S0 * Swq - S1 * Sw) / det
+            m_new = (Sw - s_new * S1) / S0
+        ok = live & (det > 0) & np.isfinite(s_new) & (s_new > 0)
+        s = np.where(ok, s_new, s)
+        m = np.where(ok, m_new, m)
+        trace.append(phi())
+    return s, m, q.astype(np.uint8).reshape(N, K), trace
+
+
+def _sum32(x: np.ndarray) -> np.ndarray:
+    """Sum of the last axis (32 float32 values) in the stated order: eight at a time left to
+    right, then (g0 + g1) + (g2 + g3).  One binary32 rounding per addition."""
+    g = x.reshape(x.shape[:-1] + (4, 8)).astype(np.float32)
+    a = g[..., 0]
+    for i in range(1, 8):
+        a = (a + g[..., i]).astype(np.float32)
+    return ((a[..., 0] + a[..., 1]).astype(np.float32) + (a[..., 2] + a[..., 3]).astype(np.float32)).astype(np.float32)
+
+
+def quantize_opt(W: np.ndarray, bits: int, F=None, rounds: int = 4):
+    """Scale-optimised block quantiser [Eq. 10, Eq. 11], same outputs as quantize().
+
+    Every step is one correctly rounded binary32 operation in a stated order (sums: _sum32),
+    except the 2 x 2 solve, done in binary64 from the binary32 sums, one rounding per operation:
+        sigma2 = sum32(w w) / 32;  omega = F * sqrt(sigma2 + w w)            (F omitted when None)
+        s = (max - min) / L, mm = min
+        repeat `rounds` times, while s > 0:
+            q = clamp(rint((w - mm) / s), 0, L)
+            S0 = sum32(omega), S1 = sum32(omega q), S2 = sum32((omega q) q),
+            Sw = sum32(omega w), Swq = sum32((omega w) q)
+            det = S0 S2 - S1 S1; stop unless det > 0
+            s' = (S0 Swq - S1 Sw) / det; stop unless s' is finite and > 0
+            mm = f32((Sw - s' S1) / S0), s = f32(s')
+    Two candidates are then coded exactly as quantize() codes a block from its binary16
+    parameters: (f16((max - min)/L), f16(min)) and (f16(s), f16(mm)); the second is kept when its
+    Phi = sum32(omega (w - (d q + m))^2) is smaller, its scale is finite and non-zero.
+    """
+    W = np.ascontiguousarray(W, dtype=np.float32)
+    N, K = W.shape
+    if K % BLOCK:
+        raise ValueError("K must be a multiple of 32")
+    L = np.float32(code_max(bits))
+    f32 = np.float32
+    Wb = W.reshape(N, K // BLOCK, BLOCK)
+    ww = (Wb * Wb).astype(f32)
+    sig2 = (_sum32(ww) / f32(32)).astype(f32)
+    om = np.sqrt((sig2[:, :, None] + ww).astype(f32)).astype(f32)
+    if F is not None:
+        om = (np.ascontiguousarray(F, dtype=f32).reshape(N, K // BLOCK, BLOCK) * om).astype(f32)
+    mn, mx = Wb.min(axis=2), Wb.max(axis=2)
+    s = ((mx - mn).astype(f32) / L).astype(f32)
+    mm = mn.copy()
+    live = s > 0
+    ow = (om * Wb).astype(f32)
+    S0, Sw = _sum32(om), _sum32(ow)
+    with np.errstate(divide="ignore", invalid="ignore", over="ignore"):
+        for _ in range(rounds):
+            t = ((Wb - mm[:, :, None]).astype(f32) / np.where(live, s, f32(1))[:, :, None]).astype(f32)
+            q = np.clip(np.rint(t), 0, L).astype(f32)
+            oq = (om * q).astype(f32)
+            S1, S2, Swq = _sum32(oq), _sum32((oq * q).astype(f32)), _sum32((ow * q).astype(f32))
+            a0, a1, a2, aw, awq = (v.astype(np.float64) for v in (S0, S1, S2, Sw, Swq))
+            det = a0 * a2 - a1 * a1
+            s_new = (a0 * awq - a1 * aw) / det
+            m_new = (aw - s_new * a1) / a0
+            ok = live & (det > 0) & np.isfinite(s_new) & (s_new > 0)
+            live = ok
+            s = np.where(ok, s_new.astype(f32), s)
+            mm = np.where(ok, m_new.astype(f32), mm)
+
+        def code(dh, mh):
+            d32, m32 = dh.astype(f32)[:, :, None], mh.astype(f32)[:, :, None]
+            t = ((Wb - m32).astype(f32) / d32).astype(f32)
+            t = np.where(d32 == 0, f32(0), t)
+            q = np.clip(np.rint(t), 0, L).astype(f32)
+            what = ((d32 * q).astype(f32) + m32).astype(f32)
+            r = (Wb - what).astype(f32)
+            return q, _sum32((om * (r * r).astype(f32)).astype(f32))
+
+        dA, mA = ((mx - mn).astype(f32) / L).astype(f32).astype(np.float16), mn.astype(np.float16)
+        dB, mB = s.astype(np.float16), mm.astype(np.float16)
+        qA, phiA = code(dA, mA)
+        qB, phiB = code(dB, mB)
+    dB32 = dB.astype(f32)
+    useB = np.isfinite(dB32) & (dB32 != 0) & np.isfinite(mB.astype(f32)) & (phiB < phiA)
+    d = np.where(useB, dB, dA)
+    m = np.where(useB, mB, mA)
+    q = np.where(useB[:, :, None], qB, qA)
+    return d, m, q.astype(np.uint8).reshape(N, K)
