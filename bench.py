@@ -174,7 +174,24 @@ def run_micro(args):
     from paper_2605_24011_b200 import aq, synth, workloads
     torch.cuda.set_device(0)
     out = {"micro": args.micro, "bits": args.bits, "steps": args.steps, "warmup": args.warmup}
-    if args.micro in ("decode_linear", "prefill_linear", "dequant"):
+    if args.micro in ("pack", "pack_opt"):
+        # set-up kernels: float32 weights (and Fisher scores) in, packed fragments out; HBM-bound on the 4 (8) B/weight read
+        N, K = args.N or 16384, args.K or 8192
+        Ws = [synth.weights_device(N, K, 7 + c) for c in range(2)]
+        Fs = [(w * w * 2500.0 + 1e-4) for w in Ws] if args.micro == "pack_opt" else None
+        held = []
+
+        def fn(i):
+            if len(held) >= 2:
+                held.pop(0).free()
+            if args.micro == "pack":
+                held.append(aq.aq_pack(args.bits, 32, Ws[i % 2]))
+            else:
+                held.append(aq.aq_pack_opt(args.bits, 32, Ws[i % 2], Fs[i % 2], rounds=4))
+
+        work, unit = N * K * (4.0 if args.micro == "pack" else 8.0) + N * K * (args.bits + 1) / 8, "GB/s"
+        out.update({"N": N, "K": K, "note": "time includes handle allocation (cudaMalloc / cudaFree) on the host side"})
+    elif args.micro in ("decode_linear", "prefill_linear", "dequant"):
         decode = args.micro == "decode_linear"
         M = args.M or (1 if decode else 512)
         N = args.N or (65536 if decode else 11008)
@@ -338,7 +355,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
     ap.add_argument("--layers", type=int, default=32, help="decoder layers (32 = the full workload)")
     ap.add_argument("--no-extras", action="store_true", help="skip prefill / dequant / oracle legs")
-    ap.add_argument("--micro", choices=("decode_linear", "prefill_linear", "dequant", "decode_stack", "prefill_stack"),
+    ap.add_argument("--micro", choices=("decode_linear", "prefill_linear", "dequant", "decode_stack", "prefill_stack", "pack", "pack_opt"),
                     help="time one kernel on a small case (the command ncu captures are taken from) instead of the benchmark")
     ap.add_argument("--configs", action="store_true",
                     help="time all five workload configurations once each and print one JSON object (not the benchmark line)")

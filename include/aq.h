@@ -75,6 +75,23 @@ aq_status_t aq_pack(int bits, int block, const float* W_dev, int64_t N, int64_t 
                     aq_stream_t stream, aq_handle_t* out);
 
 /*
+ * aq_pack_opt -- quantise and pack with optimised block parameters (Section 3.3, "Intra-Tensor Scale
+ * Optimization": Eq. 10, the weighted block objective Phi_b with omega = F sqrt(sigma_b^2 + w^2); Eq. 11,
+ * the alternation of nearest codes and the closed-form parameters).
+ *   arguments as aq_pack, plus
+ *   F_dev  : DEVICE, float32, row-major [N][K], 16-byte aligned: the diagonal Fisher scores of Eq. 9, or
+ *            NULL for F = 1 (the magnitude-weighted variant of the ablation table)
+ *   rounds : alternations of Eq. 11 (0 .. 64; 0 gives aq_pack's result)
+ * The paper's decode in Eq. 10 is s q; this container decodes scale * q + min, so the closed-form step solves the
+ * weighted least squares for the pair (scale, min).  Start: the round-to-nearest parameters.  A block keeps its
+ * round-to-nearest form when the optimised parameters, rounded to binary16, do not lower Phi_b, so no block is
+ * worse than aq_pack's under Eq. 10.  Each arithmetic step is one correctly rounded operation in a fixed order:
+ * the result is reproducible bit for bit.  Errors as aq_pack.
+ */
+aq_status_t aq_pack_opt(int bits, int block, const float* W_dev, const float* F_dev, int rounds, int64_t N, int64_t K,
+                        aq_stream_t stream, aq_handle_t* out);
+
+/*
  * aq_import -- build a handle from canonical bytes (Appendix D container).
  *   canon_host : HOST, nbytes == N*K*(bits+1)/8 bytes in the layout above
  * Synchronises `stream` before returning (the host buffer may be reused).

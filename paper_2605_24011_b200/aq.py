@@ -25,7 +25,7 @@ AQ_IN_PLAIN, AQ_IN_RMSNORM, AQ_IN_SILU_MUL = 0, 1, 2
 AQ_OUT_STORE, AQ_OUT_ADD = 0, 1
 AQ_MAX_M, AQ_DECODE_MAX_M = 4096, 8
 
-SYMBOLS = ("aq_pack", "aq_import", "aq_export", "aq_info", "aq_dequant", "aq_linear", "aq_linear_f32out", "aq_linear_noalloc",
+SYMBOLS = ("aq_pack", "aq_pack_opt", "aq_import", "aq_export", "aq_info", "aq_dequant", "aq_linear", "aq_linear_f32out", "aq_linear_noalloc",
            "aq_stack_workspace_bytes", "aq_stack_forward", "aq_stack_buffer_offset", "aq_stack_input_offset", "aq_check", "aq_free",
            "aq_status_string", "aq_last_cuda_error", "aq_kernel_launches")
 
@@ -43,6 +43,8 @@ class Stack(C.Structure):
 
 
 _lib.aq_pack.argtypes = [C.c_int, C.c_int, C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.POINTER(_H)]
+_lib.aq_pack_opt.argtypes = [C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_void_p, C.POINTER(_H)]
+_lib.aq_pack_opt.restype = C.c_int
 _lib.aq_import.argtypes = [C.c_int, C.c_int, C.c_int64, C.c_int64, C.c_void_p, C.c_size_t, C.c_void_p, C.POINTER(_H)]
 _lib.aq_export.argtypes = [_H, C.c_void_p, C.c_size_t, C.POINTER(C.c_size_t)]
 _lib.aq_info.argtypes = [_H, C.POINTER(C.c_int), C.POINTER(C.c_int), C.POINTER(C.c_int64), C.POINTER(C.c_int64),
@@ -144,6 +146,14 @@ def aq_pack(bits: int, block: int, W, stream=None) -> Handle:
     N, K = W.shape
     h = _H()
     _check(_lib.aq_pack(bits, block, _ptr(W), N, K, _stream(stream), C.byref(h)), "aq_pack")
+    return Handle(h.value)
+
+
+def aq_pack_opt(bits: int, block: int, W, F=None, rounds: int = 4, stream=None) -> Handle:
+    """W: CUDA float32 [N][K]; F: CUDA float32 [N][K] Fisher scores or None (= 1)."""
+    N, K = W.shape
+    h = _H()
+    _check(_lib.aq_pack_opt(bits, block, _ptr(W), _ptr(F), rounds, N, K, _stream(stream), C.byref(h)), "aq_pack_opt")
     return Handle(h.value)
 
 

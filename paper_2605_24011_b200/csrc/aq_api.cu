@@ -104,6 +104,24 @@ aq_status_t aq_pack(int bits, int block, const float* W_dev, int64_t N, int64_t 
     return AQ_OK;
 }
 
+aq_status_t aq_pack_opt(int bits, int block, const float* W_dev, const float* F_dev, int rounds, int64_t N, int64_t K,
+                        aq_stream_t stream, aq_handle_t* out) {
+    if (!out) return AQ_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!W_dev || !aligned16(W_dev) || (F_dev && !aligned16(F_dev)) || rounds < 0 || rounds > 64) return AQ_ERR_INVALID_ARG;
+    aq_handle_t h = nullptr;
+    aq_status_t st = new_handle(bits, block, N, K, &h);
+    if (st != AQ_OK) return st;
+    cudaStream_t s = (cudaStream_t)stream;
+    cudaError_t e = cudaMemsetAsync(h->acc, 0, (size_t)AQ_DECODE_MAX_M * h->NT * 16 * sizeof(float), s);
+    if (e == cudaSuccess) e = cudaMemsetAsync(h->flags, 0, 256, s);
+    if (e == cudaSuccess) e = launch_pack_opt(h, W_dev, F_dev, rounds, s);
+    if (e != cudaSuccess) { destroy(h); return cuda_fail(e); }
+    h->last_stream = s;
+    *out = h;
+    return AQ_OK;
+}
+
 aq_status_t aq_import(int bits, int block, int64_t N, int64_t K, const void* canon_host, size_t nbytes,
                       aq_stream_t stream, aq_handle_t* out) {
     if (!out) return AQ_ERR_INVALID_ARG;

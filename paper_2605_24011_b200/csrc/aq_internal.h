@@ -32,6 +32,7 @@ bool handle_ok(aq_handle_t h);
 
 // launchers (each checks nothing: arguments are validated by the API layer)
 cudaError_t launch_pack(const aq_handle_s* h, const float* W, cudaStream_t s);
+cudaError_t launch_pack_opt(const aq_handle_s* h, const float* W, const float* F, int rounds, cudaStream_t s);
 cudaError_t launch_import(const aq_handle_s* h, const uint8_t* canon_dev, cudaStream_t s);
 cudaError_t launch_export(const aq_handle_s* h, uint8_t* canon_dev, cudaStream_t s);
 cudaError_t launch_dequant(const aq_handle_s* h, void* out, aq_dtype_t dt, cudaStream_t s);
