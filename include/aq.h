@@ -91,6 +91,58 @@ aq_status_t aq_pack(int bits, int block, const float* W_dev, int64_t N, int64_t 
 aq_status_t aq_pack_opt(int bits, int block, const float* W_dev, const float* F_dev, int rounds, int64_t N, int64_t K,
                         aq_stream_t stream, aq_handle_t* out);
 
+/* ---- inter-tensor stage (Section 4.1): HSIC sensitivities and bit allocation ------------------------------
+ * The three device calls below share one static device scratch area: issue them on one stream (or otherwise
+ * serialised).  None of them allocates memory. */
+#define AQ_HSIC_MAX_K 16384
+
+/*
+ * aq_rbf_gram -- RBF kernel matrix of K calibration samples (Section 3, "HSIC": [K_A]_ij = k(a_i, a_j) with the
+ * Gaussian kernel k(a, a') = exp(-|a - a'|^2 / (2 sigma^2)); the paper prints no bandwidth, sigma is the caller's).
+ *   A_dev  : DEVICE, [K][d] row-major, AQ_F16 or AQ_BF16 (activations are kept at half precision), 16-byte
+ *            aligned; d % 8 == 0 (pad with zero columns: they do not change a distance)
+ *   K      : 2 .. AQ_HSIC_MAX_K samples;  d >= 8 features;  sigma > 0 and finite
+ *   G_dev  : DEVICE, float32 [K][ldg], ldg >= K; receives the full symmetric matrix, diagonal exactly 1
+ * Squared distances are formed as n_i + n_j - 2 <a_i, a_j> (clamped at 0) from exact products accumulated in
+ * binary32 on the tensor cores.  Asynchronous on `stream`; a wait that runs out is reported by aq_check.
+ */
+aq_status_t aq_rbf_gram(const void* A_dev, aq_dtype_t dtype, int64_t K, int64_t d, float sigma, float* G_dev,
+                        int64_t ldg, aq_stream_t stream);
+
+/*
+ * aq_hsic -- the empirical criterion of Eq. 2, (K-1)^-2 tr(K_A C K_B C) with C = I - 11^T/K.
+ *   KA_dev, KB_dev : DEVICE, float32 [K][ld] symmetric kernel matrices (e.g. from aq_rbf_gram), ld >= K
+ *   out_dev        : DEVICE, one binary64 value
+ * Evaluated in binary64 in a fixed order (reproducible).  Asynchronous on `stream`.
+ */
+aq_status_t aq_hsic(const float* KA_dev, const float* KB_dev, int64_t K, int64_t ld, double* out_dev,
+                    aq_stream_t stream);
+
+/*
+ * aq_sensitivity -- Eq. 5: S = -alpha HSIC(X, Z) + beta HSIC(Z, Y) for one weight matrix, from the kernel
+ * matrices of the backbone inputs X, the matrix's outputs Z and the action labels Y.
+ *   out3_dev : DEVICE, three binary64 values: S, HSIC(X, Z), HSIC(Z, Y)
+ *   alpha, beta >= 0.  Other arguments as aq_hsic.
+ */
+aq_status_t aq_sensitivity(const float* KX_dev, const float* KZ_dev, const float* KY_dev, int64_t K, int64_t ld,
+                           double alpha, double beta, double* out3_dev, aq_stream_t stream);
+
+/*
+ * aq_allocate_bits -- the layer-balanced allocation of Eq. 6 by the greedy solver of Section 4.1 (HOST only).
+ * Minimises sum_l E_l^2, E_l = sum_{j in layer l} S_j 2^(-2 b_j), subject to the parameter-weighted mean of b_j
+ * being <= budget.
+ *   S, numel, layer_of : HOST arrays of n entries: sensitivity (Eq. 5), number of weights, layer index (>= 0)
+ *   types              : HOST, n_types strictly ascending bit-widths (1..16), e.g. {2, 3, 4}
+ *   bits_out           : HOST, n entries;  objective_out : HOST, may be NULL
+ * Every matrix starts at types[0]; each step applies, among the upgrades to the next type that keep the budget,
+ * the one with the largest (E_l^2 - E~_l^2) / ((b_new - b_old) numel); it stops when none is left or the best
+ * one does not lower the objective (ties: lowest index).  AQ_ERR_INVALID_ARG for malformed input,
+ * AQ_ERR_RANGE when the budget is below types[0].
+ */
+aq_status_t aq_allocate_bits(const double* S, const int64_t* numel, const int32_t* layer_of, int64_t n,
+                             const int32_t* types, int n_types, double budget, int32_t* bits_out,
+                             double* objective_out);
+
 /*
  * aq_import -- build a handle from canonical bytes (Appendix D container).
  *   canon_host : HOST, nbytes == N*K*(bits+1)/8 bytes in the layout above

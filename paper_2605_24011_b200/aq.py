@@ -26,6 +26,7 @@ AQ_OUT_STORE, AQ_OUT_ADD = 0, 1
 AQ_MAX_M, AQ_DECODE_MAX_M = 4096, 8
 
 SYMBOLS = ("aq_pack", "aq_pack_opt", "aq_import", "aq_export", "aq_info", "aq_dequant", "aq_linear", "aq_linear_f32out", "aq_linear_noalloc",
+           "aq_rbf_gram", "aq_hsic", "aq_sensitivity", "aq_allocate_bits",
            "aq_stack_workspace_bytes", "aq_stack_forward", "aq_stack_buffer_offset", "aq_stack_input_offset", "aq_check", "aq_free",
            "aq_status_string", "aq_last_cuda_error", "aq_kernel_launches")
 
@@ -45,6 +46,15 @@ class Stack(C.Structure):
 _lib.aq_pack.argtypes = [C.c_int, C.c_int, C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.POINTER(_H)]
 _lib.aq_pack_opt.argtypes = [C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_void_p, C.POINTER(_H)]
 _lib.aq_pack_opt.restype = C.c_int
+_lib.aq_rbf_gram.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_float, C.c_void_p, C.c_int64, C.c_void_p]
+_lib.aq_rbf_gram.restype = C.c_int
+_lib.aq_hsic.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p]
+_lib.aq_hsic.restype = C.c_int
+_lib.aq_sensitivity.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_double, C.c_double, C.c_void_p, C.c_void_p]
+_lib.aq_sensitivity.restype = C.c_int
+_lib.aq_allocate_bits.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_int, C.c_double, C.c_void_p,
+                                  C.POINTER(C.c_double)]
+_lib.aq_allocate_bits.restype = C.c_int
 _lib.aq_import.argtypes = [C.c_int, C.c_int, C.c_int64, C.c_int64, C.c_void_p, C.c_size_t, C.c_void_p, C.POINTER(_H)]
 _lib.aq_export.argtypes = [_H, C.c_void_p, C.c_size_t, C.POINTER(C.c_size_t)]
 _lib.aq_info.argtypes = [_H, C.POINTER(C.c_int), C.POINTER(C.c_int), C.POINTER(C.c_int64), C.POINTER(C.c_int64),
@@ -155,6 +165,58 @@ def aq_pack_opt(bits: int, block: int, W, F=None, rounds: int = 4, stream=None) 
     h = _H()
     _check(_lib.aq_pack_opt(bits, block, _ptr(W), _ptr(F), rounds, N, K, _stream(stream), C.byref(h)), "aq_pack_opt")
     return Handle(h.value)
+
+
+def aq_rbf_gram(A, sigma: float, G=None, stream=None):
+    """A: CUDA float16 / bfloat16 [K][d]; returns (or fills) the float32 [K][K] RBF kernel matrix."""
+    import torch
+    K, d = A.shape
+    if G is None:
+        G = torch.empty((K, K), dtype=torch.float32, device=A.device)
+    _check(_lib.aq_rbf_gram(_ptr(A), dtype_code(A), K, d, float(sigma), _ptr(G), G.stride(0), _stream(stream)), "aq_rbf_gram")
+    return G
+
+
+def aq_hsic(KA, KB, out=None, stream=None):
+    """KA, KB: CUDA float32 [K][K] (same row pitch); returns a CUDA float64 tensor of one element."""
+    import torch
+    K = KA.shape[0]
+    if out is None:
+        out = torch.empty(1, dtype=torch.float64, device=KA.device)
+    if KA.stride(0) != KB.stride(0):
+        raise ValueError("aq_hsic: the two matrices need the same row pitch")
+    _check(_lib.aq_hsic(_ptr(KA), _ptr(KB), K, KA.stride(0), _ptr(out), _stream(stream)), "aq_hsic")
+    return out
+
+
+def aq_sensitivity(KX, KZ, KY, alpha: float, beta: float, out=None, stream=None):
+    """Returns a CUDA float64 tensor [S, HSIC(X, Z), HSIC(Z, Y)]."""
+    import torch
+    K = KZ.shape[0]
+    if out is None:
+        out = torch.empty(3, dtype=torch.float64, device=KZ.device)
+    if not (KX.stride(0) == KZ.stride(0) == KY.stride(0)):
+        raise ValueError("aq_sensitivity: the three matrices need the same row pitch")
+    _check(_lib.aq_sensitivity(_ptr(KX), _ptr(KZ), _ptr(KY), K, KZ.stride(0), float(alpha), float(beta), _ptr(out), _stream(stream)),
+           "aq_sensitivity")
+    return out
+
+
+def aq_allocate_bits(S, numel, layer_of, types, budget: float):
+    """Host call: returns (bits per matrix as a numpy int32 array, objective)."""
+    import numpy as np
+    S = np.ascontiguousarray(S, dtype=np.float64)
+    numel = np.ascontiguousarray(numel, dtype=np.int64)
+    layer_of = np.ascontiguousarray(layer_of, dtype=np.int32)
+    types = np.ascontiguousarray(types, dtype=np.int32)
+    n = S.shape[0]
+    if numel.shape[0] != n or layer_of.shape[0] != n:
+        raise ValueError("aq_allocate_bits: arrays of different length")
+    bits = np.empty(n, dtype=np.int32)
+    obj = C.c_double()
+    _check(_lib.aq_allocate_bits(S.ctypes.data, numel.ctypes.data, layer_of.ctypes.data, n, types.ctypes.data, types.shape[0],
+                                 float(budget), bits.ctypes.data, C.byref(obj)), "aq_allocate_bits")
+    return bits, obj.value
 
 
 def aq_pack_raw(bits, block, w_ptr, N, K, stream_ptr=0):

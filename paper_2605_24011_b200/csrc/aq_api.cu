@@ -1,4 +1,5 @@
 // C-ABI entry points of libaq: argument checks, handle ownership, dispatch.
+#include <cmath>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -233,11 +234,53 @@ aq_status_t aq_linear_f32out(aq_handle_t h, const void* x_dev, float* y_dev, int
     return linear_common(h, x_dev, y_dev, M, x_dtype, AQ_F32, stream);
 }
 
+aq_status_t aq_rbf_gram(const void* A_dev, aq_dtype_t dtype, int64_t K, int64_t d, float sigma, float* G_dev, int64_t ldg,
+                        aq_stream_t stream) {
+    if (!A_dev || !G_dev || !aligned16(A_dev) || (reinterpret_cast<uintptr_t>(G_dev) & 3u)) return AQ_ERR_INVALID_ARG;
+    if (dtype != AQ_F16 && dtype != AQ_BF16) return AQ_ERR_UNSUPPORTED;
+    if (K < 2 || K > AQ_HSIC_MAX_K || d < 8 || d % 8 != 0 || d > (1 << 24) || ldg < K) return AQ_ERR_INVALID_ARG;
+    if (!(sigma > 0.f) || !std::isfinite(sigma) || !std::isfinite(1.0f / (2.0f * sigma * sigma))) return AQ_ERR_INVALID_ARG;
+    aq_status_t st = check_arch(nullptr);
+    if (st != AQ_OK) return st;
+    const cudaError_t e = launch_rbf_gram(A_dev, dtype, K, d, sigma, G_dev, ldg, (cudaStream_t)stream);
+    return e == cudaSuccess ? AQ_OK : cuda_fail(e);
+}
+
+aq_status_t aq_hsic(const float* KA_dev, const float* KB_dev, int64_t K, int64_t ld, double* out_dev, aq_stream_t stream) {
+    if (!KA_dev || !KB_dev || !out_dev || (reinterpret_cast<uintptr_t>(out_dev) & 7u)) return AQ_ERR_INVALID_ARG;
+    if (K < 2 || K > AQ_HSIC_MAX_K || ld < K) return AQ_ERR_INVALID_ARG;
+    aq_status_t st = check_arch(nullptr);
+    if (st != AQ_OK) return st;
+    const cudaError_t e = launch_hsic(KA_dev, KB_dev, K, ld, ld, out_dev, 0, 0.0, 0.0, (cudaStream_t)stream);
+    return e == cudaSuccess ? AQ_OK : cuda_fail(e);
+}
+
+aq_status_t aq_sensitivity(const float* KX_dev, const float* KZ_dev, const float* KY_dev, int64_t K, int64_t ld, double alpha,
+                           double beta, double* out3_dev, aq_stream_t stream) {
+    if (!KX_dev || !KZ_dev || !KY_dev || !out3_dev || (reinterpret_cast<uintptr_t>(out3_dev) & 7u)) return AQ_ERR_INVALID_ARG;
+    if (K < 2 || K > AQ_HSIC_MAX_K || ld < K || !(alpha >= 0.0) || !(beta >= 0.0) || !std::isfinite(alpha) || !std::isfinite(beta))
+        return AQ_ERR_INVALID_ARG;
+    aq_status_t st = check_arch(nullptr);
+    if (st != AQ_OK) return st;
+    cudaError_t e = launch_hsic(KX_dev, KZ_dev, K, ld, ld, out3_dev, 1, alpha, beta, (cudaStream_t)stream);
+    if (e == cudaSuccess) e = launch_hsic(KZ_dev, KY_dev, K, ld, ld, out3_dev, 2, alpha, beta, (cudaStream_t)stream);
+    return e == cudaSuccess ? AQ_OK : cuda_fail(e);
+}
+
+aq_status_t aq_allocate_bits(const double* S, const int64_t* numel, const int32_t* layer_of, int64_t n, const int32_t* types,
+                             int n_types, double budget, int32_t* bits_out, double* objective_out) {
+    if (!S || !numel || !layer_of || !types || !bits_out || n < 1 || n_types < 1 || !std::isfinite(budget)) return AQ_ERR_INVALID_ARG;
+    for (int64_t j = 0; j < n; ++j)
+        if (!std::isfinite(S[j])) return AQ_ERR_INVALID_ARG;
+    const int r = allocate_bits_host(S, numel, layer_of, n, types, n_types, budget, bits_out, objective_out);
+    return r == 0 ? AQ_OK : (r == 2 ? AQ_ERR_RANGE : AQ_ERR_INVALID_ARG);
+}
+
 aq_status_t aq_check(aq_stream_t stream) {
     cudaError_t e = cudaStreamSynchronize((cudaStream_t)stream);
     if (e != cudaSuccess) return cuda_fail(e);
-    const int g = read_gemm_status(true), d = read_decode_status(true);
-    return (g || d) ? AQ_ERR_TIMEOUT : AQ_OK;
+    const int g = read_gemm_status(true), d = read_decode_status(true), t = read_stage1_status(true);
+    return (g || d || t) ? AQ_ERR_TIMEOUT : AQ_OK;
 }
 
 void aq_free(aq_handle_t h) {

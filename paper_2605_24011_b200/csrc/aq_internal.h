@@ -92,6 +92,16 @@ static inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 blo
 }
 #endif
 
+// inter-tensor stage (aq_stage1.cu)
+cudaError_t launch_rbf_gram(const void* A, aq_dtype_t dt, int64_t K, int64_t d, float sigma, float* out, int64_t ld,
+                            cudaStream_t s);
+// combine: 0 = out[0] receives Eq. 2; 1, 2 = out[combine] receives it, and with 2 also out[0] = -alpha out[1] + beta out[2]
+cudaError_t launch_hsic(const float* KA, const float* KB, int64_t K, int64_t lda, int64_t ldb, double* out, int combine,
+                        double alpha, double beta, cudaStream_t s);
+int allocate_bits_host(const double* S, const int64_t* numel, const int32_t* layer_of, int64_t n, const int32_t* types,
+                       int n_types, double budget, int32_t* bits_out, double* objective_out);   // 0 ok, 1 malformed, 2 budget
+int read_stage1_status(bool clear);
+
 int sm_count();
 void count_launch(int n = 1);       // process-wide count of this library's kernel launches
 int read_gemm_status(bool clear);   // nonzero: a bounded wait in the GEMM kernel ran out

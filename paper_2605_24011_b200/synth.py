@@ -127,3 +127,28 @@ def weights_device(N: int, K: int, seed: int, outliers: bool = False, device="cu
         mask = torch.empty((N, K), dtype=torch.float32, device=device).uniform_(0.0, 1.0, generator=g) < 0.001
         W = torch.where(mask, W * 20.0, W)
     return W
+
+
+def calibration(K: int, d_in: int, d_out: int, d_act: int, *key, relevance: float = 0.5, redundancy: float = 0.5):
+    """Calibration samples for the inter-tensor stage (Section 4.1): backbone inputs X [K][d_in], the outputs
+    Z [K][d_out] of one weight matrix and action labels Y [K][d_act], float32, roughly unit variance per feature.
+    Z mixes a random projection of X (weight `redundancy`), a latent that also drives Y (weight `relevance`) and
+    independent noise, so that HSIC(X, Z) and HSIC(Z, Y) move with the two knobs."""
+    g = _rng(0xCA, *key)
+    X = g.standard_normal((K, d_in), dtype=np.float32)
+    latent = g.standard_normal((K, d_act), dtype=np.float32)
+    P = g.standard_normal((d_in, d_out), dtype=np.float32) / np.float32(np.sqrt(d_in))
+    R = g.standard_normal((d_act, d_out), dtype=np.float32) / np.float32(np.sqrt(d_act))
+    noise = g.standard_normal((K, d_out), dtype=np.float32)
+    rest = max(0.0, 1.0 - redundancy**2 - relevance**2) ** 0.5
+    Z = (np.float32(redundancy) * np.tanh(X @ P) * np.float32(1.6) + np.float32(relevance) * (latent @ R) + np.float32(rest) * noise)
+    Y = np.tanh(latent) + np.float32(0.1) * g.standard_normal((K, d_act), dtype=np.float32)
+    return X, Z.astype(np.float32), Y.astype(np.float32)
+
+
+def sensitivities(n_layers: int, per_layer: int, *key) -> np.ndarray:
+    """Seeded stand-in for the Eq. 5 scores of a stack: positive, log-normally spread, a fifth of them negative."""
+    g = _rng(0x5E, *key)
+    S = np.exp(g.standard_normal(n_layers * per_layer)) * 1e-3
+    S[g.random(n_layers * per_layer) < 0.2] *= -0.3
+    return S
