@@ -191,6 +191,24 @@ def run_micro(args):
 
         work, unit = N * K * (4.0 if args.micro == "pack" else 8.0) + N * K * (args.bits + 1) / 8, "GB/s"
         out.update({"N": N, "K": K, "note": "time includes handle allocation (cudaMalloc / cudaFree) on the host side"})
+    elif args.micro in ("rbf_gram", "hsic"):
+        # inter-tensor stage: kernel matrix of K calibration samples with d features (tensor-bound), HSIC over two such
+        # matrices (HBM-bound: each read once)
+        K, d = args.M or 4096, args.K or 11008
+        if args.micro == "rbf_gram":
+            As = [workloads.activations_device(K, d, torch.bfloat16, 11, c) for c in range(2)]
+            G = torch.empty((K, K), dtype=torch.float32, device="cuda")
+            fn = lambda i: aq.aq_rbf_gram(As[i % 2], float(d) ** 0.5, G=G)
+            # inner products needed for a symmetric matrix: K (K + 1) / 2, each 2 d flops
+            work, unit = float(K) * (K + 1) * d, "TFLOP/s"
+        else:
+            n_copies = max(2, int(300e6 // (K * K * 4)) + 1)
+            A = workloads.activations_device(K, 512, torch.bfloat16, 12, 0)
+            Gs = [aq.aq_rbf_gram(A, 512.0 ** 0.5) for _ in range(2 * n_copies)]
+            res = torch.empty(1, dtype=torch.float64, device="cuda")
+            fn = lambda i: aq.aq_hsic(Gs[2 * (i % n_copies)], Gs[2 * (i % n_copies) + 1], out=res)
+            work, unit = 2.0 * K * K * 4, "GB/s"
+        out.update({"K_samples": K, "d": d})
     elif args.micro in ("decode_linear", "prefill_linear", "dequant"):
         decode = args.micro == "decode_linear"
         M = args.M or (1 if decode else 512)
@@ -355,7 +373,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
     ap.add_argument("--layers", type=int, default=32, help="decoder layers (32 = the full workload)")
     ap.add_argument("--no-extras", action="store_true", help="skip prefill / dequant / oracle legs")
-    ap.add_argument("--micro", choices=("decode_linear", "prefill_linear", "dequant", "decode_stack", "prefill_stack", "pack", "pack_opt"),
+    ap.add_argument("--micro", choices=("decode_linear", "prefill_linear", "dequant", "decode_stack", "prefill_stack", "pack", "pack_opt", "rbf_gram", "hsic"),
                     help="time one kernel on a small case (the command ncu captures are taken from) instead of the benchmark")
     ap.add_argument("--configs", action="store_true",
                     help="time all five workload configurations once each and print one JSON object (not the benchmark line)")

@@ -266,7 +266,24 @@ __global__ void __launch_bounds__(256) hsic_rows_kernel(const float* __restrict_
     const float* pa = KA + (int64_t)row * lda;
     const float* pb = KB + (int64_t)row * ldb;
     double ra = 0.0, rb = 0.0, p = 0.0;
-    for (int j = lane; j < K; j += 32) {
+    int j0 = 0;
+    if (((lda | ldb) & 3) == 0 && ((reinterpret_cast<uintptr_t>(KA) | reinterpret_cast<uintptr_t>(KB)) & 15u) == 0) {
+        // four columns per lane and step, two steps in flight
+        const int K4 = K & ~255;
+        for (int j = 4 * lane; j < K4; j += 256) {
+            const float4 x0 = __ldg(reinterpret_cast<const float4*>(pa + j)), y0 = __ldg(reinterpret_cast<const float4*>(pb + j));
+            const float4 x1 = __ldg(reinterpret_cast<const float4*>(pa + j + 128)), y1 = __ldg(reinterpret_cast<const float4*>(pb + j + 128));
+            const float xs[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+            const float ys[8] = {y0.x, y0.y, y0.z, y0.w, y1.x, y1.y, y1.z, y1.w};
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                const double x = (double)xs[q], y = (double)ys[q];
+                ra += x; rb += y; p = fma(x, y, p);
+            }
+        }
+        j0 = K4;
+    }
+    for (int j = j0 + lane; j < K; j += 32) {
         const double x = (double)__ldg(pa + j), y = (double)__ldg(pb + j);
         ra += x; rb += y; p = fma(x, y, p);
     }
