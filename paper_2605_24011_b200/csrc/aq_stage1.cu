@@ -201,6 +201,142 @@ __global__ void __launch_bounds__(S1_THREADS, 2) gram_rbf_kernel(const __grid_co
     }
 }
 
+
+// The same computation on CTA pairs: a 256 x 256 tile per pair, tcgen05 cta_group::2.  Each CTA brings in its own 128 rows
+// of both operands (half the shared-memory traffic per flop of the kernel above) and keeps its 128 x 256 part of the
+// accumulator; the even CTA issues the MMAs and its barriers collect both CTAs' loads.
+template <bool BF16>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(S1_THREADS, 2)
+gram_rbf_pair_kernel(const __grid_constant__ CUtensorMap tmap, const GramArgs a) {
+    constexpr int TW = 2 * S1_TILE;   // tile side
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t* sA = smem;
+    uint8_t* sB = sA + S1_STAGES * S1_OP_BYTES;
+    float* s_nj = reinterpret_cast<float*>(sB + S1_STAGES * S1_OP_BYTES);   // [256] column norms
+    uint64_t* bars = reinterpret_cast<uint64_t*>(s_nj + TW);
+    const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * S1_STAGES, bar_accum = bar_empty + 8 * S1_STAGES;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S1_STAGES + 1);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_rank();
+
+    int ti = 0, t = (int)(blockIdx.x >> 1);
+    while (t >= a.n_t - ti) { t -= a.n_t - ti; ++ti; }
+    const int tj = ti + t;
+    const bool diag = (ti == tj);
+    const int n_k = (a.d + S1_KSTAGE - 1) / S1_KSTAGE;
+    const int rowA0 = ti * TW + (int)rank * S1_TILE, rowB0 = tj * TW + (int)rank * S1_TILE;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S1_STAGES; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
+        mbar_init(bar_accum, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {   // the same warp of both CTAs allocates, with the same destination
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)TW) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();   // the partner's barriers exist before anything is counted on them
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            const uint32_t per_cta = (uint32_t)(diag ? S1_OP_BYTES : 2 * S1_OP_BYTES);
+            bool ok = true;
+            for (int kb = 0; kb < n_k && ok; ++kb) {
+                const uint32_t s = kb % S1_STAGES;
+                ok = s1_wait(bar_empty + 8 * s, ((kb / S1_STAGES) & 1) ^ 1, abort_flag, 4);
+                if (!ok) break;
+                const uint32_t full0 = cluster_map(bar_full + 8 * s, 0);
+                if (rank == 0) mbar_expect_tx(bar_full + 8 * s, 2 * per_cta);
+                tma_load_2d_pair(smem_u32(sA + s * S1_OP_BYTES), &tmap, kb * S1_KSTAGE, rowA0, full0);
+                if (!diag) tma_load_2d_pair(smem_u32(sB + s * S1_OP_BYTES), &tmap, kb * S1_KSTAGE, rowB0, full0);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && rank == 0) {
+            const uint32_t idesc = (1u << 4) | ((BF16 ? 1u : 0u) << 7) | ((BF16 ? 1u : 0u) << 10) |
+                                   ((uint32_t)(TW >> 3) << 17) | ((uint32_t)(TW >> 4) << 24);
+            bool ok = true;
+            for (int kb = 0; kb < n_k && ok; ++kb) {
+                const uint32_t s = kb % S1_STAGES;
+                ok = s1_wait(bar_full + 8 * s, (kb / S1_STAGES) & 1, abort_flag, 5);
+                if (!ok) break;
+                tc_fence_after();
+                const uint64_t ad = make_smem_desc(smem_u32(sA + s * S1_OP_BYTES));
+                const uint64_t bd = diag ? ad : make_smem_desc(smem_u32(sB + s * S1_OP_BYTES));
+#pragma unroll
+                for (int k = 0; k < S1_KSTAGE / 16; ++k)
+                    umma_f16_pair(tmem_base, ad + 2 * k, bd + 2 * k, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+                umma_commit_pair(bar_empty + 8 * s);                    // both CTAs' stage s may be refilled
+                umma_commit_pair(cluster_map(bar_empty + 8 * s, 1));
+            }
+            if (ok) {
+                umma_commit_pair(bar_accum);
+                umma_commit_pair(cluster_map(bar_accum, 1));
+            }
+        }
+    } else {
+        const int lq = warp & 3;
+        const int e = threadIdx.x - 64;   // 0..127
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int jg = tj * TW + e + h * S1_TILE;
+            s_nj[e + h * S1_TILE] = (jg < a.K) ? __ldg(a.norms + jg) : 0.f;
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        const int i = rowA0 + lq * 32 + lane;
+        const float ni = (i < a.K) ? __ldg(a.norms + i) : 0.f;
+        const bool ok = s1_wait(bar_accum, 0, abort_flag, 6);
+        if (ok) {
+            tc_fence_after();
+            const bool vec = (a.ld % 4 == 0) && ((reinterpret_cast<uintptr_t>(a.out) & 15u) == 0);
+            for (int c0 = 0; c0 < TW; c0 += 32) {
+                const int j0 = tj * TW + c0;
+                if (j0 >= a.K) break;                         // (the same for the whole warp)
+                uint32_t v[32];
+                tmem_ld32(tmem_base + ((uint32_t)(lq * 32) << 16) + (uint32_t)c0, v);
+                tmem_ld_wait();
+                float kv[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    const float dist = fmaxf(ni + s_nj[c0 + j] - 2.f * __uint_as_float(v[j]), 0.f);
+                    kv[j] = (i == j0 + j) ? 1.f : expf(-dist * a.c);
+                }
+                if (i < a.K) {
+                    float* row = a.out + (int64_t)i * a.ld + j0;
+                    if (vec && j0 + 32 <= a.K) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4) *reinterpret_cast<float4*>(row + j) = make_float4(kv[j], kv[j + 1], kv[j + 2], kv[j + 3]);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (j0 + j < a.K) row[j] = kv[j];
+                    }
+                    if (!diag) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (j0 + j < a.K) a.out[(int64_t)(j0 + j) * a.ld + i] = kv[j];
+                    }
+                }
+            }
+        }
+        tc_fence_before();
+    }
+    __syncthreads();
+    if (*abort_flag) __nanosleep(200000);
+    cluster_sync_all();   // nothing of the partner (its operand tiles, its barriers) is in use any more
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TW) : "memory");
+    }
+}
+
 cudaError_t launch_rbf_gram(const void* A, aq_dtype_t dt, int64_t K, int64_t d, float sigma, float* out, int64_t ld,
                             cudaStream_t s) {
     EncodeTiledFn enc = tensor_map_encoder();
@@ -226,29 +362,27 @@ cudaError_t launch_rbf_gram(const void* A, aq_dtype_t dt, int64_t K, int64_t d, 
         return cudaErrorInvalidValue;
     GramArgs a;
     a.norms = norms; a.out = out; a.ld = ld; a.K = (int)K; a.d = (int)d;
-    a.n_t = (int)((K + S1_TILE - 1) / S1_TILE);
     a.c = 1.0f / (2.0f * sigma * sigma);
-    constexpr int SMEM = 1024 + 2 * S1_STAGES * S1_OP_BYTES + S1_TILE * 4 + 128;
-    const unsigned grid = (unsigned)((int64_t)a.n_t * (a.n_t + 1) / 2);
-    if (bf) {
-        static bool configured = false;
-        if (!configured) {
-            e = cudaFuncSetAttribute(gram_rbf_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
-            if (e != cudaSuccess) return e;
-            configured = true;
-        }
-        gram_rbf_kernel<true><<<grid, S1_THREADS, SMEM, s>>>(tm, a);
-    } else {
-        static bool configured = false;
-        if (!configured) {
-            e = cudaFuncSetAttribute(gram_rbf_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
-            if (e != cudaSuccess) return e;
-            configured = true;
-        }
-        gram_rbf_kernel<false><<<grid, S1_THREADS, SMEM, s>>>(tm, a);
-    }
+    // CTA pairs on 256-wide tiles, or single CTAs on 128-wide tiles: whichever leaves the busiest SM less to do
+    // (work in 128 x 128 tiles; the pair kernel gets about 1.25 times as much out of the tensor pipe)
+    const int64_t n_t1 = (K + S1_TILE - 1) / S1_TILE, n_t2 = (K + 2 * S1_TILE - 1) / (2 * S1_TILE);
+    const int64_t sms = sm_count();
+    const int64_t per_sm_pairs = 2 * ((n_t2 * (n_t2 + 1) + sms - 1) / sms);       // n_t2 (n_t2 + 1) CTAs of two tiles each
+    const int64_t per_sm_single = (n_t1 * (n_t1 + 1) / 2 + sms - 1) / sms;
+    const bool pairs = 4 * per_sm_pairs < 5 * per_sm_single;
+    a.n_t = pairs ? (int)n_t2 : (int)n_t1;
+    constexpr int SMEM = 1024 + 2 * S1_STAGES * S1_OP_BYTES + 2 * S1_TILE * 4 + 128;
+    const unsigned grid = (unsigned)((int64_t)a.n_t * (a.n_t + 1) / 2) * (pairs ? 2u : 1u);
+    auto launch = [&](auto kern) -> cudaError_t {
+        cudaError_t e2 = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
+        if (e2 != cudaSuccess) return e2;
+        kern<<<grid, S1_THREADS, SMEM, s>>>(tm, a);
+        return cudaGetLastError();
+    };
+    if (pairs) e = bf ? launch(gram_rbf_pair_kernel<true>) : launch(gram_rbf_pair_kernel<false>);
+    else e = bf ? launch(gram_rbf_kernel<true>) : launch(gram_rbf_kernel<false>);
     count_launch();
-    return cudaGetLastError();
+    return e;
 }
 
 // ---- HSIC (Eq. 2) -------------------------------------------------------------------------------

@@ -89,22 +89,25 @@ def test_rbf_gram_duplicates_and_close_points(aq):
     assert abs(got[0, 1] - 1.0) < 1e-4 and abs(got[100, 3] - 1.0) < 1e-4
 
 
-def test_rbf_gram_many_samples(aq):
-    """Several tiles each way, ragged last tile; oracle on sampled rows only."""
-    K, d, sigma = 2100, 1024, 32.0
+@pytest.mark.parametrize("K,d,dtype", ((2100, 1024, "bf16"), (3000, 520, "f16"), (4096, 256, "bf16"), (5000, 72, "f16")))
+def test_rbf_gram_many_samples(aq, K, d, dtype):
+    """Several tiles each way, ragged last tile; from about 2900 samples on the CTA-pair kernel (256-wide tiles) runs.
+    Oracle on sampled rows only."""
+    sigma = math.sqrt(d)
     A32 = np.random.default_rng(36).standard_normal((K, d)).astype(np.float32)
-    t, A64 = _half(A32, "bf16")
+    t, A64 = _half(A32, dtype)
     G = aq.aq_rbf_gram(t.cuda(), sigma)
     aq.aq_check()
     got = G.double().cpu().numpy()
+    assert np.all(np.isfinite(got))
     assert np.array_equal(got, got.T) and np.array_equal(np.diag(got), np.ones(K))
     n = np.einsum("kd,kd->k", A64, A64)
-    for i in (0, 127, 128, 1023, 2047, 2048, 2099):
+    c = 1 / (2 * sigma * sigma)
+    for i in sorted({0, 127, 128, 255, 256, 1023, 2047, 2048, K - 257, K - 129, K - 1}):
         diff = A64 - A64[i]
-        ref = np.exp(-np.einsum("kd,kd->k", diff, diff) / (2 * sigma * sigma))
-        c = 1 / (2 * sigma * sigma)
+        ref = np.exp(-np.einsum("kd,kd->k", diff, diff) * c)
         bound = ref * (3 * (d / 16 + 32) * 2.0**-23 * (n + n[i]) * c + 2.0**-21 * (-np.log(ref)) + 2.0**-21) + 1e-37
-        assert np.all(np.abs(got[i] - ref) <= bound)
+        assert np.all(np.abs(got[i] - ref) <= bound), f"row {i}"
 
 
 @pytest.mark.parametrize("K", (2, 3, 64, 257, 1000))
