@@ -255,8 +255,8 @@ __global__ void __launch_bounds__(GM_THREADS, 1) gemm_kernel(const __grid_consta
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    // everything above touched only this CTA's own resources; from here on the predecessor's results are read
-    pdl_wait();
+    // The packed weights never change, so their copies and the dequantisation start at once, under the tail of the
+    // kernel before this one; the roles that read or write activations (token tiles, epilogue) call pdl_wait() first.
     pdl_launch_dependents();
 
     // this CTA's run, in slab-accumulators (even bounds)
@@ -271,6 +271,7 @@ __global__ void __launch_bounds__(GM_THREADS, 1) gemm_kernel(const __grid_consta
         if (lane == 0) {
             uint32_t bi = 0;
             bool ok = true;
+            pdl_wait();   // x is the predecessor's output
             while (ok && gemm_next_seg(pos, run_hi, a, sg)) {
                 for (int it = 2 * sg.s0; it < 2 * sg.s1 && ok; ++it) {
                     for (int j = 0; j < sg.na; ++j) {
@@ -365,6 +366,7 @@ __global__ void __launch_bounds__(GM_THREADS, 1) gemm_kernel(const __grid_consta
             // epilogue: TMEM lane quarter (warp % 4) x this warp group's columns -> out[token][row]
             if (ok) ok = mbar_wait(bar_accum, segc & 1, abort_flag, 7);
             ++segc;
+            pdl_wait();   // outputs, residuals and tile flags belong to the stream's order (returns at once after the first time)
             if (ok) {
                 tc_fence_after();
                 const int lq = dw & 3, grp = dw >> 2;
