@@ -355,6 +355,19 @@ def run_configs(args):
     c5.update({"expert_10_steps_M50_us": t, "expert_us_per_step": t / 10, "expert_gbs": 10 * info["packed_bytes"] / t / 1e3,
                "expert_tflops": 10 * 2.0 * M * info["weights"] / t / 1e6,
                "expert_note": "194.6 MB of packed weights per step: partly L2-resident across the 10 steps"})
+    # the same ten steps recorded once into a CUDA graph (1440 launches) and replayed: what a control loop would do
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        ten_steps()
+        side.synchronize()
+        with torch.cuda.graph(graph, stream=side):
+            ten_steps()
+    torch.cuda.synchronize()
+    tg = timed_us(graph.replay, 5)
+    c5.update({"expert_graph_10_steps_M50_us": tg, "expert_graph_us_per_step": tg / 10,
+               "expert_graph_gbs": 10 * info["packed_bytes"] / tg / 1e3, "expert_graph_tflops": 10 * 2.0 * M * info["weights"] / tg / 1e6})
     out["config5"] = c5
     aq.aq_check()
     print(json.dumps(out))

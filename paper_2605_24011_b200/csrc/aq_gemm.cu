@@ -493,7 +493,7 @@ static cudaError_t launch_one(const CUtensorMap& tm, const GemmOutMaps& tmo, con
     return e;
 }
 
-bool gemm_stores_first(const aq_handle_s* const* hs, int n, int M);
+bool gemm_stores_first(const aq_handle_s* const* hs, int n, int M, cudaStream_t s);
 
 // n (<= GM_MAX_OPS) matrices with the same K against one x: out[i] = (res[i]) + x W_i^T.
 // outs_ready: the caller has already put the residual (or zeros) into every output.
@@ -557,7 +557,7 @@ cudaError_t launch_gemm_group(const aq_handle_s* const* hs, int n, const void* x
     }
     if (outs_ready && !a.tma_out) return cudaErrorInvalidValue;   // (the caller checks gemm_outputs_can_be_preset first)
     static std::atomic<uint32_t> epoch_counter{0};
-    a.store_first = (a.tma_out && gemm_stores_first(hs, n, M)) ? 1 : 0;
+    a.store_first = (a.tma_out && gemm_stores_first(hs, n, M, s)) ? 1 : 0;
     a.epoch = epoch_counter.fetch_add(1) + 1;
     if (a.epoch == 0) a.epoch = epoch_counter.fetch_add(1) + 1;   // flags start out as zero: never use that value
     a.flag_slot = (int)(a.epoch % GM_FLAG_SLOTS);
@@ -582,7 +582,12 @@ cudaError_t launch_gemm(const aq_handle_s* h, const void* x, aq_dtype_t xdt, int
 }
 
 // True when outputs without a residual need no zeroing before launch_gemm_group (split tiles store first).
-bool gemm_stores_first(const aq_handle_s* const* hs, int n, int M) {
+bool gemm_stores_first(const aq_handle_s* const* hs, int n, int M, cudaStream_t s) {
+    // The protocol tells launches apart by a fresh epoch per launch.  A launch recorded into a CUDA graph would run
+    // again with the epoch it was recorded with, so while a stream is being captured outputs are zeroed and added to.
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(s, &cap) != cudaSuccess) { cudaGetLastError(); return false; }
+    if (cap != cudaStreamCaptureStatusNone) return false;
     long long R = 0;
     for (int i = 0; i < n; ++i) R += (hs[i]->NT + 7) / 8;
     const long long n_st = (M > GM_MAX_TN) ? (M + 2 * GM_MAX_TN - 1) / (2 * GM_MAX_TN) : 1;

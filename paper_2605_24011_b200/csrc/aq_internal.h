@@ -55,7 +55,7 @@ cudaError_t launch_gemm_group(const aq_handle_s* const* hs, int n, const void* x
                               float* const* outs, const int64_t* ldos, const float* const* ress, bool outs_ready,
                               cudaStream_t s);
 bool gemm_outputs_can_be_preset(float* const* outs, const int64_t* ldos, int n);
-bool gemm_stores_first(const aq_handle_s* const* hs, int n, int M);   // then only residuals need presetting
+bool gemm_stores_first(const aq_handle_s* const* hs, int n, int M, cudaStream_t s);   // then only residuals need presetting
 
 // Where a program's buffers and staged inputs sit in the caller's workspace (aq_stack.cu).
 struct StackPlan {

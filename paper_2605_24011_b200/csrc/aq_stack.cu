@@ -210,7 +210,7 @@ static cudaError_t run_stack(const aq_stack_t* p, const StackPlan& plan, const T
                         const int g0 = q - q % AQ_GEMM_MAX_GROUP, gn = std::min(AQ_GEMM_MAX_GROUP, n - g0);
                         const aq_handle_s* hs[AQ_GEMM_MAX_GROUP];
                         for (int r = 0; r < gn; ++r) hs[r] = p->ops[i + g0 + r].w;
-                        if (gemm_stores_first(hs, gn, M)) continue;
+                        if (gemm_stores_first(hs, gn, M, s)) continue;
                     }
                     pre.dst[pre.n] = reinterpret_cast<float4*>(outs[q]);
                     pre.src[pre.n] = has_res ? reinterpret_cast<const float4*>(buf(o.res)) : nullptr;
