@@ -684,17 +684,52 @@ bool build_decode_tables(const aq_stack_t* p, const StackPlan& plan, int M, int 
     for (int ph = 0; ph < n_ph; ++ph) {
         const int pfirst = plan.phase_first[ph];
         const int plast = (ph + 1 < n_ph) ? plan.phase_first[ph + 1] : p->n_ops;
-        for (int first = pfirst; first < plast; first += DS_MAX_PHASE_OPS) {
-            const int last = std::min(plast, first + DS_MAX_PHASE_OPS);
+        for (int first = pfirst; first < plast;) {
+            // as many of the phase's ops (at most DS_MAX_PHASE_OPS) as leave every CTA's staged slabs inside the
+            // shared-memory buffer; the rest of them form a further phase with the same input
             const aq_stack_op_t& f = p->ops[first];
-            DsPhase P;
-            memset(&P, 0, sizeof(P));
             const int64_t K = p->buf_width[f.src];
-            if (K > (int64_t)1 << 24) return false;
+            if (K > (int64_t)1 << 24 || n_cta > 32767) return false;
+            DsPhase P;
+            int count = std::min(plast - first, DS_MAX_PHASE_OPS), rot_after = rot;
+            for (; count >= 1; --count) {
+                memset(&P, 0, sizeof(P));
+                int r2 = rot;
+                int64_t off = 0;
+                bool ok = true;
+                for (int i = first; i < first + count && ok; ++i) {
+                    const aq_handle_s* h = p->ops[i].w;
+                    DsOp& d = P.ops[i - first];
+                    const int64_t nu = (int64_t)h->KP * h->NT;
+                    if (off + nu > (int64_t)1 << 26) { ok = false; break; }
+                    d.N = (int32_t)h->N; d.NT = h->NT; d.n_units = (int32_t)nu; d.bits = h->bits;
+                    d.units_q = (int32_t)(nu / n_cta);
+                    d.units_r_rot = (int32_t)(nu % n_cta) | (r2 << 16);
+                    r2 = (int)((r2 + nu % n_cta) % n_cta);
+                    off += nu;
+                }
+                for (int c = 0; c < n_cta && ok; ++c) {
+                    std::vector<int64_t> need;
+                    for (int i = 0; i < count; ++i) {
+                        const int64_t q = P.ops[i].units_q, r = P.ops[i].units_r_rot & 0xFFFF, ro = P.ops[i].units_r_rot >> 16;
+                        const int64_t sl = (c + ro) % n_cta;
+                        const int64_t u0 = q * sl + std::min(sl, r), u1 = u0 + q + (sl < r ? 1 : 0);
+                        if (u0 < u1)
+                            for (int64_t x = u0 / P.ops[i].NT; x <= (u1 - 1) / P.ops[i].NT; ++x) need.push_back(x);
+                    }
+                    std::sort(need.begin(), need.end());
+                    const int64_t slabs = std::unique(need.begin(), need.end()) - need.begin();
+                    if (slabs > DS_MAX_SLOTS || slabs * ds_slab_bytes(M) > DS_XS_BYTES) ok = false;
+                }
+                if (ok) { P.units_total = (int32_t)off; rot_after = r2; break; }
+            }
+            if (count < 1) return false;
+            const int last = first + count;
+            rot = rot_after;
             P.src = reinterpret_cast<const float*>(ws + plan.buf_off[f.src]);
             P.src2 = (f.in_op == AQ_IN_SILU_MUL) ? reinterpret_cast<const float*>(ws + plan.buf_off[f.src2]) : nullptr;
             P.stage = ws + plan.in_off[first];
-            P.K = (int32_t)K; P.in_op = f.in_op; P.op_first = first; P.op_count = last - first;
+            P.K = (int32_t)K; P.in_op = f.in_op; P.op_first = first; P.op_count = count;
             std::vector<int> deps;
             auto need = [&](int buf) {
                 const int w = writer[buf];
@@ -702,43 +737,20 @@ bool build_decode_tables(const aq_stack_t* p, const StackPlan& plan, int M, int 
             };
             need(f.src);
             if (f.in_op == AQ_IN_SILU_MUL) need(f.src2);
-            int64_t off = 0;
             for (int i = first; i < last; ++i) {
                 const aq_stack_op_t& o = p->ops[i];
-                const aq_handle_s* h = o.w;
                 DsOp& d = P.ops[i - first];
-                d.frags = h->frags;
+                d.frags = o.w->frags;
                 d.dst = reinterpret_cast<float*>(ws + plan.buf_off[o.dst]);
                 d.res = (o.out_op == AQ_OUT_ADD) ? reinterpret_cast<const float*>(ws + plan.buf_off[o.res]) : nullptr;
                 if (o.out_op == AQ_OUT_ADD) need(o.res);
-                const int64_t nu = (int64_t)h->KP * h->NT;
-                if (off + nu > (int64_t)1 << 26 || n_cta > 32767) return false;
-                d.N = (int32_t)h->N; d.NT = h->NT; d.n_units = (int32_t)nu; d.bits = h->bits;
-                d.units_q = (int32_t)(nu / n_cta);
-                d.units_r_rot = (int32_t)(nu % n_cta) | (rot << 16);
-                rot = (int)((rot + nu % n_cta) % n_cta);
-                off += nu;
             }
             if ((int)deps.size() > DS_MAX_DEPS) return false;
-            P.units_total = (int32_t)off;
             P.n_deps = (int)deps.size();
             for (size_t j = 0; j < deps.size(); ++j) P.deps[j] = (int16_t)deps[j];
-            // every CTA's staged slabs must fit the shared-memory buffer
-            for (int c = 0; c < n_cta; ++c) {
-                std::vector<int64_t> need;
-                for (int i = 0; i < P.op_count; ++i) {
-                    const int64_t q = P.ops[i].units_q, r = P.ops[i].units_r_rot & 0xFFFF, ro = P.ops[i].units_r_rot >> 16;
-                    const int64_t sl = (c + ro) % n_cta;
-                    const int64_t u0 = q * sl + std::min(sl, r), u1 = u0 + q + (sl < r ? 1 : 0);
-                    if (u0 < u1)
-                        for (int64_t x = u0 / P.ops[i].NT; x <= (u1 - 1) / P.ops[i].NT; ++x) need.push_back(x);
-                }
-                std::sort(need.begin(), need.end());
-                const int64_t slabs = std::unique(need.begin(), need.end()) - need.begin();
-                if (slabs > DS_MAX_SLOTS || slabs * ds_slab_bytes(M) > DS_XS_BYTES) return false;
-            }
             for (int i = first; i < last; ++i) writer[p->ops[i].dst] = i;
             phases.push_back(P);
+            first = last;
         }
     }
     return true;

@@ -61,3 +61,35 @@ def mlp_program(gate, up, down, hidden, inter):
         {"w": down, "src": 1, "src2": 2, "dst": 3, "in_op": aq.AQ_IN_SILU_MUL},
     ]
     return aq.Program(widths, ops), 3, [(0, "gate"), (0, "up"), (0, "down")]
+
+
+def independent_program(layers):
+    """The same matrices without the chain: every linear whose K equals the input width reads the program input as it
+    is; the others read the first block's outputs of that width (o: q; down: silu(gate) * up).  Nothing is normalised
+    or added and every output goes to a buffer of its own, so after the first block nothing waits for anything: the
+    streaming upper bound of the chained program.  Ops that share an input and sit together form one phase; the order
+    keeps phases at three matrices: gate up q | down | k v o in the first block, q k v | down | o gate up after it.
+    Returns (Program, out_buf, op_names)."""
+    hidden = layers[0]["shape"]["q"][1]
+    widths = [hidden]
+    ops, names = [], []
+    first = {}   # name -> output buffer of that matrix in the first block
+
+    def new_buf(w):
+        widths.append(w)
+        return len(widths) - 1
+
+    for li, L in enumerate(layers):
+        sh = L["shape"]
+        order = ("gate", "up", "q", "down", "k", "v", "o") if li == 0 else ("q", "k", "v", "down", "o", "gate", "up")
+        for nm in order:
+            N, K = sh[nm]
+            op = {"w": L[nm], "dst": new_buf(N), "in_op": aq.AQ_IN_PLAIN, "src": 0}
+            if nm == "down":
+                op.update({"src": first["gate"], "src2": first["up"], "in_op": aq.AQ_IN_SILU_MUL})
+            elif K != hidden:
+                op["src"] = first["q"]
+            ops.append(op)
+            names.append((li, nm))
+            first.setdefault(nm, op["dst"])
+    return aq.Program(widths, ops), ops[-1]["dst"], names

@@ -64,6 +64,7 @@ def llama7b_decode_stack(n_layers=32, seed=0, sample_rows=0):
     layers, samples, info = build_stack(shapes, n_layers, bits, (3, seed), outliers=True, sample_rows=sample_rows)
     prog, out_buf, names = programs.block_program(layers)
     info["bits"] = bits
+    info["layers"] = layers   # the packed matrices, for other wirings of the same stack (programs.independent_program)
     return prog, out_buf, names, samples, info
 
 

@@ -57,6 +57,29 @@ def test_tiny_block_stack(aq, M, dtype):
     assert float(out.float().abs().max()) > 0 and bool(torch.isfinite(out.float()).all())
 
 
+@pytest.mark.parametrize("M,dtype", [(1, "f16"), (8, "f16"), (40, "bf16")])
+@pytest.mark.parametrize("shapes", ("tiny", "expert_like"))
+def test_independent_inputs_program(aq, M, dtype, shapes):
+    """The second reading of a "linear stack": no chain, every linear reads the program input (or the first block's
+    q / silu(gate) * up where its K differs); per-op parity as for the chained program."""
+    from paper_2605_24011_b200 import programs
+    tdt = torch.float16 if dtype == "f16" else torch.bfloat16
+    layer = synth.tiny_layer(256, 416) if shapes == "tiny" else [("q", 512, 256), ("k", 64, 256), ("v", 64, 256), ("o", 256, 512),
+                                                                 ("gate", 416, 256), ("up", 416, 256), ("down", 256, 416)]
+    n_layers = 3
+    sizes = [N * K for _ in range(n_layers) for (_, N, K) in layer]
+    bits = synth.draw_bits(sizes, 3.0, 7)
+    layers, quant = _build_layers(aq, layer, n_layers, bits, 33)
+    prog, out_buf, names = programs.independent_program(layers)
+    assert sorted(names) == sorted((l, nm) for l in range(n_layers) for (nm, _, _) in layer)
+    ws = torch.empty(prog.workspace_bytes(M), dtype=torch.uint8, device="cuda")
+    x0 = torch.from_numpy(synth.activations(M, 256, 33, M)).to(tdt).cuda()
+    out = torch.empty((M, prog.buf_width[out_buf]), dtype=tdt, device="cuda")
+    aq.aq_stack_forward(prog, x0, out, out_buf, M, ws)
+    aq.aq_check()
+    check_program(prog, names, ws, M, tdt, quant)
+
+
 @pytest.mark.parametrize("M", (1, 8))
 def test_config2_llama_mlp_3bit(aq, M):
     """gate/up 4096 -> 11008, down 11008 -> 4096, 3-bit, x fp16 N(0,1), SiLU(gate)*up in fp32."""
