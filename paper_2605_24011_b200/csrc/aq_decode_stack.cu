@@ -276,10 +276,6 @@ struct DsShared {
     int abort_flag;
 };
 
-// Where the 16-byte chunk (block bk, quarter t) of a one-token slab lives: in the
-// row of the lane (bk, t) that multiplies it, at a position rotated by the lane
-// so that the eight chunks a lane reads never collide on a bank.
-__device__ __forceinline__ int ds_spread_offset(int lane, int bk) { return lane * 128 + ((bk ^ (lane & 7)) * 16); }
 
 // Writes 4 rounded elements (k .. k+3 of slab-local index) of the staged vector.
 template <int MT>
@@ -295,12 +291,7 @@ __device__ __forceinline__ void ds_store4(uint8_t* slab, int M, int m, int kl, u
 // The x operand of one pair-slab from its staged copy in shared memory.
 template <int MT, bool BF16>
 __device__ __forceinline__ void ds_load_x_operand(XOperand<MT>& xo, const uint8_t* slab, int M, int lane) {
-    if constexpr (MT == 1) {
-#pragma unroll
-        for (int bk = 0; bk < 8; ++bk) {
-            const uint4 v = *reinterpret_cast<const uint4*>(slab + ds_spread_offset(lane, bk));
-            xo.b[bk][0] = v.x; xo.b[bk][1] = v.y; xo.b[bk][2] = v.z; xo.b[bk][3] = v.w;
-        }
+    if constexpr (MT == 1) {   // (the B registers are read from the slab where they are used)
         const float2 xs = *reinterpret_cast<const float2*>(slab + 4096 + (lane & 3) * 8);
         xo.X0[0] = xs.x; xo.X1[0] = xs.y;
     } else {
@@ -599,28 +590,33 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArg
                 float* dst = op.dst;
                 const float* res = op.res;
                 const int N = op.N;
+                // the unit loop, one copy per code width (the width is the op's, not the unit's)
+                auto run_units = [&](auto bits_tag) {
+                    constexpr int BITS = decltype(bits_tag)::value;
 #pragma unroll 1
-                for (int u = u0; u < u1; ++u) {
-                    dead = __any_sync(0xffffffffu, !ds_mbar_wait(ds_smem(&sh.full[warp][cslot]), cparity));
-                    if (dead) {
-                        if (lane == 0) { atomicCAS(&g_decode_status, 0, 2); sh.abort_flag = 1; }
-                        break;
+                    for (int u = u0; u < u1; ++u) {
+                        dead = __any_sync(0xffffffffu, !ds_mbar_wait(ds_smem(&sh.full[warp][cslot]), cparity));
+                        if (dead) {
+                            if (lane == 0) { atomicCAS(&g_decode_status, 0, 2); sh.abort_flag = 1; }
+                            break;
+                        }
+                        const uint8_t* unit = &sh.ring[warp][cslot][0];
+                        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+                        unit_mac<BITS, MT, BF16, MT == 1>(unit, xo, lane, acc, xseg);
+                        __syncwarp();        // every lane has read its part of the slot
+                        if (lane == 0) ds_mbar_arrive(ds_smem(&sh.empty[warp][cslot]));
+                        if (++cslot == DS_SLOTS) { cslot = 0; cparity ^= 1u; }
+                        unit_commit<MT>(acc, dst, N, R * 16, N, M, lane, Pk == 0 ? res : nullptr);
+                        if (++R == NT) {
+                            R = 0; ++Pk;
+                            xseg += slab_bytes;
+                            if (u + 1 < u1) ds_load_x_operand<MT, BF16>(xo, xseg, M, lane);
+                        }
                     }
-                    const uint8_t* unit = &sh.ring[warp][cslot][0];
-                    float acc[4] = {0.f, 0.f, 0.f, 0.f};
-                    if (bits == 2) unit_mac<2, MT, BF16>(unit, xo, lane, acc);
-                    else if (bits == 3) unit_mac<3, MT, BF16>(unit, xo, lane, acc);
-                    else unit_mac<4, MT, BF16>(unit, xo, lane, acc);
-                    __syncwarp();        // every lane has read its part of the slot
-                    if (lane == 0) ds_mbar_arrive(ds_smem(&sh.empty[warp][cslot]));
-                    if (++cslot == DS_SLOTS) { cslot = 0; cparity ^= 1u; }
-                    unit_commit<MT>(acc, dst, N, R * 16, N, M, lane, Pk == 0 ? res : nullptr);
-                    if (++R == NT) {
-                        R = 0; ++Pk;
-                        xseg += slab_bytes;
-                        if (u + 1 < u1) ds_load_x_operand<MT, BF16>(xo, xseg, M, lane);
-                    }
-                }
+                };
+                if (bits == 2) run_units(std::integral_constant<int, 2>{});
+                else if (bits == 3) run_units(std::integral_constant<int, 3>{});
+                else run_units(std::integral_constant<int, 4>{});
             }
             // arrive: the CTA's last warp to finish the op publishes it
             // (the warps' commits are ordered before the release below through the acq_rel counter in shared memory)

@@ -53,6 +53,11 @@ __device__ __forceinline__ float sum8(const uint4& v) {
     return s;
 }
 
+// Where the 16-byte chunk (block bk, quarter t) of a one-token slab staged in shared memory lives: in the
+// row of the lane (bk, t) that multiplies it, at a position rotated by the lane
+// so that the eight chunks a lane reads never collide on a bank.
+__device__ __forceinline__ int ds_spread_offset(int lane, int bk) { return lane * 128 + ((bk ^ (lane & 7)) * 16); }
+
 // Per-warp state for the x operand of one pair-slab (256 k = the 8 blocks of a unit).
 // Lane (g, t) stands for B column g = (block slot g / MT, token g % MT).
 template <int MT>
@@ -134,8 +139,13 @@ __device__ __forceinline__ constexpr bool class_used_before(int c, int b0, int b
 //   MT >= 2: [row g, col 2t], [row g, col 2t+1], [row g+8, col 2t], [row g+8, col 2t+1]
 //            (columns are (block slot, token) pairs, both columns in one slot)
 //   MT == 1: the same four, where columns 2t, 2t+1 are two different blocks.
-template <int BITS, int MT, bool BF16>
-__device__ __forceinline__ void unit_mac(const uint8_t* unit, const XOperand<MT>& xo, int lane, float (&acc)[4]) {
+//
+// With xslab (one token only) the B registers are not taken from xo.b but read, block by block, from the spread-out
+// copy of the slab in shared memory: 32 registers fewer per thread for one 16-byte shared load per block.
+template <int BITS, int MT, bool BF16, bool XS = false>
+__device__ __forceinline__ void unit_mac(const uint8_t* unit, const XOperand<MT>& xo, int lane, float (&acc)[4],
+                                         const uint8_t* xslab = nullptr) {
+    static_assert(!XS || MT == 1, "the shared-memory x operand is the one-token layout");
     using IP = InPlace<BITS>;
     constexpr int FB = frag_bytes(BITS);
     constexpr int BG = XOperand<MT>::BG;
@@ -152,6 +162,13 @@ __device__ __forceinline__ void unit_mac(const uint8_t* unit, const XOperand<MT>
             load_lane_codes<BITS>(lc, unit + fi * FB, lane);
             if constexpr (!BF16) ip.prepare(lc);
         }
+        uint32_t xb[4];
+        if constexpr (XS) {
+            const uint4 v = *reinterpret_cast<const uint4*>(xslab + ds_spread_offset(lane, b));
+            xb[0] = v.x; xb[1] = v.y; xb[2] = v.z; xb[3] = v.w;
+        } else {
+            xb[0] = xo.b[b][0]; xb[1] = xo.b[b][1]; xb[2] = xo.b[b][2]; xb[3] = xo.b[b][3];
+        }
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
             const int f = 2 * j + h;
@@ -164,7 +181,7 @@ __device__ __forceinline__ void unit_mac(const uint8_t* unit, const XOperand<MT>
             // the first instruction of a group that touches an accumulator set starts it from zero
             const int k = BF16 ? 0 : IP::cls(f);
             const bool first = BF16 ? (b % BG == 0 && h == 0) : !class_used_before<BITS>(k, b - b % BG, b, h);
-            mma16816<BF16>(cs[k], a, xo.b[b][2 * h], xo.b[b][2 * h + 1], first);
+            mma16816<BF16>(cs[k], a, xb[2 * h], xb[2 * h + 1], first);
         }
         if (b % BG == BG - 1) {
             // group of blocks [b - BG + 1, b] done: take the powers of two out, apply scale and min
