@@ -49,16 +49,16 @@ constexpr int DS_THREADS = DS_CTHREADS + 32;   // + the copy warp
 constexpr int DS_SLOTS = 5;                 // ring depth per warp (units)
 constexpr int DS_SLOT_BYTES = 2560;         // the largest unit (4-bit: 2 fragments of 1280 B)
 constexpr int DS_MAX_SLOTS = 6;             // staged slabs per phase per CTA (one token; fewer with more tokens)
-constexpr int DS_XS_BYTES = DS_MAX_SLOTS * 4128;   // staged input (see ds_slab_bytes)
+constexpr int DS_XS_BYTES = DS_MAX_SLOTS * 4224;   // staged input (see ds_slab_bytes)
 constexpr int DS_MAX_PHASE_OPS = 8;
 constexpr int DS_MAX_DEPS = 12;
 constexpr int DS_RMS_HOLD = 4;              // float4 per thread kept in registers by the one-token RMS path
 constexpr uint64_t DS_WAIT_NS = 2000000000ull;   // every wait gives up after two seconds
 
 // Shared-memory bytes of one staged slab (256 k): one token is stored spread out
-// as B operands (32 lanes x 8 blocks x 16 B) plus 8 block sums; several tokens
-// are stored plainly, [token][256] halves.
-__host__ __device__ constexpr int ds_slab_bytes(int M) { return M == 1 ? 4096 + 32 : M * 512; }
+// as B operands (32 lanes x 8 blocks x 16 B) plus 8 block sums, padded to a multiple of 128 bytes (the readers form
+// addresses with an XOR); several tokens are stored plainly, [token][256] halves.
+__host__ __device__ constexpr int ds_slab_bytes(int M) { return M == 1 ? 4096 + 128 : M * 512; }
 
 __device__ int g_decode_status = 0;   // nonzero: a bounded wait ran out (1 = counter, 2 = copy)
 
@@ -587,6 +587,7 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArg
                 int Pk = u0 / NT, R = u0 - Pk * NT;
                 const uint8_t* xseg = sh.xs + (size_t)(sh.seg_slot_lo[pb][oi] + Pk - sh.seg_slab_lo[pb][oi]) * slab_bytes;
                 ds_load_x_operand<MT, BF16>(xo, xseg, M, lane);
+                uint32_t xlane = ds_spread_lane_base(xseg, lane);
                 float* dst = op.dst;
                 const float* res = op.res;
                 const int N = op.N;
@@ -602,7 +603,7 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArg
                         }
                         const uint8_t* unit = &sh.ring[warp][cslot][0];
                         float acc[4] = {0.f, 0.f, 0.f, 0.f};
-                        unit_mac<BITS, MT, BF16, MT == 1>(unit, xo, lane, acc, xseg);
+                        unit_mac<BITS, MT, BF16, MT == 1>(unit, xo, lane, acc, xlane);
                         __syncwarp();        // every lane has read its part of the slot
                         if (lane == 0) ds_mbar_arrive(ds_smem(&sh.empty[warp][cslot]));
                         if (++cslot == DS_SLOTS) { cslot = 0; cparity ^= 1u; }
@@ -610,6 +611,7 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArg
                         if (++R == NT) {
                             R = 0; ++Pk;
                             xseg += slab_bytes;
+                            xlane += (uint32_t)slab_bytes;
                             if (u + 1 < u1) ds_load_x_operand<MT, BF16>(xo, xseg, M, lane);
                         }
                     }

@@ -57,6 +57,11 @@ __device__ __forceinline__ float sum8(const uint4& v) {
 // row of the lane (bk, t) that multiplies it, at a position rotated by the lane
 // so that the eight chunks a lane reads never collide on a bank.
 __device__ __forceinline__ int ds_spread_offset(int lane, int bk) { return lane * 128 + ((bk ^ (lane & 7)) * 16); }
+// The same place as a shared-memory address: with the slab 128-byte aligned, chunk bk of a lane is at
+// (slab + lane * 128 + (lane & 7) * 16) ^ (bk * 16), one XOR with a constant per block.
+__device__ __forceinline__ uint32_t ds_spread_lane_base(const uint8_t* slab, int lane) {
+    return (uint32_t)__cvta_generic_to_shared(slab) + (uint32_t)(lane * 128 + (lane & 7) * 16);
+}
 
 // Per-warp state for the x operand of one pair-slab (256 k = the 8 blocks of a unit).
 // Lane (g, t) stands for B column g = (block slot g / MT, token g % MT).
@@ -140,11 +145,12 @@ __device__ __forceinline__ constexpr bool class_used_before(int c, int b0, int b
 //            (columns are (block slot, token) pairs, both columns in one slot)
 //   MT == 1: the same four, where columns 2t, 2t+1 are two different blocks.
 //
-// With xslab (one token only) the B registers are not taken from xo.b but read, block by block, from the spread-out
-// copy of the slab in shared memory: 32 registers fewer per thread for one 16-byte shared load per block.
+// With XS (one token only) the B registers are not taken from xo.b but read, block by block, from the spread-out
+// copy of the slab in shared memory (xlane = ds_spread_lane_base of that copy): 32 registers fewer per thread for one
+// 16-byte shared load per block.
 template <int BITS, int MT, bool BF16, bool XS = false>
 __device__ __forceinline__ void unit_mac(const uint8_t* unit, const XOperand<MT>& xo, int lane, float (&acc)[4],
-                                         const uint8_t* xslab = nullptr) {
+                                         uint32_t xlane = 0) {
     static_assert(!XS || MT == 1, "the shared-memory x operand is the one-token layout");
     using IP = InPlace<BITS>;
     constexpr int FB = frag_bytes(BITS);
@@ -164,8 +170,8 @@ __device__ __forceinline__ void unit_mac(const uint8_t* unit, const XOperand<MT>
         }
         uint32_t xb[4];
         if constexpr (XS) {
-            const uint4 v = *reinterpret_cast<const uint4*>(xslab + ds_spread_offset(lane, b));
-            xb[0] = v.x; xb[1] = v.y; xb[2] = v.z; xb[3] = v.w;
+            asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                         : "=r"(xb[0]), "=r"(xb[1]), "=r"(xb[2]), "=r"(xb[3]) : "r"(xlane ^ (uint32_t)(b * 16)));
         } else {
             xb[0] = xo.b[b][0]; xb[1] = xo.b[b][1]; xb[2] = xo.b[b][2]; xb[3] = xo.b[b][3];
         }
