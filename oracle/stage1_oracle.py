@@ -69,6 +69,17 @@ def hsic(KA: np.ndarray, KB: np.ndarray) -> float:
     return float(np.trace(KA @ C @ KB @ C) / float(K - 1) ** 2)
 
 
+def hsic_large(KA: np.ndarray, KB: np.ndarray) -> float:
+    """Eq. 2 for sample counts where the four-factor product of `hsic` is out of reach: C K_A C is formed by removing
+    row means, column means and adding back the grand mean (what multiplying by C on both sides does), then
+    tr(K_A C K_B C) = sum_ij (C K_A C)_ij [K_B]_ji.  Pinned against `hsic` on small sizes."""
+    KA = np.asarray(KA, dtype=np.float64)
+    KB = np.asarray(KB, dtype=np.float64)
+    K = KA.shape[0]
+    centred = KA - KA.mean(axis=1, keepdims=True) - KA.mean(axis=0, keepdims=True) + KA.mean()
+    return float(np.sum(centred * KB.T) / float(K - 1) ** 2)
+
+
 def sensitivity(hsic_xz: float, hsic_zy: float, alpha: float, beta: float) -> float:
     """S(W) = -alpha HSIC(X, Z) + beta HSIC(Z, Y)  [Eq. 5]."""
     return -float(alpha) * float(hsic_xz) + float(beta) * float(hsic_zy)

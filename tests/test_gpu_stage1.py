@@ -129,6 +129,36 @@ def test_hsic_given_the_same_matrices(aq, K):
     assert aq.aq_hsic(torch.from_numpy(KA).cuda(), torch.from_numpy(KB).cuda()).item() == out.item()   # reproducible
 
 
+def test_largest_sample_count(aq):
+    """K = AQ_HSIC_MAX_K samples: the kernel matrix on sampled rows, HSIC of two such matrices against the O(K^2)
+    form of the oracle (float64 on the same float32 matrices)."""
+    K, d = 16384, 64
+    g = np.random.default_rng(60)
+    A32 = g.standard_normal((K, d)).astype(np.float32)
+    B32 = (np.tanh(A32[:, :8] @ g.standard_normal((8, 16)).astype(np.float32)) + 0.3 * g.standard_normal((K, 16)).astype(np.float32))
+    (ta, A64), (tb, B64) = _half(A32, "f16"), _half(B32, "bf16")
+    GA = aq.aq_rbf_gram(ta.cuda(), 8.0)
+    GB = aq.aq_rbf_gram(tb.cuda(), 4.0)
+    out = aq.aq_hsic(GA, GB)
+    aq.aq_check()
+    for (G, X64, sigma) in ((GA, A64, 8.0), (GB, B64, 4.0)):
+        dd = X64.shape[1]
+        n = np.einsum("kd,kd->k", X64, X64)
+        c = 1 / (2 * sigma * sigma)
+        for i in (0, 255, 256, 8191, 8192, 16127, 16383):
+            got = G[i].double().cpu().numpy()
+            diff = X64 - X64[i]
+            ref = np.exp(-np.einsum("kd,kd->k", diff, diff) * c)
+            bound = ref * (3 * (dd / 16 + 32) * 2.0**-23 * (n + n[i]) * c + 2.0**-21 * (-np.log(np.maximum(ref, 1e-300))) + 2.0**-21) + 1e-37
+            assert np.all(np.abs(got - ref) <= bound), f"row {i}"
+            assert got[i] == 1.0
+    ka, kb = GA.cpu().numpy(), GB.cpu().numpy()
+    ref = S1.hsic_large(ka, kb)
+    scale = float(np.sum(ka.astype(np.float64) * kb)) / (K - 1) ** 2
+    assert abs(out.item() - ref) <= 1e-10 * scale
+    assert ref > 0
+
+
 def test_sensitivity_end_to_end(aq):
     """Eq. 5 from samples: three kernel matrices on the tensor cores, two traces, one combination."""
     K, d_in, d_out, d_act = 384, 512, 1024, 8

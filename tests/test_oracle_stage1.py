@@ -112,6 +112,17 @@ def test_hsic_self_is_centred_frobenius_norm():
     assert S1.hsic(KA, KA) == pytest.approx(np.sum(centred**2) / (K - 1) ** 2, rel=1e-12)
 
 
+def test_hsic_large_equals_the_literal_trace():
+    for K, seed in ((2, 20), (7, 21), (40, 22)):
+        g = np.random.default_rng(seed)
+        KA = S1.rbf_gram(g.standard_normal((K, 3)), 1.1)
+        KB = S1.rbf_gram(g.standard_normal((K, 2)), 0.9)
+        assert S1.hsic_large(KA, KB) == pytest.approx(S1.hsic(KA, KB), rel=1e-11, abs=1e-16)
+        # also for matrices that are not symmetric (the transpose in the trace matters)
+        A, B = g.random((K, K)), g.random((K, K))
+        assert S1.hsic_large(A, B) == pytest.approx(S1.hsic(A, B), rel=1e-10, abs=1e-14)
+
+
 def test_hsic_tells_dependence_from_independence():
     K = 200
     g = np.random.default_rng(13)
