@@ -16,7 +16,10 @@
 //     evict-first) full, running ahead across op and phase boundaries.
 //   * Dependencies.  Sums leave the warps as fp32 red.add into the output
 //     buffer.  Every op has an arrival counter in global memory; a CTA arrives
-//     once all its warps have committed their share of the op.  Before a phase
+//     once all its warps have committed their share of the op.  The arrival is
+//     a gpu-scope release, which waits for L2 to acknowledge the CTA's sums
+//     (about two microseconds under load): with one token a 17th warp does it,
+//     so that no consumer warp starts its next op late.  Before a phase
 //     a CTA waits (bounded) until the ops that wrote the buffers it reads have
 //     been arrived at by every CTA.  Ops nobody waits for soon (k and v of an
 //     attention block) therefore overlap the wait of the ops that follow.
@@ -43,9 +46,15 @@
 
 namespace aq {
 
-constexpr int DS_WARPS = 15;                // consumer warps (+ the copy warp = 4 warps per scheduler, 128 registers each)
+constexpr int DS_WARPS = 15;                // consumer warps
 constexpr int DS_CTHREADS = DS_WARPS * 32;  // consumer threads
-constexpr int DS_THREADS = DS_CTHREADS + 32;   // + the copy warp
+constexpr int DS_OPBARS = 32;               // ring of per-op arrival barriers
+// One token: a release warp besides the copy warp (17 warps put 5 on one scheduler, so the kernel must stay at 96 registers:
+// the launch bound of 640 makes the compiler do that).  More tokens need the registers: 16 warps, and the consumer warp
+// that completes an op publishes it itself.
+__host__ __device__ constexpr bool ds_release_warp(int MT) { return MT == 1; }
+__host__ __device__ constexpr int ds_threads(int MT) { return DS_CTHREADS + (ds_release_warp(MT) ? 64 : 32); }
+__host__ __device__ constexpr int ds_reg_bound(int MT) { return ds_release_warp(MT) ? 640 : 512; }
 constexpr int DS_SLOTS = 5;                 // ring depth per warp (units)
 constexpr int DS_SLOT_BYTES = 2560;         // the largest unit (4-bit: 2 fragments of 1280 B)
 constexpr int DS_MAX_SLOTS = 6;             // staged slabs per phase per CTA (one token; fewer with more tokens)
@@ -272,7 +281,9 @@ struct DsShared {
     int seg_slot_lo[2][DS_MAX_PHASE_OPS];   // ... and the slot in xs where that slab is staged (the next slabs follow)
     int slab_of_slot[2][DS_MAX_SLOTS];      // the slabs staged for this phase, ascending
     int n_slots[2];
-    int done[32];                           // warps of this CTA that finished op (index & 31)
+    alignas(8) uint64_t opbar[DS_OPBARS];   // op (index % DS_OPBARS): the consumer warps that are through with it
+    int released;                           // ops whose arrival the release warp has published
+    int done[32];                           // (no release warp) warps of this CTA that finished op (index & 31)
     int abort_flag;
 };
 
@@ -306,16 +317,18 @@ __device__ __forceinline__ void ds_load_x_operand(XOperand<MT>& xo, const uint8_
 
 // ---- the kernel ---------------------------------------------------------------------
 template <int MT, bool BF16>
-__global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArgs a) {
+__global__ void __launch_bounds__(ds_reg_bound(MT), 1) decode_stack_kernel(const DsArgs a) {
+    constexpr bool RELW = ds_release_warp(MT);
     extern __shared__ __align__(128) uint8_t ds_smem_raw[];
     DsShared& sh = *reinterpret_cast<DsShared*>(ds_smem_raw);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int M = a.M;
     const int slab_bytes = ds_slab_bytes(M);
 
-    if (threadIdx.x < 32) sh.done[threadIdx.x] = 0;
+    if (threadIdx.x < DS_OPBARS) { ds_mbar_init(ds_smem(&sh.opbar[threadIdx.x]), DS_WARPS); sh.done[threadIdx.x] = 0; }
     if (threadIdx.x == 0) {
         sh.abort_flag = 0;
+        sh.released = 0;
         ds_mbar_init(ds_smem(&sh.rec_bar[0]), 1);
         ds_mbar_init(ds_smem(&sh.rec_bar[1]), 1);
     }
@@ -327,13 +340,13 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArg
         }
     }
     // one-token slabs keep zeros everywhere but in the chunks the stagers rewrite every phase
-    for (int i = threadIdx.x; i < DS_XS_BYTES / 16; i += DS_THREADS)
+    for (int i = threadIdx.x; i < DS_XS_BYTES / 16; i += (int)blockDim.x)
         reinterpret_cast<uint4*>(sh.xs)[i] = make_uint4(0, 0, 0, 0);
     // the copy stream's tables: into shared memory when they fit
     const int mini_items = a.n_phases + a.n_mini_ops;
     const bool mini_in_smem = mini_items * 16 <= DS_MINI_BYTES;
     if (mini_in_smem)
-        for (int i = threadIdx.x; i < mini_items; i += DS_THREADS)
+        for (int i = threadIdx.x; i < mini_items; i += (int)blockDim.x)
             reinterpret_cast<uint4*>(sh.mini)[i] = __ldg(reinterpret_cast<const uint4*>(a.mini_phases) + i);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     __syncthreads();
@@ -376,6 +389,30 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArg
                 const uint64_t t = ds_now_ns();
                 if (idle == 256u) t_progress = t;
                 else if (t - t_progress > 2 * DS_WAIT_NS) { atomicCAS(&g_decode_status, 0, 2); sh.abort_flag = 1; break; }
+            }
+        }
+        return;
+    }
+
+    if (RELW && warp == DS_WARPS + 1) {
+        // ================= the release warp: publishes, op by op, that this CTA's sums are in place =================
+        // The gpu-scope release waits until the CTA's additions have been acknowledged by L2 (microseconds): here it
+        // holds up nobody, whereas a consumer warp doing it would start its next op that much later.
+        if (lane == 0) {
+            for (int opx = 0; opx < a.n_mini_ops; ++opx) {
+                const uint32_t bar = ds_smem(&sh.opbar[opx % DS_OPBARS]), parity = (uint32_t)(opx / DS_OPBARS) & 1u;
+                const uint64_t t0 = ds_now_ns();
+                bool ok = ds_mbar_try(bar, parity);
+                while (!ok) {
+#pragma unroll 1
+                    for (int i = 0; i < 32 && !ok; ++i) ok = ds_mbar_try(bar, parity);
+                    if (ok) break;
+                    if (*reinterpret_cast<volatile int*>(&sh.abort_flag)) break;
+                    if (ds_now_ns() - t0 > 2 * DS_WAIT_NS) { atomicCAS(&g_decode_status, 0, 2); sh.abort_flag = 1; break; }
+                }
+                if (!ok) break;
+                asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(a.cnt + opx) : "memory");
+                *reinterpret_cast<volatile int*>(&sh.released) = opx + 1;
             }
         }
         return;
@@ -620,15 +657,34 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArg
                 else if (bits == 3) run_units(std::integral_constant<int, 3>{});
                 else run_units(std::integral_constant<int, 4>{});
             }
-            // arrive: the CTA's last warp to finish the op publishes it
-            // (the warps' commits are ordered before the release below through the acq_rel counter in shared memory)
             __syncwarp();
-            if (lane == 0) {
-                int old;
-                asm volatile("atom.acq_rel.cta.shared::cta.add.u32 %0, [%1], 1;" : "=r"(old) : "r"(ds_smem(&sh.done[opx & 31])) : "memory");
-                if (old == DS_WARPS - 1) {
-                    sh.done[opx & 31] = 0;
-                    asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(a.cnt + opx) : "memory");
+            if constexpr (RELW) {
+                // arrive: this warp is through with the op (its additions are ordered before the arrival); the release
+                // warp publishes the op once all consumer warps have arrived
+                if (lane == 0) {
+                    // the barriers are a ring: do not lap the release warp
+                    uint32_t spins = 0;
+                    uint64_t t0 = 0;
+                    while (opx - *reinterpret_cast<volatile int*>(&sh.released) >= DS_OPBARS) {
+                        if ((++spins & 255u) == 0) {
+                            if (*reinterpret_cast<volatile int*>(&sh.abort_flag)) break;
+                            const uint64_t t = ds_now_ns();
+                            if (t0 == 0) t0 = t;
+                            if (t - t0 > DS_WAIT_NS) { atomicCAS(&g_decode_status, 0, 2); sh.abort_flag = 1; break; }
+                        }
+                    }
+                    asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];" ::"r"(ds_smem(&sh.opbar[opx % DS_OPBARS])) : "memory");
+                }
+            } else {
+                // arrive: the CTA's last warp to finish the op publishes it (the warps' commits are ordered before the
+                // release below through the acq_rel counter in shared memory)
+                if (lane == 0) {
+                    int old;
+                    asm volatile("atom.acq_rel.cta.shared::cta.add.u32 %0, [%1], 1;" : "=r"(old) : "r"(ds_smem(&sh.done[opx & 31])) : "memory");
+                    if (old == DS_WARPS - 1) {
+                        sh.done[opx & 31] = 0;
+                        asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(a.cnt + opx) : "memory");
+                    }
                 }
             }
         }
@@ -762,14 +818,14 @@ static cudaError_t launch_ds(const DsArgs& a, int grid, cudaStream_t s) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DsShared));
         if (e != cudaSuccess) return e;
         int per_sm = 0;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, DS_THREADS, sizeof(DsShared));
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, ds_threads(MT), sizeof(DsShared));
         if (e != cudaSuccess) return e;
         if (per_sm < 1) return cudaErrorCooperativeLaunchTooLarge;
         configured = true;
     }
     DsArgs args = a;
     void* params[1] = {&args};
-    cudaError_t e = cudaLaunchCooperativeKernel(reinterpret_cast<void*>(kern), dim3((unsigned)grid), dim3(DS_THREADS), params,
+    cudaError_t e = cudaLaunchCooperativeKernel(reinterpret_cast<void*>(kern), dim3((unsigned)grid), dim3(ds_threads(MT)), params,
                                                 sizeof(DsShared), s);
     if (e == cudaSuccess) count_launch();
     return e;
