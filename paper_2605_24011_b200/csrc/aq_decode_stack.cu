@@ -405,7 +405,10 @@ __global__ void __launch_bounds__(ds_reg_bound(MT), 1) decode_stack_kernel(const
                 bool ok = ds_mbar_try(bar, parity);
                 while (!ok) {
 #pragma unroll 1
-                    for (int i = 0; i < 32 && !ok; ++i) ok = ds_mbar_try(bar, parity);
+                    for (int i = 0; i < 32 && !ok; ++i) {   // (sleeping between tries: this warp shares a scheduler with consumers)
+                        __nanosleep(100);
+                        ok = ds_mbar_try(bar, parity);
+                    }
                     if (ok) break;
                     if (*reinterpret_cast<volatile int*>(&sh.abort_flag)) break;
                     if (ds_now_ns() - t0 > 2 * DS_WAIT_NS) { atomicCAS(&g_decode_status, 0, 2); sh.abort_flag = 1; break; }
