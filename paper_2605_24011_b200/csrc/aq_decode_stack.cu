@@ -281,6 +281,8 @@ struct DsShared {
     int seg_slot_lo[2][DS_MAX_PHASE_OPS];   // ... and the slot in xs where that slab is staged (the next slabs follow)
     int slab_of_slot[2][DS_MAX_SLOTS];      // the slabs staged for this phase, ascending
     int n_slots[2];
+    int4 run[DS_MAX_PHASE_OPS][DS_WARPS];   // per op of the phase and consumer warp: first unit, end, its slab, its row tile
+    int run_xslot[DS_MAX_PHASE_OPS][DS_WARPS];   // ... and the slot in xs of that slab
     alignas(8) uint64_t opbar[DS_OPBARS];   // op (index % DS_OPBARS): the consumer warps that are through with it
     int released;                           // ops whose arrival the release warp has published
     int done[32];                           // (no release warp) warps of this CTA that finished op (index & 31)
@@ -493,6 +495,16 @@ __global__ void __launch_bounds__(ds_reg_bound(MT), 1) decode_stack_kernel(const
         if (*reinterpret_cast<volatile int*>(&sh.abort_flag)) break;
         // every warp is past phase ph - 1: its record slot is free for phase ph + 1
         if (threadIdx.x == 0 && ph >= 1 && ph + 1 < a.n_phases) fetch_record(ph + 1);
+        // every warp's run in every op of the phase, worked out by one thread each (the warps then switch ops with one load)
+        if ((int)threadIdx.x < P.op_count * DS_WARPS) {
+            const int oi = (int)threadIdx.x / DS_WARPS, w = (int)threadIdx.x - oi * DS_WARPS;
+            const DsOp& op = P.ops[oi];
+            int u0, u1;
+            ds_warp_run(op.units_q, op.units_r_rot, w, u0, u1);
+            const int Pk = (u0 < u1) ? u0 / op.NT : 0;
+            sh.run[oi][w] = make_int4(u0, u1, Pk, u0 - Pk * op.NT);
+            sh.run_xslot[oi][w] = sh.seg_slot_lo[pb][oi] + Pk - sh.seg_slab_lo[pb][oi];
+        }
 
         // -- form the rounded input vector: slabs this CTA reads -> shared memory, its share -> workspace --
         {
@@ -621,11 +633,11 @@ __global__ void __launch_bounds__(ds_reg_bound(MT), 1) decode_stack_kernel(const
             const int opx = P.op_first + oi;
             const DsOp& op = P.ops[oi];
             const int NT = op.NT, bits = op.bits;
-            int u0, u1;
-            ds_warp_run(op.units_q, op.units_r_rot, warp, u0, u1);
+            const int4 rn = sh.run[oi][warp];
+            const int u0 = rn.x, u1 = rn.y;
             if (u0 < u1 && !dead) {
-                int Pk = u0 / NT, R = u0 - Pk * NT;
-                const uint8_t* xseg = sh.xs + (size_t)(sh.seg_slot_lo[pb][oi] + Pk - sh.seg_slab_lo[pb][oi]) * slab_bytes;
+                int Pk = rn.z, R = rn.w;
+                const uint8_t* xseg = sh.xs + (size_t)sh.run_xslot[oi][warp] * slab_bytes;
                 ds_load_x_operand<MT, BF16>(xo, xseg, M, lane);
                 uint32_t xlane = ds_spread_lane_base(xseg, lane);
                 float* dst = op.dst;
