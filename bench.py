@@ -514,7 +514,7 @@ def main():
 
 # dram__bytes_read.sum + dram__bytes_write.sum of the decode kernel per stack pass, from the ncu
 # capture summarised under profiles/ (None until a capture has been taken).
-DECODE_TRAFFIC_BYTES = int((354.960e6 + 3.602e6) * 2833383424 / 354.17e6)
+DECODE_TRAFFIC_BYTES = int((354.938e6 + 4.175e6) * 2833383424 / 354.17e6)
 # gemm_kernel: 21.21 MB of DRAM traffic per 11008 x 4096 launch, scaled by weights to the 224 matrices of one pass
 PREFILL_TRAFFIC_BYTES = int(21.21e6 * 6476005376 / (11008 * 4096))
 
