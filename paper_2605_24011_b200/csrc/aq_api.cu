@@ -203,7 +203,8 @@ static aq_status_t linear_common(aq_handle_t h, const void* x_dev, void* y_dev, 
     cudaError_t e;
     if (M <= AQ_DECODE_MAX_M) {
         const int64_t ld = (int64_t)h->NT * 16;
-        if ((int64_t)M * h->N <= 65536) {   // small outputs: the streaming kernel's last CTA casts them (one launch)
+        if ((int64_t)M * h->N <= 8192) {   // small outputs: the streaming kernel's last CTA casts them (one launch; one CTA
+                                           // alone takes about 0.1 us per 256 outputs, so larger ones get the cast kernel)
             e = launch_gemv(h, x_dev, xdt, M, h->acc, ld, s, y_dev, ydt);
         } else {
             e = launch_gemv(h, x_dev, xdt, M, h->acc, ld, s);

@@ -104,14 +104,25 @@ __global__ void __launch_bounds__(GEMV_WARPS * 32, 2) gemv_kernel(const GemvArgs
     if (!is_last) return;
     __threadfence();
     const int64_t total = (int64_t)a.M * a.N;
-    for (int64_t i = threadIdx.x; i < total; i += blockDim.x) {
-        const int64_t m = i / a.N, n = i - m * a.N;
-        float* p = a.acc + m * a.ldacc + n;
-        const float v = __ldcg(p);
-        *p = 0.f;
-        if (a.ydt == AQ_F32) reinterpret_cast<float*>(a.y)[i] = v;
-        else if (a.ydt == AQ_F16) reinterpret_cast<__half*>(a.y)[i] = __float2half_rn(v);
-        else reinterpret_cast<__nv_bfloat16*>(a.y)[i] = __float2bfloat16_rn(v);
+    for (int64_t i0 = threadIdx.x; i0 < total; i0 += 4 * blockDim.x) {   // four loads in flight per thread
+        float v[4];
+        float* p[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int64_t i = i0 + (int64_t)j * blockDim.x;
+            const int64_t m = i / a.N, n = i - m * a.N;
+            p[j] = a.acc + m * a.ldacc + n;
+            v[j] = (i < total) ? __ldcg(p[j]) : 0.f;
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int64_t i = i0 + (int64_t)j * blockDim.x;
+            if (i >= total) break;
+            *p[j] = 0.f;
+            if (a.ydt == AQ_F32) reinterpret_cast<float*>(a.y)[i] = v[j];
+            else if (a.ydt == AQ_F16) reinterpret_cast<__half*>(a.y)[i] = __float2half_rn(v[j]);
+            else reinterpret_cast<__nv_bfloat16*>(a.y)[i] = __float2bfloat16_rn(v[j]);
+        }
     }
     if (threadIdx.x == 0) *a.ticket = 0u;
 }
