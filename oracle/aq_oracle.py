@@ -16,7 +16,7 @@ What it states (paper passages in brackets):
   [Eq. 1's argmin; the "RTN block quantization" row of the ablation table].
 * container [Appendix D]: per tensor the packed integer codes, per-block
   scales and zero points.  The byte order below (little-endian, LSB first) is
-  this build's reading; the paper does not print one.
+  this library's reading; the paper does not print one.
 * linear: y = x W_hat^T, activations in half precision [Limitations:
   weight-only quantisation], evaluated here in float64.
 
