@@ -47,22 +47,27 @@ __global__ void __launch_bounds__(128) pack_kernel(const float* __restrict__ W, 
     uint32_t my_dm[2] = {0, 0};
     bool bad = false;
 
+    // all 16 loads of the lane first (the fragment's 8 KB are in flight at once), then the arithmetic
+    float4 ld[4][2][2];
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
 #pragma unroll
         for (int hi = 0; hi < 2; ++hi) {
             const int64_t row = (int64_t)R * 16 + g + 8 * hi;
             const int64_t k0 = S * 128 + 32 * j + 8 * t;
-            const bool in = row < N && k0 < K;
-            float v[8];
-            if (in) {
-                const float4 a = *reinterpret_cast<const float4*>(W + row * K + k0);
-                const float4 b = *reinterpret_cast<const float4*>(W + row * K + k0 + 4);
-                v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
-            } else {
-#pragma unroll
-                for (int c = 0; c < 8; ++c) v[c] = 0.f;
+            ld[j][hi][0] = ld[j][hi][1] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (row < N && k0 < K) {
+                ld[j][hi][0] = __ldcs(reinterpret_cast<const float4*>(W + row * K + k0));
+                ld[j][hi][1] = __ldcs(reinterpret_cast<const float4*>(W + row * K + k0 + 4));
             }
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+#pragma unroll
+        for (int hi = 0; hi < 2; ++hi) {
+            const float4 a = ld[j][hi][0], b = ld[j][hi][1];
+            const float v[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
             float mn = v[0], mx = v[0];
 #pragma unroll
             for (int c = 0; c < 8; ++c) {
