@@ -49,10 +49,10 @@ namespace aq {
 constexpr int DS_WARPS = 15;                // consumer warps
 constexpr int DS_CTHREADS = DS_WARPS * 32;  // consumer threads
 constexpr int DS_OPBARS = 32;               // ring of per-op arrival barriers
-// One token: a release warp besides the copy warp (17 warps put 5 on one scheduler, so the kernel must stay at 96 registers:
+// One or two tokens: a release warp besides the copy warp (17 warps put 5 on one scheduler, so the kernel must stay at 96 registers:
 // the launch bound of 640 makes the compiler do that).  More tokens need the registers: 16 warps, and the consumer warp
 // that completes an op publishes it itself.
-__host__ __device__ constexpr bool ds_release_warp(int MT) { return MT == 1; }
+__host__ __device__ constexpr bool ds_release_warp(int MT) { return MT <= 2; }
 __host__ __device__ constexpr int ds_threads(int MT) { return DS_CTHREADS + (ds_release_warp(MT) ? 64 : 32); }
 __host__ __device__ constexpr int ds_reg_bound(int MT) { return ds_release_warp(MT) ? 640 : 512; }
 constexpr int DS_SLOTS = 5;                 // ring depth per warp (units)
