@@ -9,7 +9,7 @@
  * N rows (output features) by K columns (input features) is cut, along each
  * row, into blocks of 32 consecutive elements; a block has a scale and a zero
  * point and all its elements are coded with the same number of bits n; one
- * matrix has one n (Section 1: "a single bit-width per matrix").  Eq. 1's
+ * matrix has one n (Section 1 / Section 4.1: one bit-width per matrix).  Eq. 1's
  * decode s_b (q_i - z_b) is stored as  scale * q_i + min  (min = -s_b z_b),
  * scale and min in IEEE binary16, q_i in {0 .. 2^n - 1}, n in {2, 3, 4}.
  *

@@ -8,8 +8,8 @@ What it states (paper passages in brackets):
 
 * block format [Section 3, "Weight quantization", Eq. 1]: every B = 32
   consecutive elements of a weight row share one scale and one zero point and
-  are coded with the same n bits; a matrix has one bit-width [Section 1,
-  "a single bit-width per matrix"].  Eq. 1 writes the decode as
+  are coded with the same n bits; every matrix has one bit-width [Section 1 and
+  Section 4.1: the inter-tensor stage assigns a width per matrix].  Eq. 1 writes the decode as
   s_b (q_i - z_b); here it is stored as  scale * q + min  with
   min = -s_b z_b, which names the same set of representable values.
 * quantiser: round to the nearest code of the uniform codebook {0..2^n-1}
@@ -307,7 +307,12 @@ def quantize_opt(W: np.ndarray, bits: int, F=None, rounds: int = 4):
     """Scale-optimised block quantiser [Eq. 10, Eq. 11], same outputs as quantize().
 
     Every step is one correctly rounded binary32 operation in a stated order (sums: _sum32),
-    except the 2 x 2 solve, done in binary64 from the binary32 sums, one rounding per operation:
+    except the 2 x 2 solve, done in binary64 from the binary32 sums, one rounding per operation.
+    The paper fixes neither the precision nor the order of the sums; both are a reading taken so
+    that two implementations can agree byte for byte.  What ties this function to the plain
+    statement (scale_opt_ideal, float64) is tests/test_oracle_scale_opt.py: same parameters in
+    all but the blocks where a near-tie parts the two runs, and a Phi_b no worse than the better
+    plain candidate.
         sigma2 = sum32(w w) / 32;  omega = F * sqrt(sigma2 + w w)            (F omitted when None)
         s = (max - min) / L, mm = min
         repeat `rounds` times, while s > 0:

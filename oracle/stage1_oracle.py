@@ -7,7 +7,7 @@ tuned for speed.  Everything is float64.
 
 What it states (paper passages in brackets):
 
-* RBF kernel matrix [Section 3, "HSIC": "We use the RBF kernel throughout"]:
+* RBF kernel matrix [Section 3, HSIC paragraph: the Gaussian (RBF) kernel is the one used]:
   k(a, a') = exp(-|a - a'|^2 / (2 sigma^2)).  The paper does not print the
   bandwidth; here sigma is an argument.
 * empirical HSIC [Eq. 2]: (K-1)^-2 tr(K_A C K_B C), C = I - 11^T / K.

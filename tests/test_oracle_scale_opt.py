@@ -104,3 +104,44 @@ def test_sum32_order():
         g.append(a)
     want = _f32(_f32(g[0] + g[1]) + _f32(g[2] + g[3]))
     assert float(O._sum32(x[None, :])[0]) == want
+
+
+def _opt_vs_plain(bits, Fm, seed):
+    """quantize_opt (binary32, fixed summation order) beside the plain float64 statement of Eq. 10-11."""
+    W = synth.weights(64, 512, seed, bits, outliers=True)
+    d, m, q = O.quantize_opt(W, bits, Fm, rounds=4)
+    d0, m0, q0 = O.quantize(W, bits)
+    s, mi, _, _ = O.scale_opt_ideal(W, bits, Fm, rounds=4)
+    dI, mI = s.astype(np.float16), mi.astype(np.float16)             # the plain result in the container's precision
+    qI, _ = O.quantize_ideal(W, dI, mI, bits)                        # ... and its nearest codes, in float64
+    return W, (d, m, q), (d0, m0, q0), (dI, mI, qI)
+
+
+@pytest.mark.parametrize("bits", (2, 3, 4))
+@pytest.mark.parametrize("fisher", (False, True))
+def test_quantize_opt_lands_on_the_plain_alternation(bits, fisher):
+    """Wherever quantize_opt leaves the round-to-nearest form, its (scale, min) are the float64 alternation's
+    (Eq. 11, `scale_opt_ideal`) rounded to binary16 -- except in the few blocks where a binary32 quotient and its
+    float64 twin fall on different sides of a rounding boundary in some round and the two runs part."""
+    Fm = (np.abs(synth.weights(64, 512, 174, bits)) * 50 + 0.01).astype(np.float32) if fisher else None
+    W, (d, m, q), (d0, m0, q0), (dI, mI, qI) = _opt_vs_plain(bits, Fm, 173)
+    switched = (d != d0) | (m != m0)
+    assert switched.mean() > 0.9                                     # on such data nearly every block gains
+    same = (d == dI) & (m == mI)
+    assert same[switched].mean() >= 0.99
+    # blocks that took the plain parameters also took the plain codes, except at exact near-ties of the quotient
+    blk = np.repeat(switched & same, 32, axis=1)
+    assert (q[blk] != qI[blk]).mean() < 1e-3
+
+
+@pytest.mark.parametrize("bits", (2, 3, 4))
+@pytest.mark.parametrize("fisher", (False, True))
+def test_quantize_opt_is_as_good_as_the_better_plain_candidate(bits, fisher):
+    """Per block, Phi_b (Eq. 10, float64) of quantize_opt's output is no worse than the better of round-to-nearest
+    and the float64 alternation rounded to binary16 (which is what its final selection claims to pick)."""
+    Fm = (np.abs(synth.weights(64, 512, 176, bits)) * 50 + 0.01).astype(np.float32) if fisher else None
+    W, (d, m, q), (d0, m0, q0), (dI, mI, qI) = _opt_vs_plain(bits, Fm, 175)
+    phi = O.block_phi(W, d, m, q, Fm)
+    best = np.minimum(O.block_phi(W, d0, m0, q0, Fm), O.block_phi(W, dI, mI, qI, Fm))
+    assert np.all(phi <= best * (1 + 1e-3) + 1e-30)
+    assert abs(phi.sum() / best.sum() - 1) < 1e-4
