@@ -261,7 +261,8 @@ typedef struct {
     const int64_t* buf_width;     /* HOST, n_bufs entries */
 } aq_stack_t;
 
-/* Bytes of workspace aq_stack_forward needs for M tokens (0 on a bad program). */
+/* Bytes of workspace aq_stack_forward needs for M tokens (0 on a bad program).  For M <= AQ_DECODE_MAX_M this
+ * includes 8 bytes per buffer element for the decode kernel's packed sums. */
 size_t aq_stack_workspace_bytes(const aq_stack_t* prog, int M);
 
 /*
@@ -297,6 +298,23 @@ size_t aq_stack_input_offset(const aq_stack_t* prog, int M, int op);
  * (AQ_ERR_CUDA).  Outputs of a call that timed out are undefined.
  */
 aq_status_t aq_check(aq_stream_t stream);
+
+/*
+ * aq_set_wait_limit_ns -- how long a device-side wait of the whole-program decode kernel (for an input another
+ * CTA has not finished, for a weight copy) may last before the kernel gives up, raises the status that aq_check
+ * reports as AQ_ERR_TIMEOUT, and returns with the context intact.  0 restores the default (two seconds).
+ * Applies to launches made after the call.  (Section 4.3's runtime has no counterpart: this is the library's
+ * failure detection.)
+ */
+aq_status_t aq_set_wait_limit_ns(uint64_t ns);
+
+/*
+ * aq_debug_decode_hold -- TESTING ONLY.  While on, the tables aq_stack_forward builds for the decode kernel make the
+ * first phase that reads another op's output expect one contribution more than will ever arrive, so every CTA's
+ * wait for that input runs out (after the limit above) and the time-out path can be exercised on a healthy GPU:
+ * nothing traps, faults or spins without bound.  Programs run while it is off are not affected.
+ */
+void aq_debug_decode_hold(int on);
 
 /* Releases the handle and its device memory (synchronises its last stream). */
 void aq_free(aq_handle_t h);

@@ -28,7 +28,7 @@ AQ_MAX_M, AQ_DECODE_MAX_M = 4096, 8
 SYMBOLS = ("aq_pack", "aq_pack_opt", "aq_import", "aq_export", "aq_info", "aq_dequant", "aq_linear", "aq_linear_f32out", "aq_linear_noalloc",
            "aq_rbf_gram", "aq_hsic", "aq_sensitivity", "aq_allocate_bits",
            "aq_stack_workspace_bytes", "aq_stack_forward", "aq_stack_buffer_offset", "aq_stack_input_offset", "aq_check", "aq_free",
-           "aq_status_string", "aq_last_cuda_error", "aq_kernel_launches")
+           "aq_set_wait_limit_ns", "aq_debug_decode_hold", "aq_status_string", "aq_last_cuda_error", "aq_kernel_launches")
 
 _H = C.c_void_p
 
@@ -74,6 +74,10 @@ _lib.aq_stack_forward.argtypes = [C.POINTER(Stack), C.c_void_p, C.c_void_p, C.c_
                                   C.c_size_t, C.c_void_p]
 _lib.aq_check.argtypes = [C.c_void_p]
 _lib.aq_check.restype = C.c_int
+_lib.aq_set_wait_limit_ns.argtypes = [C.c_uint64]
+_lib.aq_set_wait_limit_ns.restype = C.c_int
+_lib.aq_debug_decode_hold.argtypes = [C.c_int]
+_lib.aq_debug_decode_hold.restype = None
 _lib.aq_free.argtypes = [_H]
 _lib.aq_free.restype = None
 _lib.aq_status_string.argtypes = [C.c_int]
@@ -342,6 +346,17 @@ def stack_input(prog: Program, workspace, M: int, op: int, dtype):
     off = prog.input_offset(M, op)
     K = prog.buf_width[prog.ops[op]["src"]]
     return workspace[off:off + 2 * M * K].view(dtype).view(M, K)
+
+
+def aq_set_wait_limit_ns(ns: int) -> int:
+    """Limit of every device-side wait of the decode-stack kernel (0: the default)."""
+    _check(_lib.aq_set_wait_limit_ns(int(ns)), "aq_set_wait_limit_ns")
+    return AQ_OK
+
+
+def aq_debug_decode_hold(on: bool) -> None:
+    """Testing only: decode tables built while on wait for a contribution that never comes."""
+    _lib.aq_debug_decode_hold(1 if on else 0)
 
 
 def aq_kernel_launches() -> int:

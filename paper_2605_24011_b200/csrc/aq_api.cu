@@ -23,14 +23,22 @@ bool handle_ok(aq_handle_t h) { return h != nullptr && h->magic == AQ_HANDLE_MAG
 static std::atomic<uint64_t> g_launches{0};
 void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
 
+int current_device() {
+    int dev = 0;
+    return cudaGetDevice(&dev) == cudaSuccess ? dev : -1;
+}
+
+// SM count of the current device (cached per device).
 int sm_count() {
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
-    }
-    return n;
+    static PerDeviceValue<int> cache;
+    int n = 0;
+    const int rc = cache.get(current_device(), &n, [](int dev, int* out) {
+        int v = 0;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) { cudaGetLastError(); v = 148; }
+        *out = v;
+        return 0;
+    });
+    return rc == 0 ? n : 148;
 }
 
 static aq_status_t check_arch(int* dev_out) {
@@ -283,6 +291,13 @@ aq_status_t aq_check(aq_stream_t stream) {
     const int g = read_gemm_status(true), d = read_decode_status(true), t = read_stage1_status(true);
     return (g || d || t) ? AQ_ERR_TIMEOUT : AQ_OK;
 }
+
+aq_status_t aq_set_wait_limit_ns(uint64_t ns) {
+    set_decode_wait_ns(ns);
+    return AQ_OK;
+}
+
+void aq_debug_decode_hold(int on) { set_decode_hold(on != 0); }
 
 void aq_free(aq_handle_t h) {
     if (!handle_ok(h)) return;

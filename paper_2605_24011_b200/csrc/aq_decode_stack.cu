@@ -7,29 +7,31 @@
 // launch, so the pass runs as one cooperative grid of one CTA per SM:
 //
 //   * Work.  Consecutive ops that read the same input vector form a phase.
-//     The units (16 rows x 256 k) of a phase's matrices are concatenated and
-//     dealt as contiguous runs: first to CTAs, then to the 15 consumer warps
-//     of a CTA.
+//     Every op's units (16 rows x 256 k) are dealt as contiguous runs to the
+//     CTAs; inside a CTA the runs of a phase are concatenated into one list
+//     and consumer warp w takes positions w, w + 15, w + 30 ... of it, so all
+//     warps of a CTA reach the end of a phase within one unit of each other
+//     and a warp never "switches ops": every unit comes with a descriptor.
 //   * Weight stream.  Which bytes a warp will need does not depend on any
 //     activation, so a 16th warp (lane w serves consumer warp w) keeps every
 //     consumer's private ring of bulk copies (cp.async.bulk + mbarrier, L2
-//     evict-first) full, running ahead across op and phase boundaries.
-//   * Dependencies.  Sums leave the warps as fp32 red.add into the output
-//     buffer.  Every op has an arrival counter in global memory; a CTA arrives
-//     once all its warps have committed their share of the op.  The arrival is
-//     a gpu-scope release, which waits for L2 to acknowledge the CTA's sums
-//     (about two microseconds under load): with one token a 17th warp does it,
-//     so that no consumer warp starts its next op late.  Before a phase
-//     a CTA waits (bounded) until the ops that wrote the buffers it reads have
-//     been arrived at by every CTA.  Ops nobody waits for soon (k and v of an
-//     attention block) therefore overlap the wait of the ops that follow.
+//     evict-first) full, running ahead across op and phase boundaries, and
+//     writes each unit's descriptor (op, unit index) beside it.
+//   * Sums and dependencies.  A unit's 16 row sums leave the warp as ONE
+//     64-bit red.add each: the sum in 2^-24 fixed point in the upper 52 bits
+//     plus 1 in the lower 12 bits.  A row is complete when its count equals the
+//     number of k-slabs of the matrix, so whoever needs a value polls the value
+//     itself: no arrival counters, no fences, no release, and the result does
+//     not depend on the order of the additions.  A CTA starts a phase as soon
+//     as the elements IT reads are complete, not when the whole op is.
 //   * Glue.  At the start of a phase each CTA forms, in shared memory, the
 //     rounded input vector for the k-slabs its warps will touch (RMS scaling /
 //     SiLU(g)*u / plain) with one round trip to L2, and writes its share of the
-//     vector to the caller's workspace, where every op's input stays readable.
-//     For one token the vector is stored already spread out as the B operand of
-//     the tensor-core instruction (non-zero only in the column of its block),
-//     so a warp picks its operand up with eight 16-byte loads.
+//     float32 buffer and of the rounded vector to the caller's workspace,
+//     where every op's input and output stay readable.  For one token the
+//     vector is stored already spread out as the B operand of the tensor-core
+//     instruction (non-zero only in the column of its block), so a warp picks
+//     its operand up with eight 16-byte loads.
 //
 // Every wait is bounded: when one runs out the kernel raises a status word,
 // gives copies in flight time to land and returns.
@@ -46,55 +48,62 @@
 
 namespace aq {
 
+typedef unsigned long long u64;
+
 constexpr int DS_WARPS = 15;                // consumer warps
 constexpr int DS_CTHREADS = DS_WARPS * 32;  // consumer threads
-constexpr int DS_OPBARS = 32;               // ring of per-op arrival barriers
-// One or two tokens: a release warp besides the copy warp (17 warps put 5 on one scheduler, so the kernel must stay at 96 registers:
-// the launch bound of 640 makes the compiler do that).  More tokens need the registers: 16 warps, and the consumer warp
-// that completes an op publishes it itself.
-__host__ __device__ constexpr bool ds_release_warp(int MT) { return MT <= 2; }
-__host__ __device__ constexpr int ds_threads(int MT) { return DS_CTHREADS + (ds_release_warp(MT) ? 64 : 32); }
-__host__ __device__ constexpr int ds_reg_bound(int MT) { return ds_release_warp(MT) ? 640 : 512; }
+constexpr int DS_THREADS = DS_CTHREADS + 32;   // + the copy warp
 constexpr int DS_SLOTS = 5;                 // ring depth per warp (units)
 constexpr int DS_SLOT_BYTES = 2560;         // the largest unit (4-bit: 2 fragments of 1280 B)
 constexpr int DS_MAX_SLOTS = 6;             // staged slabs per phase per CTA (one token; fewer with more tokens)
 constexpr int DS_XS_BYTES = DS_MAX_SLOTS * 4224;   // staged input (see ds_slab_bytes)
 constexpr int DS_MAX_PHASE_OPS = 8;
-constexpr int DS_MAX_DEPS = 12;
-constexpr int DS_RMS_HOLD = 4;              // float4 per thread kept in registers by the one-token RMS path
-constexpr uint64_t DS_WAIT_NS = 2000000000ull;   // every wait gives up after two seconds
+constexpr int DS_RMS_HOLD = 4;              // groups of four elements per thread kept in registers by the one-token RMS path
+constexpr u64 DS_WAIT_NS_DEFAULT = 2000000000ull;   // every wait gives up after two seconds
+
+// A packed sum: bits [12, 64) hold the value in units of 2^-24 (two's complement), bits [0, 12) the number of
+// contributions added so far.
+constexpr int DS_CNT_BITS = 12;
+constexpr u64 DS_CNT_MASK = (1ull << DS_CNT_BITS) - 1;
+constexpr int DS_MAX_CONTRIB = (1 << DS_CNT_BITS) - 1;
+constexpr float DS_FIX_ONE = 16777216.f;            // 2^24
+constexpr float DS_FIX_MAX = 134217600.f;           // just below 2^27: what the 52-bit field holds with room to add
+constexpr int DS_RES_PLAIN = 0x100;
 
 // Shared-memory bytes of one staged slab (256 k): one token is stored spread out
 // as B operands (32 lanes x 8 blocks x 16 B) plus 8 block sums, padded to a multiple of 128 bytes (the readers form
 // addresses with an XOR); several tokens are stored plainly, [token][256] halves.
 __host__ __device__ constexpr int ds_slab_bytes(int M) { return M == 1 ? 4096 + 128 : M * 512; }
 
-__device__ int g_decode_status = 0;   // nonzero: a bounded wait ran out (1 = counter, 2 = copy)
+__device__ int g_decode_status = 0;   // nonzero: a bounded wait ran out (1 = an input never completed, 2 = a copy)
 
 struct DsOp {
     const uint8_t* frags;
-    float* dst;            // float32 [M][N]
-    const float* res;      // float32 [M][N] added once (by the k-slab-0 units), or null
+    u64* dst;              // packed sums [M][N]
+    const void* res;       // [M][N] added once (by the k-slab-0 units), or null: packed sums that are complete before the
+                           // phase starts, or plain float32 when bit 8 of `bits` is set (the program input)
     int32_t N;             // true rows
     int32_t NT;            // 16-row tiles
-    int32_t n_units;       // KP * NT = units_q * (number of CTAs) + units_r
-    int32_t bits;
-    int32_t units_q;
+    uint32_t nt_magic;     // floor(2^32 / NT) + 1: u / NT = umulhi(u, magic) or one more (u < 2^26); 0 when NT = 1
+    int32_t bits;          // code width | DS_RES_PLAIN
+    int32_t units_q;       // KP * NT = units_q * (number of CTAs) + units_r
     int32_t units_r_rot;   // units_r | rot << 16: CTA c takes the run of slot (c + rot) mod (number of CTAs)
 };
 
 struct DsPhase {
-    const float* src;      // float32 [M][K]
-    const float* src2;     // second input of AQ_IN_SILU_MUL, else null
+    const u64* src;        // packed [M][K], or null when the source is plain float32
+    const u64* src2;       // second input of AQ_IN_SILU_MUL (packed), else null
+    const float* src_f;    // plain float32 [M][K] source (the program input), used when src is null
+    const float* src2_f;
+    float* rec;            // float32 [M][K]: the caller's copy of src, written share by share (null: nothing to write)
+    float* rec2;
     void* stage;           // [M][K] of the activation dtype: the rounded input, kept for the caller
     int32_t K;
     int32_t in_op;
-    int32_t op_first;      // index of ops[0] in the program (names its arrival counter)
     int32_t op_count;
-    int32_t units_total;
-    int32_t n_deps;
-    int16_t deps[DS_MAX_DEPS];   // ops that must be complete before this phase reads its inputs
-    int32_t pad_[2];
+    uint32_t expect;       // contributions that complete an element of src
+    uint32_t expect2;
+    int32_t pad_[1];
     DsOp ops[DS_MAX_PHASE_OPS];
 };
 static_assert(sizeof(DsOp) == 48, "DsOp layout");
@@ -115,13 +124,26 @@ struct DsMiniPhase {
 static_assert(sizeof(DsMiniOp) == 16 && sizeof(DsMiniPhase) == 16, "mini tables are copied as 16-byte items");
 constexpr int DS_MINI_BYTES = 8192;
 
+// A stretch of a buffer no phase reads: converted to float32 for the caller once the last phase is done.
+struct DsTail {
+    const u64* src;
+    float* out;
+    int32_t n;
+    uint32_t expect;
+    int32_t pad_[2];
+};
+static_assert(sizeof(DsTail) == 32, "DsTail layout");
+constexpr int DS_TAIL_CHUNK = 2048;
+
 struct DsArgs {
     const DsPhase* phases;
     const DsMiniPhase* mini_phases;   // n_phases entries, followed by
     const DsMiniOp* mini_ops;         // n_mini_ops entries (contiguous: one copy brings both)
-    uint32_t* cnt;         // per-op arrival counters, zero at launch
+    const DsTail* tails;
+    u64 wait_ns;
     int n_phases;
     int n_mini_ops;
+    int n_tails;
     int M;
 };
 
@@ -164,34 +186,84 @@ __device__ __forceinline__ uint64_t ds_now_ns() {
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-// Bounded wait on a shared-memory barrier; false when DS_WAIT_NS passed.
-__device__ __forceinline__ bool ds_mbar_wait(uint32_t bar, uint32_t parity) {
+// Bounded wait on a shared-memory barrier; false when wait_ns passed.
+__device__ __forceinline__ bool ds_mbar_wait(uint32_t bar, uint32_t parity, u64 wait_ns) {
     if (ds_mbar_try(bar, parity)) return true;
     const uint64_t t0 = ds_now_ns();
     for (;;) {
 #pragma unroll 1
         for (int i = 0; i < 64; ++i)
             if (ds_mbar_try(bar, parity)) return true;
-        if (ds_now_ns() - t0 > DS_WAIT_NS) return false;
+        if (ds_now_ns() - t0 > wait_ns) return false;
     }
-}
-__device__ __forceinline__ uint32_t ds_ld_acquire(const uint32_t* p) {
-    uint32_t v;
-    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-    return v;
 }
 // Barrier among the consumer warps only (the copy warp never joins).
 __device__ __forceinline__ void ds_consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(DS_CTHREADS) : "memory"); }
+// The same barrier, returning the OR of `flag` over all consumer threads: every thread gets the same answer, so a
+// decision to leave the phase loop is taken by all warps or by none (a flag read after a plain barrier could change
+// between two threads' reads).
+__device__ __forceinline__ bool ds_consumer_sync_or(int flag) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 q, %1, 0;\n\t"
+        "bar.red.or.pred p, 1, %2, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(r) : "r"(flag), "n"(DS_CTHREADS) : "memory");
+    return r != 0;
+}
 
-// ---- the warp's position in its stream of units ---------------------------------
-struct DsCursor {
-    int ph;                // phase (n_phases: past the end)
-    int oi;                // op inside the phase
-    int u, u_end;          // position inside the current op
-    const uint8_t* base;   // the op's fragments
-    int ub;                // bytes per unit
-};
+// ---- packed sums ------------------------------------------------------------------
+__device__ __forceinline__ u64 ds_pack(float v) {
+    v = fminf(fmaxf(v, -DS_FIX_MAX), DS_FIX_MAX);
+    return ((u64)__float2ll_rn(v * DS_FIX_ONE) << DS_CNT_BITS) + 1ull;
+}
+__device__ __forceinline__ float ds_unpack(u64 w) { return __ll2float_rn((long long)w >> DS_CNT_BITS) * (1.f / DS_FIX_ONE); }
+__device__ __forceinline__ void ds_ld2(const u64* p, u64& a, u64& b) {
+    asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(a), "=l"(b) : "l"(p) : "memory");
+}
+__device__ __forceinline__ u64 ds_ld1(const u64* p) {
+    u64 a;
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(a) : "l"(p) : "memory");
+    return a;
+}
+__device__ __forceinline__ void ds_red_add(u64* p, u64 v) {
+    asm volatile("red.relaxed.gpu.global.add.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+struct DsQuad { u64 w[4]; };
+__device__ __forceinline__ void ds_ld_quad(const u64* p, DsQuad& q) { ds_ld2(p, q.w[0], q.w[1]); ds_ld2(p + 2, q.w[2], q.w[3]); }
+__device__ __forceinline__ bool ds_quad_ready(const DsQuad& q, uint32_t expect) {
+    return (uint32_t)(q.w[0] & DS_CNT_MASK) == expect && (uint32_t)(q.w[1] & DS_CNT_MASK) == expect &&
+           (uint32_t)(q.w[2] & DS_CNT_MASK) == expect && (uint32_t)(q.w[3] & DS_CNT_MASK) == expect;
+}
+__device__ __forceinline__ float4 ds_quad_value(const DsQuad& q) {
+    return make_float4(ds_unpack(q.w[0]), ds_unpack(q.w[1]), ds_unpack(q.w[2]), ds_unpack(q.w[3]));
+}
+// Re-reads four packed sums until all are complete; false (status raised) when the wait runs out or the grid gave up.
+__device__ __noinline__ bool ds_quad_wait(const u64* p, DsQuad& q, uint32_t expect, u64 wait_ns, int* abort_flag) {
+    const uint64_t t0 = ds_now_ns();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 16; ++i) {
+            ds_ld_quad(p, q);
+            if (ds_quad_ready(q, expect)) return true;
+        }
+        if (*reinterpret_cast<volatile int*>(&g_decode_status) != 0) { *abort_flag = 1; return false; }
+        if (ds_now_ns() - t0 > wait_ns) { atomicCAS(&g_decode_status, 0, 1); *abort_flag = 1; return false; }
+    }
+}
 
+// q holds a first reading of the four sums at p: true once they are complete (re-read as long as needed, into a
+// copy of its own so that q itself can stay in registers).
+__device__ __forceinline__ bool ds_quad_complete(const u64* p, DsQuad& q, uint32_t expect, u64 wait_ns, int* abort_flag) {
+    if (ds_quad_ready(q, expect)) return true;
+    DsQuad t;
+    const bool ok = ds_quad_wait(p, t, expect, wait_ns, abort_flag);
+    q = t;
+    return ok;
+}
+
+// ---- the CTA's share of an op --------------------------------------------------------
 // Every op's units are dealt on their own: with n = q G + r units and G CTAs, slot
 // s takes q + 1 units if s < r, else q; CTA c takes slot (c + rot) mod G, where rot
 // moves on from op to op so that the odd units do not always land on the same CTAs.
@@ -202,36 +274,33 @@ __device__ __forceinline__ void ds_cta_run(int q, int r_rot, int& a, int& b) {
     a = q * s + min(s, r);
     b = a + q + (s < r ? 1 : 0);
 }
-// ... and the run of one of its consumer warps (the warps too take turns with the short shares).
-__device__ __forceinline__ void ds_warp_run(int q, int r_rot, int warp, int& wa, int& wb) {
-    int a, b;
-    ds_cta_run(q, r_rot, a, b);
-    const int n = b - a;
-    int w = warp + ((r_rot >> 16) * 7) % DS_WARPS;
-    if (w >= DS_WARPS) w -= DS_WARPS;
-    wa = a + (n * w) / DS_WARPS;
-    wb = a + (n * (w + 1)) / DS_WARPS;
-}
 
-// Moves the cursor to the next op (from (ph, oi) on) in which the warp owns units.
-// mp / mo: the mini tables (in shared memory when they fit, else in global memory).
-__device__ __forceinline__ void ds_seek(DsCursor& c, const DsMiniPhase* mp, const DsMiniOp* mo, int n_phases, int warp) {
-    while (c.ph < n_phases) {
-        const DsMiniPhase P = mp[c.ph];
-        while (c.oi < P.op_count) {
-            const DsMiniOp op = mo[P.op_first + c.oi];
-            int u0, u1;
-            ds_warp_run((int)(op.q_bits & 0x0FFFFFFFu), (int)op.r_rot, warp, u0, u1);
-            if (u0 < u1) {
-                c.u = u0; c.u_end = u1;
-                c.ub = 2 * frag_bytes((int)(op.q_bits >> 28));
-                c.base = op.frags;
-                return;
-            }
-            ++c.oi;
+// The copy stream's position: consumer w reads positions w, w + DS_WARPS, ... of the list made of the CTA's runs
+// of the phase's ops, one after the other.
+struct DsCursor {
+    int ph, oi;            // phase (n_phases: past the end) and op inside it
+    int pos, base;         // position in the phase's list; position at which op oi's run starts
+    int a, len;            // op oi's run: first unit, number of units
+    const uint8_t* frags;
+    int ub;                // bytes per unit
+};
+__device__ __forceinline__ void ds_cursor_load(DsCursor& c, const DsMiniPhase* mp, const DsMiniOp* mo) {
+    const DsMiniOp op = mo[mp[c.ph].op_first + c.oi];
+    int a, b;
+    ds_cta_run((int)(op.q_bits & 0x0FFFFFFFu), (int)op.r_rot, a, b);
+    c.a = a; c.len = b - a;
+    c.frags = op.frags;
+    c.ub = 2 * frag_bytes((int)(op.q_bits >> 28));
+}
+// Moves (ph, oi, base) on until op oi's run contains pos; a new phase starts again at position `lane`.
+__device__ __forceinline__ void ds_cursor_settle(DsCursor& c, const DsMiniPhase* mp, const DsMiniOp* mo, int n_phases, int lane) {
+    while (c.ph < n_phases && c.pos - c.base >= c.len) {
+        c.base += c.len;
+        if (++c.oi >= mp[c.ph].op_count) {
+            ++c.ph; c.oi = 0; c.base = 0; c.pos = lane;
+            if (c.ph >= n_phases) return;
         }
-        ++c.ph;
-        c.oi = 0;
+        ds_cursor_load(c, mp, mo);
     }
 }
 
@@ -256,16 +325,6 @@ __device__ __forceinline__ uint2 ds_round4(const float4& v, float* sum) {
     return r;
 }
 
-// Four consecutive elements of the input vector of token m at k (k % 4 == 0, k < K), before rounding.
-__device__ __forceinline__ float4 ds_form4(const DsPhase& P, int m, int k, float scale) {
-    const float4 s = __ldcg(reinterpret_cast<const float4*>(P.src + (int64_t)m * P.K + k));
-    if (P.in_op == AQ_IN_SILU_MUL) {
-        const float4 t = __ldcg(reinterpret_cast<const float4*>(P.src2 + (int64_t)m * P.K + k));
-        return make_float4(ds_silu_mul(s.x, t.x), ds_silu_mul(s.y, t.y), ds_silu_mul(s.z, t.z), ds_silu_mul(s.w, t.w));
-    }
-    return make_float4(s.x * scale, s.y * scale, s.z * scale, s.w * scale);
-}
-
 // ---- shared memory ------------------------------------------------------------------
 struct DsShared {
     alignas(128) uint8_t ring[DS_WARPS][DS_SLOTS][DS_SLOT_BYTES];
@@ -275,20 +334,16 @@ struct DsShared {
     alignas(8) uint64_t full[DS_WARPS][DS_SLOTS];    // copy landed
     alignas(8) uint64_t empty[DS_WARPS][DS_SLOTS];   // consumer has read the slot
     alignas(8) uint64_t rec_bar[2];
+    alignas(8) uint2 desc[DS_WARPS][DS_SLOTS];       // the unit in the slot: (op inside the phase, unit index inside the op)
     float red[AQ_DECODE_MAX_M][DS_WARPS];
     float scale[AQ_DECODE_MAX_M];
     int seg_slab_lo[2][DS_MAX_PHASE_OPS];   // per op of the phase: first pair-slab this CTA reads for it
-    int seg_slot_lo[2][DS_MAX_PHASE_OPS];   // ... and the slot in xs where that slab is staged (the next slabs follow)
+    int seg_xoff[2][DS_MAX_PHASE_OPS];      // ... and (slot in xs of that slab) - (that slab): slab P of the op is staged in slot xoff + P
     int slab_of_slot[2][DS_MAX_SLOTS];      // the slabs staged for this phase, ascending
     int n_slots[2];
-    int4 run[DS_MAX_PHASE_OPS][DS_WARPS];   // per op of the phase and consumer warp: first unit, end, its slab, its row tile
-    int run_xslot[DS_MAX_PHASE_OPS][DS_WARPS];   // ... and the slot in xs of that slab
-    alignas(8) uint64_t opbar[DS_OPBARS];   // op (index % DS_OPBARS): the consumer warps that are through with it
-    int released;                           // ops whose arrival the release warp has published
-    int done[32];                           // (no release warp) warps of this CTA that finished op (index & 31)
+    int total[2];                           // units of the phase dealt to this CTA
     int abort_flag;
 };
-
 
 // Writes 4 rounded elements (k .. k+3 of slab-local index) of the staged vector.
 template <int MT>
@@ -317,20 +372,65 @@ __device__ __forceinline__ void ds_load_x_operand(XOperand<MT>& xo, const uint8_
     }
 }
 
+// Cross-lane reduction of a unit's partial sums and one packed red.add per (token, row).  When `res` is given its
+// value field (complete, same shape as out) rides along.
+template <int MT>
+__device__ __forceinline__ void ds_unit_commit(float (&acc)[4], u64* out, const void* res, bool res_plain, int64_t ld, int row0,
+                                               int N, int M, int lane) {
+    const int g = lane >> 2, t = lane & 3;
+    auto put = [&](int tok, int row, float v) {
+        if (tok < M && row < N) {
+            const int64_t o = (int64_t)tok * ld + row;
+            u64 w = ds_pack(v);
+            if (res) {
+                if (res_plain) w += ds_pack(__ldcg(reinterpret_cast<const float*>(res) + o)) - 1ull;
+                else w += ds_ld1(reinterpret_cast<const u64*>(res) + o) & ~DS_CNT_MASK;
+            }
+            ds_red_add(out + o, w);
+        }
+    };
+    if constexpr (MT == 1) {
+        const float v0 = acc[0] + acc[1], v1 = acc[2] + acc[3];
+        float keep = (t & 1) ? v1 : v0;
+        const float send = (t & 1) ? v0 : v1;
+        keep += __shfl_xor_sync(0xffffffffu, send, 1);
+        keep += __shfl_xor_sync(0xffffffffu, keep, 2);
+        if (t < 2) put(0, row0 + g + 8 * t, keep);
+    } else if constexpr (MT == 2) {
+        float kA = (t & 1) ? acc[1] : acc[0], kB = (t & 1) ? acc[3] : acc[2];
+        const float sA = (t & 1) ? acc[0] : acc[1], sB = (t & 1) ? acc[2] : acc[3];
+        kA += __shfl_xor_sync(0xffffffffu, sA, 1);
+        kB += __shfl_xor_sync(0xffffffffu, sB, 1);
+        float v = (t & 2) ? kB : kA;
+        const float s = (t & 2) ? kA : kB;
+        v += __shfl_xor_sync(0xffffffffu, s, 2);
+        put(t & 1, row0 + g + 8 * (t >> 1), v);
+    } else if constexpr (MT == 4) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[i] += __shfl_xor_sync(0xffffffffu, acc[i], 2);
+        const int tk = 2 * (t & 1);
+        const int hi = t >> 1;
+        put(tk, row0 + g + 8 * hi, hi ? acc[2] : acc[0]);
+        put(tk + 1, row0 + g + 8 * hi, hi ? acc[3] : acc[1]);
+    } else {
+        const int tk = 2 * t;
+        put(tk, row0 + g, acc[0]); put(tk, row0 + g + 8, acc[2]);
+        put(tk + 1, row0 + g, acc[1]); put(tk + 1, row0 + g + 8, acc[3]);
+    }
+}
+
 // ---- the kernel ---------------------------------------------------------------------
 template <int MT, bool BF16>
-__global__ void __launch_bounds__(ds_reg_bound(MT), 1) decode_stack_kernel(const DsArgs a) {
-    constexpr bool RELW = ds_release_warp(MT);
+__global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArgs a) {
     extern __shared__ __align__(128) uint8_t ds_smem_raw[];
     DsShared& sh = *reinterpret_cast<DsShared*>(ds_smem_raw);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int M = a.M;
     const int slab_bytes = ds_slab_bytes(M);
+    const u64 wait_ns = a.wait_ns;
 
-    if (threadIdx.x < DS_OPBARS) { ds_mbar_init(ds_smem(&sh.opbar[threadIdx.x]), DS_WARPS); sh.done[threadIdx.x] = 0; }
     if (threadIdx.x == 0) {
         sh.abort_flag = 0;
-        sh.released = 0;
         ds_mbar_init(ds_smem(&sh.rec_bar[0]), 1);
         ds_mbar_init(ds_smem(&sh.rec_bar[1]), 1);
     }
@@ -362,8 +462,12 @@ __global__ void __launch_bounds__(ds_reg_bound(MT), 1) decode_stack_kernel(const
     if (warp == DS_WARPS) {
         // ================= the copy warp: lane w keeps consumer warp w's ring full =================
         DsCursor c;
-        c.ph = a.n_phases; c.oi = 0; c.u = c.u_end = 0; c.base = nullptr; c.ub = 0;
-        if (lane < DS_WARPS) { c.ph = 0; ds_seek(c, mp, mo, a.n_phases, lane); }
+        c.ph = a.n_phases; c.oi = 0; c.pos = 0; c.base = 0; c.a = 0; c.len = 0; c.frags = nullptr; c.ub = 0;
+        if (lane < DS_WARPS && a.n_phases > 0) {
+            c.ph = 0; c.pos = lane;
+            ds_cursor_load(c, mp, mo);
+            ds_cursor_settle(c, mp, mo, a.n_phases, lane);
+        }
         uint32_t iseq = 0;   // copies issued for this consumer
         uint64_t t_progress = ds_now_ns();
         uint32_t idle = 0;
@@ -375,49 +479,26 @@ __global__ void __launch_bounds__(ds_reg_bound(MT), 1) decode_stack_kernel(const
                 const uint32_t slot = iseq % DS_SLOTS, n = iseq / DS_SLOTS;
                 const bool is_free = (n == 0) || ds_mbar_test(ds_smem(&sh.empty[lane][slot]), (n - 1) & 1u);
                 if (is_free) {
+                    const int u = c.a + (c.pos - c.base);
+                    sh.desc[lane][slot] = make_uint2((uint32_t)c.oi, (uint32_t)u);   // (ordered before the copy's arrival
+                                                                                     // by the release of expect_tx)
                     const uint32_t bar = ds_smem(&sh.full[lane][slot]);
                     ds_expect_tx(bar, (uint32_t)c.ub);
-                    ds_bulk_load(ds_smem(&sh.ring[lane][slot][0]), c.base + (int64_t)c.u * c.ub, (uint32_t)c.ub, bar, pol);
+                    ds_bulk_load(ds_smem(&sh.ring[lane][slot][0]), c.frags + (int64_t)u * c.ub, (uint32_t)c.ub, bar, pol);
                     ++iseq;
-                    if (++c.u == c.u_end) { ++c.oi; ds_seek(c, mp, mo, a.n_phases, lane); }
+                    c.pos += DS_WARPS;
+                    ds_cursor_settle(c, mp, mo, a.n_phases, lane);
                     moved = true;
                 }
             }
             if (!__any_sync(0xffffffffu, active)) break;
             if (__any_sync(0xffffffffu, moved)) { idle = 0; continue; }
-            __nanosleep(200);   // a consumer needs about a microsecond per unit: no need to spin on its barriers
+            __nanosleep(200);   // a consumer needs about half a microsecond per unit: no need to spin on its barriers
             if ((++idle & 255u) == 0) {   // nothing to do for a while: stop if the CTA gave up, or after the time limit
                 if (*reinterpret_cast<volatile int*>(&sh.abort_flag)) break;
                 const uint64_t t = ds_now_ns();
                 if (idle == 256u) t_progress = t;
-                else if (t - t_progress > 2 * DS_WAIT_NS) { atomicCAS(&g_decode_status, 0, 2); sh.abort_flag = 1; break; }
-            }
-        }
-        return;
-    }
-
-    if (RELW && warp == DS_WARPS + 1) {
-        // ================= the release warp: publishes, op by op, that this CTA's sums are in place =================
-        // The gpu-scope release waits until the CTA's additions have been acknowledged by L2 (microseconds): here it
-        // holds up nobody, whereas a consumer warp doing it would start its next op that much later.
-        if (lane == 0) {
-            for (int opx = 0; opx < a.n_mini_ops; ++opx) {
-                const uint32_t bar = ds_smem(&sh.opbar[opx % DS_OPBARS]), parity = (uint32_t)(opx / DS_OPBARS) & 1u;
-                const uint64_t t0 = ds_now_ns();
-                bool ok = ds_mbar_try(bar, parity);
-                while (!ok) {
-#pragma unroll 1
-                    for (int i = 0; i < 32 && !ok; ++i) {   // (sleeping between tries: this warp shares a scheduler with consumers)
-                        __nanosleep(100);
-                        ok = ds_mbar_try(bar, parity);
-                    }
-                    if (ok) break;
-                    if (*reinterpret_cast<volatile int*>(&sh.abort_flag)) break;
-                    if (ds_now_ns() - t0 > 2 * DS_WAIT_NS) { atomicCAS(&g_decode_status, 0, 2); sh.abort_flag = 1; break; }
-                }
-                if (!ok) break;
-                asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(a.cnt + opx) : "memory");
-                *reinterpret_cast<volatile int*>(&sh.released) = opx + 1;
+                else if (t - t_progress > 2 * wait_ns) { atomicCAS(&g_decode_status, 0, 2); sh.abort_flag = 1; break; }
             }
         }
         return;
@@ -430,7 +511,7 @@ __global__ void __launch_bounds__(ds_reg_bound(MT), 1) decode_stack_kernel(const
         ds_bulk_load(ds_smem(&sh.rec[q & 1]), a.phases + q, (uint32_t)sizeof(DsPhase), bar, pol_keep);
     };
     if (threadIdx.x == 0) {
-        fetch_record(0);
+        if (a.n_phases > 0) fetch_record(0);
         if (a.n_phases > 1) fetch_record(1);
     }
 
@@ -443,75 +524,61 @@ __global__ void __launch_bounds__(ds_reg_bound(MT), 1) decode_stack_kernel(const
         const int pb = ph & 1;
         const DsPhase& P = sh.rec[pb];
         // -- the phase's descriptors (fetched one phase ahead) --
-        if (!ds_mbar_wait(ds_smem(&sh.rec_bar[pb]), (uint32_t)(ph >> 1) & 1u)) {
+        if (!ds_mbar_wait(ds_smem(&sh.rec_bar[pb]), (uint32_t)(ph >> 1) & 1u, wait_ns)) {
             atomicCAS(&g_decode_status, 0, 2);
             sh.abort_flag = 1;
         }
-        if (*reinterpret_cast<volatile int*>(&sh.abort_flag) == 0) {
-            // -- which slabs of the input this CTA's warps will read (independent of the data) --
-            if (threadIdx.x == DS_CTHREADS - 1) {
-                int lo[DS_MAX_PHASE_OPS], hi[DS_MAX_PHASE_OPS];
-                for (int oi = 0; oi < P.op_count; ++oi) {
-                    int u0, u1;
-                    ds_cta_run(P.ops[oi].units_q, P.ops[oi].units_r_rot, u0, u1);
-                    lo[oi] = (u0 < u1) ? u0 / P.ops[oi].NT : 0;
-                    hi[oi] = (u0 < u1) ? (u1 - 1) / P.ops[oi].NT : -1;
-                    sh.seg_slab_lo[pb][oi] = lo[oi];
-                }
-                // ascending list of the distinct slabs: repeatedly take the smallest one above the last
-                int n = 0, last = -1;
-                for (;;) {
-                    int nxt = 0x7fffffff;
-                    for (int oi = 0; oi < P.op_count; ++oi) {
-                        if (hi[oi] > last) nxt = min(nxt, max(lo[oi], last + 1));
-                    }
-                    if (nxt == 0x7fffffff || n == DS_MAX_SLOTS) break;
-                    sh.slab_of_slot[pb][n++] = nxt;
-                    last = nxt;
-                }
-                sh.n_slots[pb] = n;
-                for (int oi = 0; oi < P.op_count; ++oi) {
-                    int sl = 0;
-                    while (sl < n && sh.slab_of_slot[pb][sl] != lo[oi]) ++sl;
-                    sh.seg_slot_lo[pb][oi] = sl;
-                }
+        // -- which slabs of the input this CTA's warps will read (independent of the data) --
+        if (threadIdx.x == DS_CTHREADS - 1 && *reinterpret_cast<volatile int*>(&sh.abort_flag) == 0) {
+            int lo[DS_MAX_PHASE_OPS], hi[DS_MAX_PHASE_OPS];
+            int total = 0;
+            for (int oi = 0; oi < P.op_count; ++oi) {
+                int u0, u1;
+                ds_cta_run(P.ops[oi].units_q, P.ops[oi].units_r_rot, u0, u1);
+                total += u1 - u0;
+                lo[oi] = (u0 < u1) ? u0 / P.ops[oi].NT : 0;
+                hi[oi] = (u0 < u1) ? (u1 - 1) / P.ops[oi].NT : -1;
+                sh.seg_slab_lo[pb][oi] = lo[oi];
             }
-            // -- wait for the writers of what this phase reads --
-            if ((int)threadIdx.x < P.n_deps) {
-                const uint32_t* c = a.cnt + P.deps[threadIdx.x];
-                uint32_t i = 0;
-                uint64_t t0 = 0;
-                while (ds_ld_acquire(c) < gridDim.x) {
-                    if ((++i & 63u) == 0) {   // now and then: did another CTA give up, or has this wait run out?
-                        if (*reinterpret_cast<volatile int*>(&g_decode_status) != 0) { sh.abort_flag = 1; break; }
-                        const uint64_t t = ds_now_ns();
-                        if (t0 == 0) t0 = t;
-                        if (t - t0 > DS_WAIT_NS) { atomicCAS(&g_decode_status, 0, 1); sh.abort_flag = 1; break; }
-                    }
+            sh.total[pb] = total;
+            // ascending list of the distinct slabs: repeatedly take the smallest one above the last
+            int n = 0, last = -1;
+            for (;;) {
+                int nxt = 0x7fffffff;
+                for (int oi = 0; oi < P.op_count; ++oi) {
+                    if (hi[oi] > last) nxt = min(nxt, max(lo[oi], last + 1));
                 }
+                if (nxt == 0x7fffffff || n == DS_MAX_SLOTS) break;
+                sh.slab_of_slot[pb][n++] = nxt;
+                last = nxt;
+            }
+            sh.n_slots[pb] = n;
+            for (int oi = 0; oi < P.op_count; ++oi) {
+                int sl = 0;
+                while (sl < n && sh.slab_of_slot[pb][sl] != lo[oi]) ++sl;
+                sh.seg_xoff[pb][oi] = sl - lo[oi];
             }
         }
-        ds_consumer_sync();
-        if (*reinterpret_cast<volatile int*>(&sh.abort_flag)) break;
-        // every warp is past phase ph - 1: its record slot is free for phase ph + 1
+        // every warp is through with phase ph - 1: the staged slabs and its record slot are free
+        if (ds_consumer_sync_or(*reinterpret_cast<volatile int*>(&sh.abort_flag))) break;
         if (threadIdx.x == 0 && ph >= 1 && ph + 1 < a.n_phases) fetch_record(ph + 1);
-        // every warp's run in every op of the phase, worked out by one thread each (the warps then switch ops with one load)
-        if ((int)threadIdx.x < P.op_count * DS_WARPS) {
-            const int oi = (int)threadIdx.x / DS_WARPS, w = (int)threadIdx.x - oi * DS_WARPS;
-            const DsOp& op = P.ops[oi];
-            int u0, u1;
-            ds_warp_run(op.units_q, op.units_r_rot, w, u0, u1);
-            const int Pk = (u0 < u1) ? u0 / op.NT : 0;
-            sh.run[oi][w] = make_int4(u0, u1, Pk, u0 - Pk * op.NT);
-            sh.run_xslot[oi][w] = sh.seg_slot_lo[pb][oi] + Pk - sh.seg_slab_lo[pb][oi];
-        }
 
         // -- form the rounded input vector: slabs this CTA reads -> shared memory, its share -> workspace --
         {
             const int n_slots = sh.n_slots[pb];
             const int q4 = P.K >> 2;                                  // groups of 4 elements per token
             const int g0 = (int)(((int64_t)q4 * blockIdx.x) / gridDim.x), g1 = (int)(((int64_t)q4 * (blockIdx.x + 1)) / gridDim.x);
-            uint16_t* rec_out = reinterpret_cast<uint16_t*>(P.stage);
+            uint16_t* stage_out = reinterpret_cast<uint16_t*>(P.stage);
+            const uint32_t expect = P.expect, expect2 = P.expect2;
+            // four consecutive source elements (group i4 of token m), complete; zeros after a failed wait
+            auto source4 = [&](const u64* p, const float* pf, uint32_t ex, int m, int i4) -> float4 {
+                const int64_t o = (int64_t)m * P.K + 4 * (int64_t)i4;
+                if (p == nullptr) return __ldcg(reinterpret_cast<const float4*>(pf + o));
+                DsQuad q;
+                ds_ld_quad(p + o, q);
+                if (!ds_quad_complete(p + o, q, ex, wait_ns, &sh.abort_flag)) return make_float4(0.f, 0.f, 0.f, 0.f);
+                return ds_quad_value(q);
+            };
             // the staged copy of slab `slab`, or null when this CTA does not read it
             auto slot_of = [&](int slab) -> uint8_t* {
                 for (int sl = 0; sl < n_slots; ++sl)
@@ -534,20 +601,39 @@ __global__ void __launch_bounds__(ds_reg_bound(MT), 1) decode_stack_kernel(const
                         if ((lane & 7) == 0) *reinterpret_cast<float*>(sl + 4096 + (kl >> 5) * 4) = sum;
                     }
                 }
-                if (rec) *reinterpret_cast<uint2*>(rec_out + (int64_t)m * P.K + i4 * 4) = r;
+                if (rec) *reinterpret_cast<uint2*>(stage_out + (int64_t)m * P.K + i4 * 4) = r;
             };
             if (P.in_op == AQ_IN_RMSNORM && MT == 1 && q4 <= DS_RMS_HOLD * DS_CTHREADS) {
-                // one token, row held in registers: one trip to L2, destinations worked out while it is under way
+                // one token, row held in registers: one trip to L2 when the row is complete
                 float4 v[DS_RMS_HOLD];
                 uint8_t* dest[DS_RMS_HOLD];
+                if (P.src != nullptr) {
+                    DsQuad q[DS_RMS_HOLD];
 #pragma unroll
-                for (int n = 0; n < DS_RMS_HOLD; ++n) {
-                    const int i4 = threadIdx.x + n * DS_CTHREADS;
-                    v[n] = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (i4 < q4) v[n] = __ldcg(reinterpret_cast<const float4*>(P.src) + i4);
+                    for (int n = 0; n < DS_RMS_HOLD; ++n) {
+                        const int i4 = threadIdx.x + n * DS_CTHREADS;
+                        if (i4 < q4) ds_ld_quad(P.src + 4 * (int64_t)i4, q[n]);
+                    }
+#pragma unroll
+                    for (int n = 0; n < DS_RMS_HOLD; ++n) dest[n] = slot_of((threadIdx.x + n * DS_CTHREADS) >> 6);
+#pragma unroll
+                    for (int n = 0; n < DS_RMS_HOLD; ++n) {
+                        const int i4 = threadIdx.x + n * DS_CTHREADS;
+                        v[n] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (i4 < q4) {
+                            if (ds_quad_complete(P.src + 4 * (int64_t)i4, q[n], expect, wait_ns, &sh.abort_flag)) v[n] = ds_quad_value(q[n]);
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int n = 0; n < DS_RMS_HOLD; ++n) {
+                        const int i4 = threadIdx.x + n * DS_CTHREADS;
+                        v[n] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (i4 < q4) v[n] = __ldcg(reinterpret_cast<const float4*>(P.src_f) + i4);
+                    }
+#pragma unroll
+                    for (int n = 0; n < DS_RMS_HOLD; ++n) dest[n] = slot_of((threadIdx.x + n * DS_CTHREADS) >> 6);
                 }
-#pragma unroll
-                for (int n = 0; n < DS_RMS_HOLD; ++n) dest[n] = slot_of((threadIdx.x + n * DS_CTHREADS) >> 6);
                 float ss = 0.f;
 #pragma unroll
                 for (int n = 0; n < DS_RMS_HOLD; ++n) {
@@ -565,17 +651,18 @@ __global__ void __launch_bounds__(ds_reg_bound(MT), 1) decode_stack_kernel(const
 #pragma unroll
                 for (int n = 0; n < DS_RMS_HOLD; ++n) {
                     const int i4 = threadIdx.x + n * DS_CTHREADS;
-                    if (n * DS_CTHREADS < q4)   // the same for every thread: warps stay whole
-                        place(dest[n], 0, i4, make_float4(v[n].x * scale, v[n].y * scale, v[n].z * scale, v[n].w * scale),
-                              i4 >= g0 && i4 < g1);
+                    if (n * DS_CTHREADS < q4) {   // the same for every thread: warps stay whole
+                        const bool mine = i4 >= g0 && i4 < g1;
+                        if (mine && P.rec) reinterpret_cast<float4*>(P.rec)[i4] = v[n];
+                        place(dest[n], 0, i4, make_float4(v[n].x * scale, v[n].y * scale, v[n].z * scale, v[n].w * scale), mine);
+                    }
                 }
             } else {
                 if (P.in_op == AQ_IN_RMSNORM) {
                     for (int m = 0; m < M; ++m) {
-                        const float4* s4 = reinterpret_cast<const float4*>(P.src + (int64_t)m * P.K);
                         float ss = 0.f;
                         for (int i = threadIdx.x; i < q4; i += DS_CTHREADS) {
-                            const float4 v = __ldcg(s4 + i);
+                            const float4 v = source4(P.src, P.src_f, expect, m, i);
                             ss = fmaf(v.x, v.x, ss); ss = fmaf(v.y, v.y, ss); ss = fmaf(v.z, v.z, ss); ss = fmaf(v.w, v.w, ss);
                         }
 #pragma unroll
@@ -591,7 +678,7 @@ __global__ void __launch_bounds__(ds_reg_bound(MT), 1) decode_stack_kernel(const
                     }
                     ds_consumer_sync();
                 }
-                // one list of work: first the slabs this CTA reads, then its share of the record
+                // one list of work: first the slabs this CTA reads, then its share of the caller's copies
                 const int per_slab = 64 * M;
                 const int n_a = n_slots * per_slab;
                 const int n_b = (g1 - g0) * M;
@@ -613,94 +700,75 @@ __global__ void __launch_bounds__(ds_reg_bound(MT), 1) decode_stack_kernel(const
                         i4 = g0 + w - m * (g1 - g0);
                         valid = true;
                     }
+                    const bool share = it >= n_a;
                     float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (valid) v = ds_form4(P, m, i4 * 4, P.in_op == AQ_IN_RMSNORM ? sh.scale[m] : 1.f);
+                    if (valid) {
+                        const float4 s = source4(P.src, P.src_f, expect, m, i4);
+                        if (share && P.rec) *reinterpret_cast<float4*>(P.rec + (int64_t)m * P.K + 4 * (int64_t)i4) = s;
+                        if (P.in_op == AQ_IN_SILU_MUL) {
+                            const float4 t = source4(P.src2, P.src2_f, expect2, m, i4);
+                            if (share && P.rec2) *reinterpret_cast<float4*>(P.rec2 + (int64_t)m * P.K + 4 * (int64_t)i4) = t;
+                            v = make_float4(ds_silu_mul(s.x, t.x), ds_silu_mul(s.y, t.y), ds_silu_mul(s.z, t.z), ds_silu_mul(s.w, t.w));
+                        } else {
+                            const float sc = (P.in_op == AQ_IN_RMSNORM) ? sh.scale[m] : 1.f;
+                            v = make_float4(s.x * sc, s.y * sc, s.z * sc, s.w * sc);
+                        }
+                    }
                     if (it0 + (int)(threadIdx.x - lane) < n_a) {
                         place(sl, m, i4, v, false);              // n_a is a multiple of 32: the whole warp is inside the slab items
                     } else if (valid) {
                         float sum;
                         const uint2 r = ds_round4<BF16>(v, &sum);
-                        *reinterpret_cast<uint2*>(rec_out + (int64_t)m * P.K + i4 * 4) = r;
+                        *reinterpret_cast<uint2*>(stage_out + (int64_t)m * P.K + i4 * 4) = r;
                     }
                 }
             }
         }
-        ds_consumer_sync();
+        if (ds_consumer_sync_or(*reinterpret_cast<volatile int*>(&sh.abort_flag))) break;
 
-        // -- consume this warp's units of the phase --
+        // -- consume this warp's units of the phase: positions warp, warp + 15, ... of the CTA's list --
+        const int total = sh.total[pb];
 #pragma unroll 1
-        for (int oi = 0; oi < P.op_count; ++oi) {
-            const int opx = P.op_first + oi;
-            const DsOp& op = P.ops[oi];
-            const int NT = op.NT, bits = op.bits;
-            const int4 rn = sh.run[oi][warp];
-            const int u0 = rn.x, u1 = rn.y;
-            if (u0 < u1 && !dead) {
-                int Pk = rn.z, R = rn.w;
-                const uint8_t* xseg = sh.xs + (size_t)sh.run_xslot[oi][warp] * slab_bytes;
-                ds_load_x_operand<MT, BF16>(xo, xseg, M, lane);
-                uint32_t xlane = ds_spread_lane_base(xseg, lane);
-                float* dst = op.dst;
-                const float* res = op.res;
-                const int N = op.N;
-                // the unit loop, one copy per code width (the width is the op's, not the unit's)
-                auto run_units = [&](auto bits_tag) {
-                    constexpr int BITS = decltype(bits_tag)::value;
-#pragma unroll 1
-                    for (int u = u0; u < u1; ++u) {
-                        dead = __any_sync(0xffffffffu, !ds_mbar_wait(ds_smem(&sh.full[warp][cslot]), cparity));
-                        if (dead) {
-                            if (lane == 0) { atomicCAS(&g_decode_status, 0, 2); sh.abort_flag = 1; }
-                            break;
-                        }
-                        const uint8_t* unit = &sh.ring[warp][cslot][0];
-                        float acc[4] = {0.f, 0.f, 0.f, 0.f};
-                        unit_mac<BITS, MT, BF16, MT == 1>(unit, xo, lane, acc, xlane);
-                        __syncwarp();        // every lane has read its part of the slot
-                        if (lane == 0) ds_mbar_arrive(ds_smem(&sh.empty[warp][cslot]));
-                        if (++cslot == DS_SLOTS) { cslot = 0; cparity ^= 1u; }
-                        unit_commit<MT>(acc, dst, N, R * 16, N, M, lane, Pk == 0 ? res : nullptr);
-                        if (++R == NT) {
-                            R = 0; ++Pk;
-                            xseg += slab_bytes;
-                            xlane += (uint32_t)slab_bytes;
-                            if (u + 1 < u1) ds_load_x_operand<MT, BF16>(xo, xseg, M, lane);
-                        }
-                    }
-                };
-                if (bits == 2) run_units(std::integral_constant<int, 2>{});
-                else if (bits == 3) run_units(std::integral_constant<int, 3>{});
-                else run_units(std::integral_constant<int, 4>{});
+        for (int pos = warp; pos < total && !dead; pos += DS_WARPS) {
+            dead = __any_sync(0xffffffffu, !ds_mbar_wait(ds_smem(&sh.full[warp][cslot]), cparity, wait_ns));
+            if (dead) {
+                if (lane == 0) { atomicCAS(&g_decode_status, 0, 2); sh.abort_flag = 1; }
+                break;
             }
-            __syncwarp();
-            if constexpr (RELW) {
-                // arrive: this warp is through with the op (its additions are ordered before the arrival); the release
-                // warp publishes the op once all consumer warps have arrived
-                if (lane == 0) {
-                    // the barriers are a ring: do not lap the release warp
-                    uint32_t spins = 0;
-                    uint64_t t0 = 0;
-                    while (opx - *reinterpret_cast<volatile int*>(&sh.released) >= DS_OPBARS) {
-                        if ((++spins & 255u) == 0) {
-                            if (*reinterpret_cast<volatile int*>(&sh.abort_flag)) break;
-                            const uint64_t t = ds_now_ns();
-                            if (t0 == 0) t0 = t;
-                            if (t - t0 > DS_WAIT_NS) { atomicCAS(&g_decode_status, 0, 2); sh.abort_flag = 1; break; }
-                        }
-                    }
-                    asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];" ::"r"(ds_smem(&sh.opbar[opx % DS_OPBARS])) : "memory");
-                }
-            } else {
-                // arrive: the CTA's last warp to finish the op publishes it (the warps' commits are ordered before the
-                // release below through the acq_rel counter in shared memory)
-                if (lane == 0) {
-                    int old;
-                    asm volatile("atom.acq_rel.cta.shared::cta.add.u32 %0, [%1], 1;" : "=r"(old) : "r"(ds_smem(&sh.done[opx & 31])) : "memory");
-                    if (old == DS_WARPS - 1) {
-                        sh.done[opx & 31] = 0;
-                        asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(a.cnt + opx) : "memory");
-                    }
-                }
+            const uint2 ds = sh.desc[warp][cslot];
+            const DsOp& op = P.ops[ds.x];
+            const int NT = op.NT;
+            int Pk = op.nt_magic ? (int)__umulhi(ds.y, op.nt_magic) : (int)ds.y;   // (no magic: NT = 1)
+            int R = (int)ds.y - Pk * NT;
+            if (R < 0) { --Pk; R += NT; }
+            const uint8_t* xseg = sh.xs + (size_t)(sh.seg_xoff[pb][ds.x] + Pk) * slab_bytes;
+            ds_load_x_operand<MT, BF16>(xo, xseg, M, lane);
+            const uint32_t xlane = ds_spread_lane_base(xseg, lane);
+            const uint8_t* unit = &sh.ring[warp][cslot][0];
+            float acc[4] = {0.f, 0.f, 0.f, 0.f};
+            const int bits = op.bits & 0xFF;
+            const bool res_plain = (op.bits & DS_RES_PLAIN) != 0;
+            if (bits == 2) unit_mac<2, MT, BF16, MT == 1>(unit, xo, lane, acc, xlane);
+            else if (bits == 3) unit_mac<3, MT, BF16, MT == 1>(unit, xo, lane, acc, xlane);
+            else unit_mac<4, MT, BF16, MT == 1>(unit, xo, lane, acc, xlane);
+            __syncwarp();        // every lane has read its part of the slot
+            if (lane == 0) ds_mbar_arrive(ds_smem(&sh.empty[warp][cslot]));
+            if (++cslot == DS_SLOTS) { cslot = 0; cparity ^= 1u; }
+            ds_unit_commit<MT>(acc, op.dst, Pk == 0 ? op.res : nullptr, res_plain, op.N, R * 16, op.N, M, lane);
+        }
+    }
+
+    // -- buffers no phase reads (and the last outputs): float32 copies for the caller, one chunk per warp --
+    if (*reinterpret_cast<volatile int*>(&sh.abort_flag) == 0) {
+#pragma unroll 1
+        for (int e = (int)blockIdx.x * DS_WARPS + warp; e < a.n_tails; e += (int)gridDim.x * DS_WARPS) {
+            const DsTail T = a.tails[e];
+            bool ok = true;
+            for (int i = lane * 4; i < T.n && ok; i += 128) {      // n is a multiple of 4
+                DsQuad q;
+                ds_ld_quad(T.src + i, q);
+                if (!ds_quad_complete(T.src + i, q, T.expect, wait_ns, &sh.abort_flag)) ok = false;
+                else *reinterpret_cast<float4*>(T.out + i) = ds_quad_value(q);
             }
         }
     }
@@ -715,11 +783,13 @@ namespace {
 struct DecodePlan {
     std::vector<uint8_t> key;
     std::vector<aq_handle_t> handles;
-    uint8_t* dev = nullptr;       // [phase records][mini phases, mini ops][arrival counters]
-    size_t phases_bytes = 0, mini_bytes = 0, cnt_bytes = 0;
+    uint8_t* dev = nullptr;       // [phase records][mini phases, mini ops][tail chunks]
+    size_t phases_bytes = 0, mini_bytes = 0, tail_bytes = 0;
     int n_mini_ops = 0;
     int n_phases = 0;
+    int n_tails = 0;
     int device = 0;
+    bool pinned = false;          // recorded into a CUDA graph: its device tables must outlive the plan cache's turnover
     uint64_t stamp = 0;
 };
 
@@ -727,6 +797,8 @@ std::mutex g_plan_mutex;
 std::vector<DecodePlan*> g_plans;
 uint64_t g_plan_clock = 0;
 constexpr size_t MAX_PLANS = 16;
+u64 g_wait_ns = DS_WAIT_NS_DEFAULT;
+bool g_hold = false;          // testing: the first packed input of a program expects one contribution too many
 
 void drop_plan(DecodePlan* p) {
     if (p->dev) cudaFree(p->dev);
@@ -741,14 +813,21 @@ template <typename T> void key_put(std::vector<uint8_t>& k, const T& v) {
 }  // namespace
 
 // Device tables of a program: one record per phase (at most DS_MAX_PHASE_OPS ops that
-// read the same input vector).  False when the program does not fit this kernel.
+// read the same input vector) and the list of buffers nobody reads.  False when the program
+// does not fit this kernel.
 bool build_decode_tables(const aq_stack_t* p, const StackPlan& plan, int M, int n_cta, uint8_t* ws,
-                         std::vector<DsPhase>& phases) {
-    if (M < 1 || M > AQ_DECODE_MAX_M || p->n_ops > 32000) return false;
+                         std::vector<DsPhase>& phases, std::vector<DsTail>& tails) {
+    if (M < 1 || M > AQ_DECODE_MAX_M || p->n_ops > 32000 || plan.pk_off.empty()) return false;
     phases.clear();
-    std::vector<int> writer(p->n_bufs, -1);
-    std::vector<char> waited(p->n_ops, 0);
+    tails.clear();
+    std::vector<int> writer(p->n_bufs, -1);         // op that writes the buffer
+    std::vector<char> whole(p->n_bufs, 0);          // every CTA has seen the whole buffer complete (a normalised input)
+    std::vector<char> recorded(p->n_bufs, 0);       // some phase writes the caller's float32 copy
+    auto packed = [&](int b) { return reinterpret_cast<u64*>(ws + plan.pk_off[b]); };
+    auto plain = [&](int b) { return reinterpret_cast<float*>(ws + plan.buf_off[b]); };
+    auto expect_of = [&](int b) { return (uint32_t)p->ops[writer[b]].w->KP; };
     int rot = 0;   // where the next op's odd units start
+    bool hold = g_hold;
     const int n_ph = (int)plan.phase_first.size();
     for (int ph = 0; ph < n_ph; ++ph) {
         const int pfirst = plan.phase_first[ph];
@@ -770,8 +849,9 @@ bool build_decode_tables(const aq_stack_t* p, const StackPlan& plan, int M, int 
                     const aq_handle_s* h = p->ops[i].w;
                     DsOp& d = P.ops[i - first];
                     const int64_t nu = (int64_t)h->KP * h->NT;
-                    if (off + nu > (int64_t)1 << 26) { ok = false; break; }
-                    d.N = (int32_t)h->N; d.NT = h->NT; d.n_units = (int32_t)nu; d.bits = h->bits;
+                    if (off + nu > (int64_t)1 << 26 || h->KP > DS_MAX_CONTRIB) { ok = false; break; }
+                    d.N = (int32_t)h->N; d.NT = h->NT; d.bits = h->bits;
+                    d.nt_magic = h->NT > 1 ? (uint32_t)(((uint64_t)1 << 32) / (uint64_t)h->NT + 1) : 0u;
                     d.units_q = (int32_t)(nu / n_cta);
                     d.units_r_rot = (int32_t)(nu % n_cta) | (r2 << 16);
                     r2 = (int)((r2 + nu % n_cta) % n_cta);
@@ -790,36 +870,55 @@ bool build_decode_tables(const aq_stack_t* p, const StackPlan& plan, int M, int 
                     const int64_t slabs = std::unique(need.begin(), need.end()) - need.begin();
                     if (slabs > DS_MAX_SLOTS || slabs * ds_slab_bytes(M) > DS_XS_BYTES) ok = false;
                 }
-                if (ok) { P.units_total = (int32_t)off; rot_after = r2; break; }
+                if (ok) { rot_after = r2; break; }
             }
             if (count < 1) return false;
             const int last = first + count;
             rot = rot_after;
-            P.src = reinterpret_cast<const float*>(ws + plan.buf_off[f.src]);
-            P.src2 = (f.in_op == AQ_IN_SILU_MUL) ? reinterpret_cast<const float*>(ws + plan.buf_off[f.src2]) : nullptr;
-            P.stage = ws + plan.in_off[first];
-            P.K = (int32_t)K; P.in_op = f.in_op; P.op_first = first; P.op_count = count;
-            std::vector<int> deps;
-            auto need = [&](int buf) {
-                const int w = writer[buf];
-                if (w >= 0 && !waited[w]) { waited[w] = 1; deps.push_back(w); }
+            auto source = [&](int b, const u64*& sp, const float*& sf, float*& rec, uint32_t& ex) {
+                if (writer[b] < 0) { sp = nullptr; sf = plain(b); rec = nullptr; ex = 0; return; }   // the program input
+                sp = packed(b); sf = nullptr; ex = expect_of(b);
+                rec = recorded[b] ? nullptr : plain(b);
+                recorded[b] = 1;
             };
-            need(f.src);
-            if (f.in_op == AQ_IN_SILU_MUL) need(f.src2);
+            source(f.src, P.src, P.src_f, P.rec, P.expect);
+            if (hold && P.src) { P.expect += 1; hold = false; }   // (a count no row reaches: every CTA's wait runs out)
+            if (f.in_op == AQ_IN_SILU_MUL) source(f.src2, P.src2, P.src2_f, P.rec2, P.expect2);
+            if (f.in_op == AQ_IN_RMSNORM) whole[f.src] = 1;
+            P.stage = ws + plan.in_off[first];
+            P.K = (int32_t)K; P.in_op = f.in_op; P.op_count = count;
             for (int i = first; i < last; ++i) {
                 const aq_stack_op_t& o = p->ops[i];
                 DsOp& d = P.ops[i - first];
                 d.frags = o.w->frags;
-                d.dst = reinterpret_cast<float*>(ws + plan.buf_off[o.dst]);
-                d.res = (o.out_op == AQ_OUT_ADD) ? reinterpret_cast<const float*>(ws + plan.buf_off[o.res]) : nullptr;
-                if (o.out_op == AQ_OUT_ADD) need(o.res);
+                d.dst = packed(o.dst);
+                d.res = nullptr;
+                if (o.out_op == AQ_OUT_ADD) {
+                    // the residual is read without a wait: it must be complete for every CTA when the phase starts,
+                    // i.e. the program input (plain float32) or an input that every CTA has already read as a whole
+                    // (a normalised one)
+                    if (writer[o.res] < 0) { d.res = plain(o.res); d.bits |= DS_RES_PLAIN; }
+                    else if (whole[o.res]) d.res = packed(o.res);
+                    else return false;
+                }
             }
-            if ((int)deps.size() > DS_MAX_DEPS) return false;
-            P.n_deps = (int)deps.size();
-            for (size_t j = 0; j < deps.size(); ++j) P.deps[j] = (int16_t)deps[j];
             for (int i = first; i < last; ++i) writer[p->ops[i].dst] = i;
             phases.push_back(P);
             first = last;
+        }
+    }
+    // what no phase has copied out for the caller
+    for (int b = 1; b < p->n_bufs; ++b) {
+        if (writer[b] < 0 || recorded[b]) continue;
+        const int64_t n = (int64_t)M * p->buf_width[b];
+        if (n % 4) return false;
+        for (int64_t i = 0; i < n; i += DS_TAIL_CHUNK) {
+            DsTail t;
+            memset(&t, 0, sizeof(t));
+            t.src = packed(b) + i; t.out = plain(b) + i;
+            t.n = (int32_t)std::min<int64_t>(DS_TAIL_CHUNK, n - i);
+            t.expect = expect_of(b);
+            tails.push_back(t);
         }
     }
     return true;
@@ -828,19 +927,21 @@ bool build_decode_tables(const aq_stack_t* p, const StackPlan& plan, int M, int 
 template <int MT, bool BF16>
 static cudaError_t launch_ds(const DsArgs& a, int grid, cudaStream_t s) {
     auto kern = decode_stack_kernel<MT, BF16>;
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DsShared));
-        if (e != cudaSuccess) return e;
-        int per_sm = 0;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, ds_threads(MT), sizeof(DsShared));
-        if (e != cudaSuccess) return e;
-        if (per_sm < 1) return cudaErrorCooperativeLaunchTooLarge;
-        configured = true;
+    static PerDeviceOnce configured;
+    {
+        const int rc = configured.run(current_device(), [&] {
+            cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DsShared));
+            if (e != cudaSuccess) return (int)e;
+            int per_sm = 0;
+            e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, DS_THREADS, sizeof(DsShared));
+            if (e != cudaSuccess) return (int)e;
+            return per_sm < 1 ? (int)cudaErrorCooperativeLaunchTooLarge : 0;
+        });
+        if (rc != 0) return rc < 0 ? cudaErrorInvalidDevice : (cudaError_t)rc;
     }
     DsArgs args = a;
     void* params[1] = {&args};
-    cudaError_t e = cudaLaunchCooperativeKernel(reinterpret_cast<void*>(kern), dim3((unsigned)grid), dim3(ds_threads(MT)), params,
+    cudaError_t e = cudaLaunchCooperativeKernel(reinterpret_cast<void*>(kern), dim3((unsigned)grid), dim3(DS_THREADS), params,
                                                 sizeof(DsShared), s);
     if (e == cudaSuccess) count_launch();
     return e;
@@ -850,11 +951,15 @@ int launch_decode_stack(const aq_stack_t* p, const StackPlan& plan, int M, aq_dt
                         cudaError_t* err) {
     *err = cudaSuccess;
     const int grid = sm_count();
-    int dev = 0;
-    cudaGetDevice(&dev);
+    const int dev = current_device();
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(s, &cap) != cudaSuccess) { cudaGetLastError(); cap = cudaStreamCaptureStatusNone; }
+    const bool capturing = (cap != cudaStreamCaptureStatusNone);
     // key: everything the device tables are computed from
     std::vector<uint8_t> key;
     key_put(key, M); key_put(key, dev); key_put(key, grid); key_put(key, ws);
+    std::lock_guard<std::mutex> lock(g_plan_mutex);
+    key_put(key, g_hold);
     key_put(key, p->n_ops); key_put(key, p->n_bufs);
     for (int i = 0; i < p->n_ops; ++i) {
         key_put(key, p->ops[i]);
@@ -862,13 +967,22 @@ int launch_decode_stack(const aq_stack_t* p, const StackPlan& plan, int M, aq_dt
     }
     for (int b = 0; b < p->n_bufs; ++b) key_put(key, p->buf_width[b]);
 
-    std::lock_guard<std::mutex> lock(g_plan_mutex);
     DecodePlan* dp = nullptr;
     for (DecodePlan* q : g_plans)
         if (q->key == key) { dp = q; break; }
     if (!dp) {
+        if (capturing) return 1;   // tables are built (allocation, synchronous copies) by an eager call only
         std::vector<DsPhase> phases;
-        if (!build_decode_tables(p, plan, M, grid, ws, phases)) return 1;
+        std::vector<DsTail> tails;
+        if (!build_decode_tables(p, plan, M, grid, ws, phases, tails)) return 1;
+        if (g_plans.size() >= MAX_PLANS) {   // make room: the oldest plan no graph refers to
+            size_t oldest = g_plans.size();
+            for (size_t i = 0; i < g_plans.size(); ++i)
+                if (!g_plans[i]->pinned && (oldest == g_plans.size() || g_plans[i]->stamp < g_plans[oldest]->stamp)) oldest = i;
+            if (oldest == g_plans.size()) return 1;   // all pinned: this program runs op by op
+            drop_plan(g_plans[oldest]);
+            g_plans.erase(g_plans.begin() + oldest);
+        }
         dp = new DecodePlan();
         dp->key = key;
         dp->device = dev;
@@ -886,38 +1000,38 @@ int launch_decode_stack(const aq_stack_t* p, const StackPlan& plan, int M, aq_dt
             for (int j = 0; j < phases[i].op_count; ++j) {
                 DsMiniOp mop;
                 mop.frags = phases[i].ops[j].frags;
-                mop.q_bits = (uint32_t)phases[i].ops[j].units_q | ((uint32_t)phases[i].ops[j].bits << 28);
+                mop.q_bits = (uint32_t)phases[i].ops[j].units_q | ((uint32_t)(phases[i].ops[j].bits & 0xFF) << 28);
                 mop.r_rot = (uint32_t)phases[i].ops[j].units_r_rot;
                 const uint8_t* b = reinterpret_cast<const uint8_t*>(&mop);
                 mini.insert(mini.end(), b, b + sizeof(mop));
             }
         dp->mini_bytes = (mini.size() + 255) / 256 * 256;
-        dp->cnt_bytes = ((size_t)p->n_ops * sizeof(uint32_t) + 255) / 256 * 256;
+        dp->tail_bytes = (tails.size() * sizeof(DsTail) + 255) / 256 * 256;
         dp->n_phases = (int)phases.size();
-        cudaError_t e = cudaMalloc(&dp->dev, dp->phases_bytes + dp->mini_bytes + dp->cnt_bytes);
+        dp->n_tails = (int)tails.size();
+        cudaError_t e = cudaMalloc(&dp->dev, dp->phases_bytes + dp->mini_bytes + dp->tail_bytes + 256);
         if (e == cudaSuccess) e = cudaMemcpy(dp->dev, phases.data(), phases.size() * sizeof(DsPhase), cudaMemcpyHostToDevice);
         if (e == cudaSuccess) e = cudaMemcpy(dp->dev + dp->phases_bytes, mini.data(), mini.size(), cudaMemcpyHostToDevice);
+        if (e == cudaSuccess && !tails.empty())
+            e = cudaMemcpy(dp->dev + dp->phases_bytes + dp->mini_bytes, tails.data(), tails.size() * sizeof(DsTail), cudaMemcpyHostToDevice);
         if (e != cudaSuccess) { cudaGetLastError(); drop_plan(dp); *err = e; return -1; }
-        if (g_plans.size() >= MAX_PLANS) {
-            size_t oldest = 0;
-            for (size_t i = 1; i < g_plans.size(); ++i)
-                if (g_plans[i]->stamp < g_plans[oldest]->stamp) oldest = i;
-            drop_plan(g_plans[oldest]);
-            g_plans.erase(g_plans.begin() + oldest);
-        }
         g_plans.push_back(dp);
     }
     dp->stamp = ++g_plan_clock;
+    if (capturing) dp->pinned = true;
 
     DsArgs a;
     a.phases = reinterpret_cast<const DsPhase*>(dp->dev);
     a.mini_phases = reinterpret_cast<const DsMiniPhase*>(dp->dev + dp->phases_bytes);
     a.mini_ops = reinterpret_cast<const DsMiniOp*>(dp->dev + dp->phases_bytes + (size_t)dp->n_phases * sizeof(DsMiniPhase));
+    a.tails = reinterpret_cast<const DsTail*>(dp->dev + dp->phases_bytes + dp->mini_bytes);
     a.n_mini_ops = dp->n_mini_ops;
-    a.cnt = reinterpret_cast<uint32_t*>(dp->dev + dp->phases_bytes + dp->mini_bytes);
     a.n_phases = dp->n_phases;
+    a.n_tails = dp->n_tails;
     a.M = M;
-    cudaError_t e = cudaMemsetAsync(a.cnt, 0, dp->cnt_bytes, s);
+    a.wait_ns = g_wait_ns;
+    // the packed sums start from zero
+    cudaError_t e = cudaMemsetAsync(ws + plan.pk_begin, 0, plan.pk_end - plan.pk_begin, s);
     if (e == cudaSuccess) {
         const bool bf = (dt == AQ_BF16);
         if (M == 1) e = bf ? launch_ds<1, true>(a, grid, s) : launch_ds<1, false>(a, grid, s);
@@ -945,6 +1059,16 @@ int read_decode_status(bool clear) {
     cudaMemcpyFromSymbol(&v, g_decode_status, sizeof(int));
     if (clear && v) { int z = 0; cudaMemcpyToSymbol(g_decode_status, &z, sizeof(int)); }
     return v;
+}
+
+void set_decode_hold(bool on) {
+    std::lock_guard<std::mutex> lock(g_plan_mutex);
+    g_hold = on;
+}
+
+void set_decode_wait_ns(unsigned long long ns) {
+    std::lock_guard<std::mutex> lock(g_plan_mutex);
+    g_wait_ns = ns ? ns : DS_WAIT_NS_DEFAULT;
 }
 
 }  // namespace aq

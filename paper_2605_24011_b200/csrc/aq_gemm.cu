@@ -482,11 +482,12 @@ template <bool BF16>
 static cudaError_t launch_one(const CUtensorMap& tm, const GemmOutMaps& tmo, const GemmArgs& a, int grid, cudaStream_t s) {
     constexpr int SMEM = 1024 + GM_ASTAGES * GM_A_BYTES + GM_BSLOTS * GM_B_BYTES + GM_PSTAGES * 8 * frag_bytes(4) + 256;
     auto kern = gemm_kernel<BF16>;
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
-        if (e != cudaSuccess) return e;
-        configured = true;
+    static PerDeviceOnce configured;
+    {
+        const int rc = configured.run(current_device(), [&] {
+            return (int)cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
+        });
+        if (rc != 0) return rc < 0 ? cudaErrorInvalidDevice : (cudaError_t)rc;
     }
     cudaError_t e = launch_pdl(kern, dim3((unsigned)grid), dim3(GM_THREADS), SMEM, s, tm, tmo, a);
     count_launch();

@@ -131,12 +131,13 @@ template <int BITS, int MT, bool BF16>
 static cudaError_t launch_one(const GemvArgs& a, cudaStream_t s) {
     constexpr int UB = 2 * frag_bytes(BITS);
     constexpr int SMEM = GEMV_WARPS * GEMV_STAGES * UB;
-    static bool configured = false;   // per (template instance); attribute is per device context
+    static PerDeviceOnce configured;   // per template instance and device: the attribute belongs to the device's context
     auto kern = gemv_kernel<BITS, MT, BF16>;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
-        if (e != cudaSuccess) return e;
-        configured = true;
+    {
+        const int rc = configured.run(current_device(), [&] {
+            return (int)cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
+        });
+        if (rc != 0) return rc < 0 ? cudaErrorInvalidDevice : (cudaError_t)rc;
     }
     const int64_t warps_wanted = a.n_units;
     int grid = 2 * sm_count();

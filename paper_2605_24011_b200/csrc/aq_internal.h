@@ -6,6 +6,7 @@
 #include <vector>
 
 #include "../../include/aq.h"
+#include "aq_per_device.h"
 
 #define AQ_HANDLE_MAGIC 0x41514831u   /* "AQH1" */
 
@@ -62,6 +63,8 @@ struct StackPlan {
     std::vector<size_t> buf_off;    // per buffer: float32 [M][width]
     std::vector<size_t> in_off;     // per op: its phase's staged input [M][K] (activation dtype)
     std::vector<int> phase_first;   // first op of each phase (ops that share one input vector)
+    std::vector<size_t> pk_off;     // per buffer (M <= AQ_DECODE_MAX_M only): its packed 64-bit sums [M][width]
+    size_t pk_begin = 0, pk_end = 0;   // the packed sums' region: zero at the start of a decode pass
     size_t stage_off = 0;           // end of the float32 buffers
     size_t total = 0;
 };
@@ -72,6 +75,8 @@ int launch_decode_stack(const aq_stack_t* p, const StackPlan& plan, int M, aq_dt
                         cudaError_t* err);
 void decode_stack_forget(aq_handle_t h);   // drops cached device tables that name h
 int read_decode_status(bool clear);        // nonzero: a bounded wait in the decode-stack kernel ran out
+void set_decode_wait_ns(unsigned long long ns);   // limit of every wait in that kernel (0: the default, two seconds)
+void set_decode_hold(bool on);             // testing: tables built while on expect a contribution that never comes
 
 // Programmatic dependent launch, used along the prefill path: a kernel launched with launch_pdl may become
 // resident while its predecessor on the stream still runs; it must execute pdl_wait() before it touches anything the
@@ -102,7 +107,8 @@ int allocate_bits_host(const double* S, const int64_t* numel, const int32_t* lay
                        int n_types, double budget, int32_t* bits_out, double* objective_out);   // 0 ok, 1 malformed, 2 budget
 int read_stage1_status(bool clear);
 
-int sm_count();
+int current_device();               // cudaGetDevice, or -1
+int sm_count();                     // of the current device
 void count_launch(int n = 1);       // process-wide count of this library's kernel launches
 int read_gemm_status(bool clear);   // nonzero: a bounded wait in the GEMM kernel ran out
 

@@ -58,6 +58,15 @@ static bool plan_stack(const aq_stack_t* p, int M, StackPlan& plan) {
         plan.in_off[i] = off;
         off += align_up((size_t)M * p->buf_width[p->ops[i].src] * 2, 256);
     }
+    if (M <= AQ_DECODE_MAX_M) {   // the whole-program decode kernel accumulates packed 64-bit sums, one per element
+        plan.pk_off.assign(p->n_bufs, 0);
+        plan.pk_begin = off;
+        for (int b = 1; b < p->n_bufs; ++b) {
+            plan.pk_off[b] = off;
+            off += align_up((size_t)M * p->buf_width[b] * 8, 256);
+        }
+        plan.pk_end = off;
+    }
     plan.total = off;
     (void)maxw;
     return true;
@@ -159,10 +168,6 @@ static cudaError_t run_stack(const aq_stack_t* p, const StackPlan& plan, const T
                              aq_dtype_t dt, uint8_t* ws, cudaStream_t s) {
     cudaError_t e = cudaSuccess;
     const bool decode = (M <= AQ_DECODE_MAX_M);
-    if (decode) {   // the streaming kernel accumulates with red.add: outputs start at zero
-        e = cudaMemsetAsync(ws, 0, plan.stage_off, s);
-        if (e != cudaSuccess) return e;
-    }
     auto buf = [&](int b) { return reinterpret_cast<float*>(ws + plan.buf_off[b]); };
     {
         const int64_t n = (int64_t)M * p->buf_width[0];
@@ -181,6 +186,9 @@ static cudaError_t run_stack(const aq_stack_t* p, const StackPlan& plan, const T
             count_launch();
         }
         if (r == 0) return cudaGetLastError();
+        // op by op: the streaming kernel accumulates with red.add, so every output starts at zero
+        e = cudaMemsetAsync(ws + plan.buf_off[1], 0, plan.stage_off - plan.buf_off[1], s);
+        if (e != cudaSuccess) return e;
     }
     int i = 0;
     while (i < p->n_ops) {

@@ -41,8 +41,10 @@ def test_quantiser_invariants(W, bits):
     # scale zero <=> every code of the block is zero is implied one way: scale 0 gives codes 0
     zero = (d64 == 0)
     assert np.all(q.reshape(N, K // 32, 32)[zero] == 0)
-    # the extreme elements of a block with a usable scale take the extreme codes (up to one step of rounding)
-    usable = finite & (d64 > 0)
+    # the extreme elements of a block with a usable scale take the extreme codes (up to one step of rounding), as long
+    # as rounding min and scale to binary16 moved the grid by less than half a step (a block like 59985 .. 59986, whose
+    # minimum rounds to a multiple of 32, lands wholly on one end of the grid: covered by the error bound above)
+    usable = finite & (d64 > 0) & (slack <= d64 / 2)
     qb = q.reshape(N, K // 32, 32)
     assert np.all(qb.min(axis=2)[usable] <= 1)
     assert np.all(qb.max(axis=2)[usable] >= L - 1)
