@@ -59,6 +59,7 @@ constexpr int DS_MAX_SLOTS = 6;             // staged slabs per phase per CTA (o
 constexpr int DS_XS_BYTES = DS_MAX_SLOTS * 4224;   // staged input (see ds_slab_bytes)
 constexpr int DS_MAX_PHASE_OPS = 8;
 constexpr int DS_RMS_HOLD = 4;              // groups of four elements per thread kept in registers by the one-token RMS path
+constexpr int DS_DESC_BITS_SHIFT = 8;       // descriptor word 0: op inside the phase | code width << 8
 constexpr u64 DS_WAIT_NS_DEFAULT = 2000000000ull;   // every wait gives up after two seconds
 
 // A packed sum: bits [12, 64) hold the value in units of 2^-24 (two's complement), bits [0, 12) the number of
@@ -115,14 +116,27 @@ struct DsMiniOp {
     const uint8_t* frags;
     uint32_t q_bits;       // units_q | bits << 28
     uint32_t r_rot;        // units_r | rot << 16
+    int32_t NT;
+    uint32_t nt_magic;
+    int32_t pad_[2];
 };
 struct DsMiniPhase {
     int32_t op_first;      // index into the mini-op table
     int32_t op_count;
     int32_t pad_[2];
 };
-static_assert(sizeof(DsMiniOp) == 16 && sizeof(DsMiniPhase) == 16, "mini tables are copied as 16-byte items");
-constexpr int DS_MINI_BYTES = 8192;
+static_assert(sizeof(DsMiniOp) == 32 && sizeof(DsMiniPhase) == 16, "mini tables are copied as 16-byte items");
+constexpr int DS_MINI_BYTES = 10240;
+
+// What one CTA needs to know of one phase besides the phase record: worked out on the host, since it depends on
+// nothing but the shapes (a single thread doing this in the kernel sat on every phase's critical path).
+struct DsCtaPhase {
+    int32_t total;                          // units of the phase dealt to this CTA
+    int32_t n_slots;                        // staged slabs
+    int32_t slab_of_slot[DS_MAX_SLOTS];     // the pair-slabs staged for the phase, ascending
+    int32_t xoff[DS_MAX_PHASE_OPS];         // per op: (slot of its first slab) - (that slab): slab P sits in slot xoff + P
+};
+static_assert(sizeof(DsCtaPhase) == 64, "DsCtaPhase layout");
 
 // A stretch of a buffer no phase reads: converted to float32 for the caller once the last phase is done.
 struct DsTail {
@@ -140,6 +154,7 @@ struct DsArgs {
     const DsMiniPhase* mini_phases;   // n_phases entries, followed by
     const DsMiniOp* mini_ops;         // n_mini_ops entries (contiguous: one copy brings both)
     const DsTail* tails;
+    const DsCtaPhase* ctab;           // [phase][CTA]
     u64 wait_ns;
     int n_phases;
     int n_mini_ops;
@@ -283,6 +298,9 @@ struct DsCursor {
     int a, len;            // op oi's run: first unit, number of units
     const uint8_t* frags;
     int ub;                // bytes per unit
+    int NT;                // the op's row tiles and the magic number that divides by them
+    uint32_t magic;
+    uint32_t word0;        // op inside the phase | bits << 8, for the unit's descriptor
 };
 __device__ __forceinline__ void ds_cursor_load(DsCursor& c, const DsMiniPhase* mp, const DsMiniOp* mo) {
     const DsMiniOp op = mo[mp[c.ph].op_first + c.oi];
@@ -291,6 +309,8 @@ __device__ __forceinline__ void ds_cursor_load(DsCursor& c, const DsMiniPhase* m
     c.a = a; c.len = b - a;
     c.frags = op.frags;
     c.ub = 2 * frag_bytes((int)(op.q_bits >> 28));
+    c.NT = op.NT; c.magic = op.nt_magic;
+    c.word0 = (uint32_t)c.oi | ((op.q_bits >> 28) << DS_DESC_BITS_SHIFT);
 }
 // Moves (ph, oi, base) on until op oi's run contains pos; a new phase starts again at position `lane`.
 __device__ __forceinline__ void ds_cursor_settle(DsCursor& c, const DsMiniPhase* mp, const DsMiniOp* mo, int n_phases, int lane) {
@@ -334,14 +354,10 @@ struct DsShared {
     alignas(8) uint64_t full[DS_WARPS][DS_SLOTS];    // copy landed
     alignas(8) uint64_t empty[DS_WARPS][DS_SLOTS];   // consumer has read the slot
     alignas(8) uint64_t rec_bar[2];
-    alignas(8) uint2 desc[DS_WARPS][DS_SLOTS];       // the unit in the slot: (op inside the phase, unit index inside the op)
+    alignas(16) uint4 desc[DS_WARPS][DS_SLOTS];      // the unit in the slot: (op | bits << 8, pair-slab, row tile, -)
+    alignas(16) DsCtaPhase ctab[2];         // this CTA's tables of the current and the next phase
     float red[AQ_DECODE_MAX_M][DS_WARPS];
     float scale[AQ_DECODE_MAX_M];
-    int seg_slab_lo[2][DS_MAX_PHASE_OPS];   // per op of the phase: first pair-slab this CTA reads for it
-    int seg_xoff[2][DS_MAX_PHASE_OPS];      // ... and (slot in xs of that slab) - (that slab): slab P of the op is staged in slot xoff + P
-    int slab_of_slot[2][DS_MAX_SLOTS];      // the slabs staged for this phase, ascending
-    int n_slots[2];
-    int total[2];                           // units of the phase dealt to this CTA
     int abort_flag;
 };
 
@@ -373,21 +389,28 @@ __device__ __forceinline__ void ds_load_x_operand(XOperand<MT>& xo, const uint8_
 }
 
 // Cross-lane reduction of a unit's partial sums and one packed red.add per (token, row).  When `res` is given its
-// value field (complete, same shape as out) rides along.
+// value (complete, same shape as out) rides along.  Free of branches when res is null (bounds are predicates), so
+// that the compiler can weave it into the next unit's arithmetic.
+__device__ __forceinline__ void ds_red_add_if(u64* p, u64 v, bool on) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.u32 p, %2, 0;\n\t"
+        "@p red.relaxed.gpu.global.add.u64 [%0], %1;\n\t}"
+        ::"l"(p), "l"(v), "r"((uint32_t)on) : "memory");
+}
 template <int MT>
-__device__ __forceinline__ void ds_unit_commit(float (&acc)[4], u64* out, const void* res, bool res_plain, int64_t ld, int row0,
+__device__ __forceinline__ void ds_unit_commit(const float (&acc)[4], u64* out, const void* res, bool res_plain, int64_t ld, int row0,
                                                int N, int M, int lane) {
     const int g = lane >> 2, t = lane & 3;
-    auto put = [&](int tok, int row, float v) {
-        if (tok < M && row < N) {
-            const int64_t o = (int64_t)tok * ld + row;
-            u64 w = ds_pack(v);
-            if (res) {
-                if (res_plain) w += ds_pack(__ldcg(reinterpret_cast<const float*>(res) + o)) - 1ull;
-                else w += ds_ld1(reinterpret_cast<const u64*>(res) + o) & ~DS_CNT_MASK;
-            }
-            ds_red_add(out + o, w);
+    auto put = [&](int tok, int row, float v, bool lane_on) {
+        const bool on = lane_on && tok < M && row < N;
+        const int64_t o = (int64_t)tok * ld + row;
+        u64 w = ds_pack(v);
+        if (res != nullptr && on) {
+            if (res_plain) w += ds_pack(__ldcg(reinterpret_cast<const float*>(res) + o)) - 1ull;
+            else w += ds_ld1(reinterpret_cast<const u64*>(res) + o) & ~DS_CNT_MASK;
         }
+        ds_red_add_if(out + o, w, on);
     };
     if constexpr (MT == 1) {
         const float v0 = acc[0] + acc[1], v1 = acc[2] + acc[3];
@@ -395,7 +418,7 @@ __device__ __forceinline__ void ds_unit_commit(float (&acc)[4], u64* out, const 
         const float send = (t & 1) ? v0 : v1;
         keep += __shfl_xor_sync(0xffffffffu, send, 1);
         keep += __shfl_xor_sync(0xffffffffu, keep, 2);
-        if (t < 2) put(0, row0 + g + 8 * t, keep);
+        put(0, row0 + g + 8 * (t & 1), keep, t < 2);
     } else if constexpr (MT == 2) {
         float kA = (t & 1) ? acc[1] : acc[0], kB = (t & 1) ? acc[3] : acc[2];
         const float sA = (t & 1) ? acc[0] : acc[1], sB = (t & 1) ? acc[2] : acc[3];
@@ -404,19 +427,44 @@ __device__ __forceinline__ void ds_unit_commit(float (&acc)[4], u64* out, const 
         float v = (t & 2) ? kB : kA;
         const float s = (t & 2) ? kA : kB;
         v += __shfl_xor_sync(0xffffffffu, s, 2);
-        put(t & 1, row0 + g + 8 * (t >> 1), v);
+        put(t & 1, row0 + g + 8 * (t >> 1), v, true);
     } else if constexpr (MT == 4) {
+        float c[4];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) acc[i] += __shfl_xor_sync(0xffffffffu, acc[i], 2);
+        for (int i = 0; i < 4; ++i) c[i] = acc[i] + __shfl_xor_sync(0xffffffffu, acc[i], 2);
         const int tk = 2 * (t & 1);
         const int hi = t >> 1;
-        put(tk, row0 + g + 8 * hi, hi ? acc[2] : acc[0]);
-        put(tk + 1, row0 + g + 8 * hi, hi ? acc[3] : acc[1]);
+        put(tk, row0 + g + 8 * hi, hi ? c[2] : c[0], true);
+        put(tk + 1, row0 + g + 8 * hi, hi ? c[3] : c[1], true);
     } else {
         const int tk = 2 * t;
-        put(tk, row0 + g, acc[0]); put(tk, row0 + g + 8, acc[2]);
-        put(tk + 1, row0 + g, acc[1]); put(tk + 1, row0 + g + 8, acc[3]);
+        put(tk, row0 + g, acc[0], true); put(tk, row0 + g + 8, acc[2], true);
+        put(tk + 1, row0 + g, acc[1], true); put(tk + 1, row0 + g + 8, acc[3], true);
     }
+}
+
+// A unit whose sums have not left the warp yet: they do at the start of the next unit's arithmetic, where the
+// shuffles, the conversion and the red.add hide behind tensor-core work instead of standing between two units.
+struct DsPending {
+    float acc[4];
+    u64* out;
+    int row0, N;
+    bool on;
+};
+template <int MT>
+__device__ __forceinline__ void ds_flush(DsPending& pd, int M, int lane) {
+    if (pd.on) ds_unit_commit<MT>(pd.acc, pd.out, nullptr, false, pd.N, pd.row0, pd.N, M, lane);   // (pd.on is the same in every lane)
+    pd.on = false;
+}
+
+// One unit: the previous unit's commit, then this unit's multiply-accumulate.
+template <int BITS, int MT, bool BF16>
+__device__ __forceinline__ void ds_unit_body(const uint8_t* unit, const uint8_t* xseg, XOperand<MT>& xo, DsPending& pd, int M, int lane,
+                                             float (&acc)[4]) {
+    ds_load_x_operand<MT, BF16>(xo, xseg, M, lane);
+    const uint32_t xlane = ds_spread_lane_base(xseg, lane);
+    ds_flush<MT>(pd, M, lane);
+    unit_mac<BITS, MT, BF16, MT == 1>(unit, xo, lane, acc, xlane);
 }
 
 // ---- the kernel ---------------------------------------------------------------------
@@ -445,7 +493,7 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArg
     for (int i = threadIdx.x; i < DS_XS_BYTES / 16; i += (int)blockDim.x)
         reinterpret_cast<uint4*>(sh.xs)[i] = make_uint4(0, 0, 0, 0);
     // the copy stream's tables: into shared memory when they fit
-    const int mini_items = a.n_phases + a.n_mini_ops;
+    const int mini_items = a.n_phases + 2 * a.n_mini_ops;   // in 16-byte pieces
     const bool mini_in_smem = mini_items * 16 <= DS_MINI_BYTES;
     if (mini_in_smem)
         for (int i = threadIdx.x; i < mini_items; i += (int)blockDim.x)
@@ -463,6 +511,7 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArg
         // ================= the copy warp: lane w keeps consumer warp w's ring full =================
         DsCursor c;
         c.ph = a.n_phases; c.oi = 0; c.pos = 0; c.base = 0; c.a = 0; c.len = 0; c.frags = nullptr; c.ub = 0;
+        c.NT = 1; c.magic = 0; c.word0 = 0;
         if (lane < DS_WARPS && a.n_phases > 0) {
             c.ph = 0; c.pos = lane;
             ds_cursor_load(c, mp, mo);
@@ -479,9 +528,12 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArg
                 const uint32_t slot = iseq % DS_SLOTS, n = iseq / DS_SLOTS;
                 const bool is_free = (n == 0) || ds_mbar_test(ds_smem(&sh.empty[lane][slot]), (n - 1) & 1u);
                 if (is_free) {
-                    const int u = c.a + (c.pos - c.base);
-                    sh.desc[lane][slot] = make_uint2((uint32_t)c.oi, (uint32_t)u);   // (ordered before the copy's arrival
-                                                                                     // by the release of expect_tx)
+                    const uint32_t u = (uint32_t)(c.a + (c.pos - c.base));
+                    int Pk = c.magic ? (int)__umulhi(u, c.magic) : (int)u;   // u / NT (no magic: NT = 1)
+                    int R = (int)u - Pk * c.NT;
+                    if (R < 0) { --Pk; R += c.NT; }
+                    // (ordered before the copy's arrival by the release of expect_tx)
+                    sh.desc[lane][slot] = make_uint4(c.word0, (uint32_t)Pk, (uint32_t)R, 0u);
                     const uint32_t bar = ds_smem(&sh.full[lane][slot]);
                     ds_expect_tx(bar, (uint32_t)c.ub);
                     ds_bulk_load(ds_smem(&sh.ring[lane][slot][0]), c.frags + (int64_t)u * c.ub, (uint32_t)c.ub, bar, pol);
@@ -505,10 +557,11 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArg
     }
 
     // ================= consumer warps =================
-    auto fetch_record = [&](int q) {
+    auto fetch_record = [&](int q) {   // the phase's record and this CTA's tables for it, on one barrier
         const uint32_t bar = ds_smem(&sh.rec_bar[q & 1]);
-        ds_expect_tx(bar, (uint32_t)sizeof(DsPhase));
+        ds_expect_tx(bar, (uint32_t)(sizeof(DsPhase) + sizeof(DsCtaPhase)));
         ds_bulk_load(ds_smem(&sh.rec[q & 1]), a.phases + q, (uint32_t)sizeof(DsPhase), bar, pol_keep);
+        ds_bulk_load(ds_smem(&sh.ctab[q & 1]), a.ctab + (size_t)q * gridDim.x + blockIdx.x, (uint32_t)sizeof(DsCtaPhase), bar, pol_keep);
     };
     if (threadIdx.x == 0) {
         if (a.n_phases > 0) fetch_record(0);
@@ -518,46 +571,19 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArg
     uint32_t cslot = 0, cparity = 0;   // next ring slot to consume and the parity of its `full` barrier
     bool dead = false;                 // this warp gave up on a wait
     XOperand<MT> xo;
+    DsPending pd;
+    pd.on = false; pd.out = nullptr; pd.row0 = 0; pd.N = 0;
+    pd.acc[0] = pd.acc[1] = pd.acc[2] = pd.acc[3] = 0.f;
 
 #pragma unroll 1
     for (int ph = 0; ph < a.n_phases; ++ph) {
         const int pb = ph & 1;
         const DsPhase& P = sh.rec[pb];
+        const DsCtaPhase& C = sh.ctab[pb];
         // -- the phase's descriptors (fetched one phase ahead) --
         if (!ds_mbar_wait(ds_smem(&sh.rec_bar[pb]), (uint32_t)(ph >> 1) & 1u, wait_ns)) {
             atomicCAS(&g_decode_status, 0, 2);
             sh.abort_flag = 1;
-        }
-        // -- which slabs of the input this CTA's warps will read (independent of the data) --
-        if (threadIdx.x == DS_CTHREADS - 1 && *reinterpret_cast<volatile int*>(&sh.abort_flag) == 0) {
-            int lo[DS_MAX_PHASE_OPS], hi[DS_MAX_PHASE_OPS];
-            int total = 0;
-            for (int oi = 0; oi < P.op_count; ++oi) {
-                int u0, u1;
-                ds_cta_run(P.ops[oi].units_q, P.ops[oi].units_r_rot, u0, u1);
-                total += u1 - u0;
-                lo[oi] = (u0 < u1) ? u0 / P.ops[oi].NT : 0;
-                hi[oi] = (u0 < u1) ? (u1 - 1) / P.ops[oi].NT : -1;
-                sh.seg_slab_lo[pb][oi] = lo[oi];
-            }
-            sh.total[pb] = total;
-            // ascending list of the distinct slabs: repeatedly take the smallest one above the last
-            int n = 0, last = -1;
-            for (;;) {
-                int nxt = 0x7fffffff;
-                for (int oi = 0; oi < P.op_count; ++oi) {
-                    if (hi[oi] > last) nxt = min(nxt, max(lo[oi], last + 1));
-                }
-                if (nxt == 0x7fffffff || n == DS_MAX_SLOTS) break;
-                sh.slab_of_slot[pb][n++] = nxt;
-                last = nxt;
-            }
-            sh.n_slots[pb] = n;
-            for (int oi = 0; oi < P.op_count; ++oi) {
-                int sl = 0;
-                while (sl < n && sh.slab_of_slot[pb][sl] != lo[oi]) ++sl;
-                sh.seg_xoff[pb][oi] = sl - lo[oi];
-            }
         }
         // every warp is through with phase ph - 1: the staged slabs and its record slot are free
         if (ds_consumer_sync_or(*reinterpret_cast<volatile int*>(&sh.abort_flag))) break;
@@ -565,25 +591,32 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArg
 
         // -- form the rounded input vector: slabs this CTA reads -> shared memory, its share -> workspace --
         {
-            const int n_slots = sh.n_slots[pb];
+            const int n_slots = C.n_slots;
             const int q4 = P.K >> 2;                                  // groups of 4 elements per token
             const int g0 = (int)(((int64_t)q4 * blockIdx.x) / gridDim.x), g1 = (int)(((int64_t)q4 * (blockIdx.x + 1)) / gridDim.x);
             uint16_t* stage_out = reinterpret_cast<uint16_t*>(P.stage);
             const uint32_t expect = P.expect, expect2 = P.expect2;
+            uint32_t spins = 0;
+            uint64_t t_wait0 = 0;
+            // after a round of readings that found something incomplete: true when the wait has to end
+            auto give_up = [&]() -> bool {
+                if ((++spins & 7u) != 0) return false;
+                if (*reinterpret_cast<volatile int*>(&g_decode_status) != 0) { sh.abort_flag = 1; return true; }
+                const uint64_t t = ds_now_ns();
+                if (t_wait0 == 0) t_wait0 = t;
+                if (t - t_wait0 > wait_ns) { atomicCAS(&g_decode_status, 0, 1); sh.abort_flag = 1; return true; }
+                return false;
+            };
             // four consecutive source elements (group i4 of token m), complete; zeros after a failed wait
             auto source4 = [&](const u64* p, const float* pf, uint32_t ex, int m, int i4) -> float4 {
                 const int64_t o = (int64_t)m * P.K + 4 * (int64_t)i4;
                 if (p == nullptr) return __ldcg(reinterpret_cast<const float4*>(pf + o));
                 DsQuad q;
-                ds_ld_quad(p + o, q);
-                if (!ds_quad_complete(p + o, q, ex, wait_ns, &sh.abort_flag)) return make_float4(0.f, 0.f, 0.f, 0.f);
-                return ds_quad_value(q);
-            };
-            // the staged copy of slab `slab`, or null when this CTA does not read it
-            auto slot_of = [&](int slab) -> uint8_t* {
-                for (int sl = 0; sl < n_slots; ++sl)
-                    if (sh.slab_of_slot[pb][sl] == slab) return sh.xs + (size_t)sl * slab_bytes;
-                return nullptr;
+                for (;;) {
+                    ds_ld_quad(p + o, q);
+                    if (ds_quad_ready(q, ex)) return ds_quad_value(q);
+                    if (give_up()) return make_float4(0.f, 0.f, 0.f, 0.f);
+                }
             };
             // stores group i4 (elements 4 i4 ..) of token m into slab copy `sl`; whole warps call this together
             auto place = [&](uint8_t* sl, int m, int i4, float4 v, bool rec) {
@@ -604,25 +637,33 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArg
                 if (rec) *reinterpret_cast<uint2*>(stage_out + (int64_t)m * P.K + i4 * 4) = r;
             };
             if (P.in_op == AQ_IN_RMSNORM && MT == 1 && q4 <= DS_RMS_HOLD * DS_CTHREADS) {
-                // one token, row held in registers: one trip to L2 when the row is complete
+                // one token, row held in registers: one trip to L2 once the row is complete (all of a thread's readings
+                // go out together and are repeated together until every one of them is complete)
                 float4 v[DS_RMS_HOLD];
-                uint8_t* dest[DS_RMS_HOLD];
+                int slabs[DS_MAX_SLOTS];
+#pragma unroll
+                for (int x = 0; x < DS_MAX_SLOTS; ++x) slabs[x] = C.slab_of_slot[x];
                 if (P.src != nullptr) {
                     DsQuad q[DS_RMS_HOLD];
+                    for (;;) {
+                        bool ready = true;
 #pragma unroll
-                    for (int n = 0; n < DS_RMS_HOLD; ++n) {
-                        const int i4 = threadIdx.x + n * DS_CTHREADS;
-                        if (i4 < q4) ds_ld_quad(P.src + 4 * (int64_t)i4, q[n]);
-                    }
-#pragma unroll
-                    for (int n = 0; n < DS_RMS_HOLD; ++n) dest[n] = slot_of((threadIdx.x + n * DS_CTHREADS) >> 6);
-#pragma unroll
-                    for (int n = 0; n < DS_RMS_HOLD; ++n) {
-                        const int i4 = threadIdx.x + n * DS_CTHREADS;
-                        v[n] = make_float4(0.f, 0.f, 0.f, 0.f);
-                        if (i4 < q4) {
-                            if (ds_quad_complete(P.src + 4 * (int64_t)i4, q[n], expect, wait_ns, &sh.abort_flag)) v[n] = ds_quad_value(q[n]);
+                        for (int n = 0; n < DS_RMS_HOLD; ++n) {
+                            const int i4 = threadIdx.x + n * DS_CTHREADS;
+                            if (i4 < q4) ds_ld_quad(P.src + 4 * (int64_t)i4, q[n]);
                         }
+#pragma unroll
+                        for (int n = 0; n < DS_RMS_HOLD; ++n) {
+                            const int i4 = threadIdx.x + n * DS_CTHREADS;
+                            if (i4 < q4) ready = ready && ds_quad_ready(q[n], expect);
+                        }
+                        if (ready || give_up()) break;
+                    }
+                    const bool failed = *reinterpret_cast<volatile int*>(&sh.abort_flag) != 0;
+#pragma unroll
+                    for (int n = 0; n < DS_RMS_HOLD; ++n) {
+                        const int i4 = threadIdx.x + n * DS_CTHREADS;
+                        v[n] = (i4 < q4 && !failed) ? ds_quad_value(q[n]) : make_float4(0.f, 0.f, 0.f, 0.f);
                     }
                 } else {
 #pragma unroll
@@ -631,9 +672,8 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArg
                         v[n] = make_float4(0.f, 0.f, 0.f, 0.f);
                         if (i4 < q4) v[n] = __ldcg(reinterpret_cast<const float4*>(P.src_f) + i4);
                     }
-#pragma unroll
-                    for (int n = 0; n < DS_RMS_HOLD; ++n) dest[n] = slot_of((threadIdx.x + n * DS_CTHREADS) >> 6);
                 }
+                __syncwarp();
                 float ss = 0.f;
 #pragma unroll
                 for (int n = 0; n < DS_RMS_HOLD; ++n) {
@@ -654,7 +694,12 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArg
                     if (n * DS_CTHREADS < q4) {   // the same for every thread: warps stay whole
                         const bool mine = i4 >= g0 && i4 < g1;
                         if (mine && P.rec) reinterpret_cast<float4*>(P.rec)[i4] = v[n];
-                        place(dest[n], 0, i4, make_float4(v[n].x * scale, v[n].y * scale, v[n].z * scale, v[n].w * scale), mine);
+                        const int slab = i4 >> 6;
+                        int sl = -1;
+#pragma unroll
+                        for (int x = 0; x < DS_MAX_SLOTS; ++x) sl = (x < n_slots && slabs[x] == slab) ? x : sl;
+                        place(sl >= 0 ? sh.xs + (size_t)sl * slab_bytes : nullptr, 0, i4,
+                              make_float4(v[n].x * scale, v[n].y * scale, v[n].z * scale, v[n].w * scale), mine);
                     }
                 }
             } else {
@@ -665,6 +710,7 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArg
                             const float4 v = source4(P.src, P.src_f, expect, m, i);
                             ss = fmaf(v.x, v.x, ss); ss = fmaf(v.y, v.y, ss); ss = fmaf(v.z, v.z, ss); ss = fmaf(v.w, v.w, ss);
                         }
+                        __syncwarp();
 #pragma unroll
                         for (int d = 16; d > 0; d >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, d);
                         if (lane == 0) sh.red[m][warp] = ss;
@@ -683,6 +729,7 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArg
                 const int n_a = n_slots * per_slab;
                 const int n_b = (g1 - g0) * M;
                 const int n_all = n_a + n_b;
+                const bool two = (P.in_op == AQ_IN_SILU_MUL);
                 for (int it0 = 0; it0 < n_all; it0 += DS_CTHREADS) {
                     const int it = it0 + threadIdx.x;
                     int m = 0, i4 = 0;
@@ -691,7 +738,7 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArg
                     if (it < n_a) {
                         const int s_ = it / per_slab, w = it - s_ * per_slab;
                         m = w >> 6;
-                        i4 = sh.slab_of_slot[pb][s_] * 64 + (w & 63);
+                        i4 = C.slab_of_slot[s_] * 64 + (w & 63);
                         sl = sh.xs + (size_t)s_ * slab_bytes;
                         valid = i4 < q4;
                     } else if (it < n_all) {
@@ -703,17 +750,37 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArg
                     const bool share = it >= n_a;
                     float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
                     if (valid) {
-                        const float4 s = source4(P.src, P.src_f, expect, m, i4);
-                        if (share && P.rec) *reinterpret_cast<float4*>(P.rec + (int64_t)m * P.K + 4 * (int64_t)i4) = s;
-                        if (P.in_op == AQ_IN_SILU_MUL) {
-                            const float4 t = source4(P.src2, P.src2_f, expect2, m, i4);
-                            if (share && P.rec2) *reinterpret_cast<float4*>(P.rec2 + (int64_t)m * P.K + 4 * (int64_t)i4) = t;
+                        // both sources' readings go out together and are repeated together until complete
+                        const int64_t o = (int64_t)m * P.K + 4 * (int64_t)i4;
+                        float4 s = make_float4(0.f, 0.f, 0.f, 0.f), t = s;
+                        DsQuad qa, qb;
+                        for (;;) {
+                            if (P.src) ds_ld_quad(P.src + o, qa);
+                            else s = __ldcg(reinterpret_cast<const float4*>(P.src_f + o));
+                            if (two) {
+                                if (P.src2) ds_ld_quad(P.src2 + o, qb);
+                                else t = __ldcg(reinterpret_cast<const float4*>(P.src2_f + o));
+                            }
+                            bool ready = true;
+                            if (P.src) ready = ds_quad_ready(qa, expect);
+                            if (two && P.src2) ready = ready && ds_quad_ready(qb, expect2);
+                            if (ready) {
+                                if (P.src) s = ds_quad_value(qa);
+                                if (two && P.src2) t = ds_quad_value(qb);
+                                break;
+                            }
+                            if (give_up()) { s = t = make_float4(0.f, 0.f, 0.f, 0.f); break; }
+                        }
+                        if (share && P.rec) *reinterpret_cast<float4*>(P.rec + o) = s;
+                        if (two) {
+                            if (share && P.rec2) *reinterpret_cast<float4*>(P.rec2 + o) = t;
                             v = make_float4(ds_silu_mul(s.x, t.x), ds_silu_mul(s.y, t.y), ds_silu_mul(s.z, t.z), ds_silu_mul(s.w, t.w));
                         } else {
                             const float sc = (P.in_op == AQ_IN_RMSNORM) ? sh.scale[m] : 1.f;
                             v = make_float4(s.x * sc, s.y * sc, s.z * sc, s.w * sc);
                         }
                     }
+                    __syncwarp();
                     if (it0 + (int)(threadIdx.x - lane) < n_a) {
                         place(sl, m, i4, v, false);              // n_a is a multiple of 32: the whole warp is inside the slab items
                     } else if (valid) {
@@ -727,7 +794,7 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArg
         if (ds_consumer_sync_or(*reinterpret_cast<volatile int*>(&sh.abort_flag))) break;
 
         // -- consume this warp's units of the phase: positions warp, warp + 15, ... of the CTA's list --
-        const int total = sh.total[pb];
+        const int total = C.total;
 #pragma unroll 1
         for (int pos = warp; pos < total && !dead; pos += DS_WARPS) {
             dead = __any_sync(0xffffffffu, !ds_mbar_wait(ds_smem(&sh.full[warp][cslot]), cparity, wait_ns));
@@ -735,27 +802,26 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArg
                 if (lane == 0) { atomicCAS(&g_decode_status, 0, 2); sh.abort_flag = 1; }
                 break;
             }
-            const uint2 ds = sh.desc[warp][cslot];
-            const DsOp& op = P.ops[ds.x];
-            const int NT = op.NT;
-            int Pk = op.nt_magic ? (int)__umulhi(ds.y, op.nt_magic) : (int)ds.y;   // (no magic: NT = 1)
-            int R = (int)ds.y - Pk * NT;
-            if (R < 0) { --Pk; R += NT; }
-            const uint8_t* xseg = sh.xs + (size_t)(sh.seg_xoff[pb][ds.x] + Pk) * slab_bytes;
-            ds_load_x_operand<MT, BF16>(xo, xseg, M, lane);
-            const uint32_t xlane = ds_spread_lane_base(xseg, lane);
+            const uint4 ds = sh.desc[warp][cslot];
+            const uint8_t* xseg = sh.xs + (size_t)(C.xoff[ds.x & 0xFFu] + (int)ds.y) * slab_bytes;
             const uint8_t* unit = &sh.ring[warp][cslot][0];
             float acc[4] = {0.f, 0.f, 0.f, 0.f};
-            const int bits = op.bits & 0xFF;
-            const bool res_plain = (op.bits & DS_RES_PLAIN) != 0;
-            if (bits == 2) unit_mac<2, MT, BF16, MT == 1>(unit, xo, lane, acc, xlane);
-            else if (bits == 3) unit_mac<3, MT, BF16, MT == 1>(unit, xo, lane, acc, xlane);
-            else unit_mac<4, MT, BF16, MT == 1>(unit, xo, lane, acc, xlane);
+            const int bits = (int)(ds.x >> DS_DESC_BITS_SHIFT);
+            if (bits == 2) ds_unit_body<2, MT, BF16>(unit, xseg, xo, pd, M, lane, acc);
+            else if (bits == 3) ds_unit_body<3, MT, BF16>(unit, xseg, xo, pd, M, lane, acc);
+            else ds_unit_body<4, MT, BF16>(unit, xseg, xo, pd, M, lane, acc);
             __syncwarp();        // every lane has read its part of the slot
             if (lane == 0) ds_mbar_arrive(ds_smem(&sh.empty[warp][cslot]));
             if (++cslot == DS_SLOTS) { cslot = 0; cparity ^= 1u; }
-            ds_unit_commit<MT>(acc, op.dst, Pk == 0 ? op.res : nullptr, res_plain, op.N, R * 16, op.N, M, lane);
+            const DsOp& op = P.ops[ds.x & 0xFFu];
+            if (ds.y == 0 && op.res != nullptr) {   // (rare: the residual rides along with the first k-slab's sums)
+                ds_unit_commit<MT>(acc, op.dst, op.res, (op.bits & DS_RES_PLAIN) != 0, op.N, (int)ds.z * 16, op.N, M, lane);
+            } else {
+                pd.acc[0] = acc[0]; pd.acc[1] = acc[1]; pd.acc[2] = acc[2]; pd.acc[3] = acc[3];
+                pd.out = op.dst; pd.N = op.N; pd.row0 = (int)ds.z * 16; pd.on = true;
+            }
         }
+        ds_flush<MT>(pd, M, lane);   // nothing of this phase stays behind: other CTAs wait for these sums
     }
 
     // -- buffers no phase reads (and the last outputs): float32 copies for the caller, one chunk per warp --
@@ -783,8 +849,8 @@ namespace {
 struct DecodePlan {
     std::vector<uint8_t> key;
     std::vector<aq_handle_t> handles;
-    uint8_t* dev = nullptr;       // [phase records][mini phases, mini ops][tail chunks]
-    size_t phases_bytes = 0, mini_bytes = 0, tail_bytes = 0;
+    uint8_t* dev = nullptr;       // [phase records][mini phases, mini ops][tail chunks][per-CTA phase tables]
+    size_t phases_bytes = 0, mini_bytes = 0, tail_bytes = 0, ctab_bytes = 0;
     int n_mini_ops = 0;
     int n_phases = 0;
     int n_tails = 0;
@@ -816,10 +882,11 @@ template <typename T> void key_put(std::vector<uint8_t>& k, const T& v) {
 // read the same input vector) and the list of buffers nobody reads.  False when the program
 // does not fit this kernel.
 bool build_decode_tables(const aq_stack_t* p, const StackPlan& plan, int M, int n_cta, uint8_t* ws,
-                         std::vector<DsPhase>& phases, std::vector<DsTail>& tails) {
+                         std::vector<DsPhase>& phases, std::vector<DsTail>& tails, std::vector<DsCtaPhase>& ctab) {
     if (M < 1 || M > AQ_DECODE_MAX_M || p->n_ops > 32000 || plan.pk_off.empty()) return false;
     phases.clear();
     tails.clear();
+    ctab.clear();
     std::vector<int> writer(p->n_bufs, -1);         // op that writes the buffer
     std::vector<char> whole(p->n_bufs, 0);          // every CTA has seen the whole buffer complete (a normalised input)
     std::vector<char> recorded(p->n_bufs, 0);       // some phase writes the caller's float32 copy
@@ -839,6 +906,7 @@ bool build_decode_tables(const aq_stack_t* p, const StackPlan& plan, int M, int 
             const int64_t K = p->buf_width[f.src];
             if (K > (int64_t)1 << 24 || n_cta > 32767) return false;
             DsPhase P;
+            std::vector<DsCtaPhase> ctab_phase;
             int count = std::min(plast - first, DS_MAX_PHASE_OPS), rot_after = rot;
             for (; count >= 1; --count) {
                 memset(&P, 0, sizeof(P));
@@ -857,19 +925,37 @@ bool build_decode_tables(const aq_stack_t* p, const StackPlan& plan, int M, int 
                     r2 = (int)((r2 + nu % n_cta) % n_cta);
                     off += nu;
                 }
+                std::vector<DsCtaPhase> tab(ok ? n_cta : 0);
                 for (int c = 0; c < n_cta && ok; ++c) {
+                    // the slabs CTA c reads for the phase, ascending, and where each op's first slab sits among them
+                    DsCtaPhase& T = tab[c];
+                    memset(&T, 0, sizeof(T));
                     std::vector<int64_t> need;
+                    int64_t lo[DS_MAX_PHASE_OPS];
                     for (int i = 0; i < count; ++i) {
                         const int64_t q = P.ops[i].units_q, r = P.ops[i].units_r_rot & 0xFFFF, ro = P.ops[i].units_r_rot >> 16;
                         const int64_t sl = (c + ro) % n_cta;
                         const int64_t u0 = q * sl + std::min(sl, r), u1 = u0 + q + (sl < r ? 1 : 0);
-                        if (u0 < u1)
+                        T.total += (int32_t)(u1 - u0);
+                        lo[i] = -1;
+                        if (u0 < u1) {
+                            lo[i] = u0 / P.ops[i].NT;
                             for (int64_t x = u0 / P.ops[i].NT; x <= (u1 - 1) / P.ops[i].NT; ++x) need.push_back(x);
+                        }
                     }
                     std::sort(need.begin(), need.end());
-                    const int64_t slabs = std::unique(need.begin(), need.end()) - need.begin();
-                    if (slabs > DS_MAX_SLOTS || slabs * ds_slab_bytes(M) > DS_XS_BYTES) ok = false;
+                    need.erase(std::unique(need.begin(), need.end()), need.end());
+                    const int64_t slabs = (int64_t)need.size();
+                    if (slabs > DS_MAX_SLOTS || slabs * ds_slab_bytes(M) > DS_XS_BYTES) { ok = false; break; }
+                    T.n_slots = (int32_t)slabs;
+                    for (int64_t x = 0; x < slabs; ++x) T.slab_of_slot[x] = (int32_t)need[x];
+                    for (int i = 0; i < count; ++i) {
+                        if (lo[i] < 0) continue;
+                        const int64_t slot = std::lower_bound(need.begin(), need.end(), lo[i]) - need.begin();
+                        T.xoff[i] = (int32_t)(slot - lo[i]);   // (the op's slabs are consecutive, so are their slots)
+                    }
                 }
+                if (ok) ctab_phase = tab;
                 if (ok) { rot_after = r2; break; }
             }
             if (count < 1) return false;
@@ -904,6 +990,7 @@ bool build_decode_tables(const aq_stack_t* p, const StackPlan& plan, int M, int 
             }
             for (int i = first; i < last; ++i) writer[p->ops[i].dst] = i;
             phases.push_back(P);
+            ctab.insert(ctab.end(), ctab_phase.begin(), ctab_phase.end());
             first = last;
         }
     }
@@ -974,7 +1061,8 @@ int launch_decode_stack(const aq_stack_t* p, const StackPlan& plan, int M, aq_dt
         if (capturing) return 1;   // tables are built (allocation, synchronous copies) by an eager call only
         std::vector<DsPhase> phases;
         std::vector<DsTail> tails;
-        if (!build_decode_tables(p, plan, M, grid, ws, phases, tails)) return 1;
+        std::vector<DsCtaPhase> ctab;
+        if (!build_decode_tables(p, plan, M, grid, ws, phases, tails, ctab)) return 1;
         if (g_plans.size() >= MAX_PLANS) {   // make room: the oldest plan no graph refers to
             size_t oldest = g_plans.size();
             for (size_t i = 0; i < g_plans.size(); ++i)
@@ -999,6 +1087,8 @@ int launch_decode_stack(const aq_stack_t* p, const StackPlan& plan, int M, aq_dt
         for (size_t i = 0; i < phases.size(); ++i)
             for (int j = 0; j < phases[i].op_count; ++j) {
                 DsMiniOp mop;
+                memset(&mop, 0, sizeof(mop));
+                mop.NT = phases[i].ops[j].NT; mop.nt_magic = phases[i].ops[j].nt_magic;
                 mop.frags = phases[i].ops[j].frags;
                 mop.q_bits = (uint32_t)phases[i].ops[j].units_q | ((uint32_t)(phases[i].ops[j].bits & 0xFF) << 28);
                 mop.r_rot = (uint32_t)phases[i].ops[j].units_r_rot;
@@ -1009,11 +1099,15 @@ int launch_decode_stack(const aq_stack_t* p, const StackPlan& plan, int M, aq_dt
         dp->tail_bytes = (tails.size() * sizeof(DsTail) + 255) / 256 * 256;
         dp->n_phases = (int)phases.size();
         dp->n_tails = (int)tails.size();
-        cudaError_t e = cudaMalloc(&dp->dev, dp->phases_bytes + dp->mini_bytes + dp->tail_bytes + 256);
+        dp->ctab_bytes = (ctab.size() * sizeof(DsCtaPhase) + 255) / 256 * 256;
+        cudaError_t e = cudaMalloc(&dp->dev, dp->phases_bytes + dp->mini_bytes + dp->tail_bytes + dp->ctab_bytes + 256);
         if (e == cudaSuccess) e = cudaMemcpy(dp->dev, phases.data(), phases.size() * sizeof(DsPhase), cudaMemcpyHostToDevice);
         if (e == cudaSuccess) e = cudaMemcpy(dp->dev + dp->phases_bytes, mini.data(), mini.size(), cudaMemcpyHostToDevice);
         if (e == cudaSuccess && !tails.empty())
             e = cudaMemcpy(dp->dev + dp->phases_bytes + dp->mini_bytes, tails.data(), tails.size() * sizeof(DsTail), cudaMemcpyHostToDevice);
+        if (e == cudaSuccess)
+            e = cudaMemcpy(dp->dev + dp->phases_bytes + dp->mini_bytes + dp->tail_bytes, ctab.data(), ctab.size() * sizeof(DsCtaPhase),
+                           cudaMemcpyHostToDevice);
         if (e != cudaSuccess) { cudaGetLastError(); drop_plan(dp); *err = e; return -1; }
         g_plans.push_back(dp);
     }
@@ -1025,6 +1119,7 @@ int launch_decode_stack(const aq_stack_t* p, const StackPlan& plan, int M, aq_dt
     a.mini_phases = reinterpret_cast<const DsMiniPhase*>(dp->dev + dp->phases_bytes);
     a.mini_ops = reinterpret_cast<const DsMiniOp*>(dp->dev + dp->phases_bytes + (size_t)dp->n_phases * sizeof(DsMiniPhase));
     a.tails = reinterpret_cast<const DsTail*>(dp->dev + dp->phases_bytes + dp->mini_bytes);
+    a.ctab = reinterpret_cast<const DsCtaPhase*>(dp->dev + dp->phases_bytes + dp->mini_bytes + dp->tail_bytes);
     a.n_mini_ops = dp->n_mini_ops;
     a.n_phases = dp->n_phases;
     a.n_tails = dp->n_tails;
