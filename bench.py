@@ -229,6 +229,7 @@ def run_micro(args):
             fn = lambda i: aq.aq_linear(hs[i % n_copies], x, y)
             work, unit = (N * K * (args.bits + 1) / 8, "GB/s") if decode else (2.0 * M * N * K, "TFLOP/s")
         out.update({"M": M, "N": N, "K": K, "copies": n_copies})
+        args.warmup = max(args.warmup, n_copies)   # every copy's handle has sized its scratch before the clock starts
     else:
         decode = args.micro == "decode_stack"
         M = args.M or (1 if decode else 512)

@@ -188,10 +188,13 @@ aq_status_t aq_dequant(aq_handle_t h, void* out_dev, aq_dtype_t out_dtype, aq_st
  *   M     : 1 .. AQ_MAX_M.  M <= AQ_DECODE_MAX_M runs the weight-streaming
  *           kernel, larger M the tensor-core GEMM.
  * Accumulation is binary32.  Error against the exact product, per output, with T = sum_k |x_k w_hat_k|: the
- * weight-streaming kernel multiplies exact codes (about K 2^-24 T); the GEMM rounds each dequantised weight to the
- * activation type before the tensor core, so at most 2^-11 T for AQ_F16 and 2^-8 T for AQ_BF16 (8 significant bits;
- * with signs at random about 2^-8 T / sqrt(3 K)).  Calls on one handle must be ordered on a stream
- * (the handle owns accumulation scratch that concurrent calls would share).
+ * weight-streaming kernel multiplies exact codes (about K 2^-24 T); the GEMM rounds each dequantised weight to
+ * binary16 before the tensor core, so at most 2^-11 T for either activation type (bfloat16 activations are widened
+ * to binary16 first, which is exact inside binary16's range; a token row with a magnitude of 2^15 or more is scaled
+ * by a power of two and scaled back after the sum).  Calls on one handle must be ordered on a stream (the handle
+ * owns accumulation scratch that concurrent calls would share).  With M > AQ_DECODE_MAX_M the handle allocates
+ * further scratch (float32 sums, the widened activations) the first time it sees such a call and again when a
+ * later call needs more; calls in between allocate nothing.
  */
 aq_status_t aq_linear(aq_handle_t h, const void* x_dev, void* y_dev, int M,
                       aq_dtype_t xy_dtype, aq_stream_t stream);

@@ -71,6 +71,7 @@ static aq_status_t new_handle(int bits, int block, int64_t N, int64_t K, aq_hand
     h->n_frags = (int64_t)h->NT * h->KP * 2;
     h->dev_bytes = (size_t)h->n_frags * frag_bytes(bits);
     h->frags = nullptr; h->acc = nullptr; h->flags = nullptr; h->last_stream = nullptr;
+    h->big = nullptr; h->big_bytes = 0;
     const size_t acc_bytes = (size_t)AQ_DECODE_MAX_M * h->NT * 16 * sizeof(float);
     if (cudaMalloc(&h->frags, h->dev_bytes) != cudaSuccess || cudaMalloc(&h->acc, acc_bytes) != cudaSuccess ||
         cudaMalloc(&h->flags, 256) != cudaSuccess) {
@@ -84,7 +85,7 @@ static aq_status_t new_handle(int bits, int block, int64_t N, int64_t K, aq_hand
 }
 
 static void destroy(aq_handle_s* h) {
-    cudaFree(h->frags); cudaFree(h->acc); cudaFree(h->flags);
+    cudaFree(h->frags); cudaFree(h->acc); cudaFree(h->flags); cudaFree(h->big);
     h->magic = 0;
     delete h;
 }
@@ -218,15 +219,34 @@ static aq_status_t linear_common(aq_handle_t h, const void* x_dev, void* y_dev, 
             e = launch_gemv(h, x_dev, xdt, M, h->acc, ld, s);
             if (e == cudaSuccess) e = launch_finalize(h->acc, h->acc, ld, y_dev, ydt, M, h->N, s);
         }
-    } else if (ydt == AQ_F32) {
-        e = launch_gemm(h, x_dev, xdt, M, (float*)y_dev, h->N, nullptr, s);
     } else {
-        float* tmp = nullptr;
-        e = cudaMallocAsync(&tmp, (size_t)M * h->N * sizeof(float), s);
-        if (e != cudaSuccess) { cudaGetLastError(); return AQ_ERR_ALLOC; }
-        e = launch_gemm(h, x_dev, xdt, M, tmp, h->N, nullptr, s);
-        if (e == cudaSuccess) e = launch_finalize(tmp, nullptr, h->N, y_dev, ydt, M, h->N, s);
-        cudaFreeAsync(tmp, s);
+        // scratch owned by the handle: float32 sums when the output is half precision, the binary16 copy of bfloat16
+        // activations with its row scales and flag; allocated on the first such call and when a later one needs more
+        auto up = [](size_t v) { return (v + 255) / 256 * 256; };
+        const size_t out_bytes = (ydt == AQ_F32) ? 0 : up((size_t)M * h->N * sizeof(float));
+        const size_t x16_bytes = (xdt == AQ_BF16) ? up((size_t)M * h->K * 2) : 0;
+        const size_t rs_bytes = (xdt == AQ_BF16) ? up((size_t)M * sizeof(float) + 16) : 0;
+        const size_t need = out_bytes + x16_bytes + rs_bytes;
+        if (need > h->big_bytes) {
+            cudaFree(h->big);   // (waits for whatever still uses the old one)
+            h->big = nullptr; h->big_bytes = 0;
+            if (cudaMalloc(&h->big, need) != cudaSuccess) { cudaGetLastError(); return AQ_ERR_ALLOC; }
+            h->big_bytes = need;
+        }
+        float* sums = (ydt == AQ_F32) ? (float*)y_dev : reinterpret_cast<float*>(h->big);
+        const void* xop = x_dev;
+        const float* rs = nullptr;
+        const int* flag = nullptr;
+        e = cudaSuccess;
+        if (xdt == AQ_BF16) {
+            void* x16 = h->big + out_bytes;
+            float* rsw = reinterpret_cast<float*>(h->big + out_bytes + x16_bytes);
+            int* fw = reinterpret_cast<int*>(h->big + out_bytes + x16_bytes + (size_t)M * sizeof(float));
+            e = launch_rows_to_f16(x_dev, x16, rsw, fw, M, h->K, s);
+            xop = x16; rs = rsw; flag = fw;
+        }
+        if (e == cudaSuccess) e = launch_gemm(h, xop, rs, flag, M, sums, h->N, nullptr, s);
+        if (e == cudaSuccess && ydt != AQ_F32) e = launch_finalize(sums, nullptr, h->N, y_dev, ydt, M, h->N, s);
     }
     if (e != cudaSuccess) return cuda_fail(e);
     h->last_stream = s;

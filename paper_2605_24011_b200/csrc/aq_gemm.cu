@@ -2,6 +2,13 @@
 // weights, out[m][n] = (res[m][n]) + sum_k x[m][k] w_hat[n][k]  (Appendix D:
 // dequantise on the fly inside the low-bit kernel; Eq. 1 for the decode).
 //
+// Both operands enter the tensor core as binary16: a dequantised weight is
+// fp16(scale * q + min) (one half-precision FMA, 11 significant bits, so the
+// worst case of the product sum is 2^-11 sum|x w|).  bfloat16 activations are
+// widened to binary16 by the caller of this kernel (exact wherever the value is
+// inside binary16's range; a token row that is not comes scaled by a power of
+// two, undone in the epilogue through tok_scale).
+//
 // Bound: tensor cores (dense contraction, 2 M flops per weight).  tcgen05
 // UMMA with the accumulators in TMEM:
 //   A (M side, 128)   = weight rows, dequantised by eight warps from the packed
@@ -78,6 +85,8 @@ struct GemmArgs {
     int store_first;       // 1: split tiles of matrices without a residual use the store-then-add protocol above
     int flag_slot;
     uint32_t epoch;
+    const float* tok_scale;    // per token: the power of two its row of x was divided by, or null
+    const int* scaled_flag;    // nonzero when some entry of tok_scale is not 1 (null: none is)
 };
 
 struct GemmOutMaps { CUtensorMap m[GM_MAX_OPS]; };
@@ -133,43 +142,22 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     return false;
 }
 
-template <bool BF16>
-__device__ __forceinline__ uint32_t pack2(float a, float b) {
-    if constexpr (BF16) {
-        __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
-        return *reinterpret_cast<uint32_t*>(&v);
-    } else {
-        __half2 v = __floats2half2_rn(a, b);
-        return *reinterpret_cast<uint32_t*>(&v);
-    }
-}
-
-// Two dequantised weights (k-adjacent, one row) as the 32-bit A-tile element.
-// p holds the two codes OR-ed into the mantissa of the half-precision constant
-// 128.0 (bf16) or 1024.0 (fp16) in each half.
-//   bf16: widen each half to fp32 (a shift / a mask), one FMA with the scale and
-//         with (min - 128 scale), round the pair to bf16;
-//   fp16: subtract 1024 (exact), one half2 FMA with scale and min.
-template <bool BF16>
-__device__ __forceinline__ uint32_t dequant_pair(uint32_t p, float d, float mb, __half2 d2, __half2 m2) {
-    if constexpr (BF16) {
-        const float f0 = __uint_as_float(p << 16), f1 = __uint_as_float(p & 0xffff0000u);
-        return pack2<true>(fmaf(f0, d, mb), fmaf(f1, d, mb));
-    } else {
-        const __half2 q = __hsub2(*reinterpret_cast<const __half2*>(&p), __float2half2_rn(1024.f));
-        const __half2 w = __hfma2(q, d2, m2);
-        return *reinterpret_cast<const uint32_t*>(&w);
-    }
+// Two dequantised weights (k-adjacent, one row) as the 32-bit A-tile element.  p holds the two codes OR-ed into
+// the mantissa of the binary16 constant 1024.0 in each half: subtract 1024 (exact), one half2 FMA with scale and min.
+__device__ __forceinline__ uint32_t dequant_pair(uint32_t p, __half2 d2, __half2 m2) {
+    const __half2 q = __hsub2(*reinterpret_cast<const __half2*>(&p), __float2half2_rn(1024.f));
+    const __half2 w = __hfma2(q, d2, m2);
+    return *reinterpret_cast<const uint32_t*>(&w);
 }
 
 // One dequantise warp's share of a k-slab: its fragment (16 rows x 128 k) becomes
 // rows 16 dw .. 16 dw + 15 of two A stages.  `have` is false for row tiles past the
 // end of the matrix (zeros are written).  Returns false when a wait ran out.
-template <int BITS, bool BF16>
+template <int BITS>
 __device__ __forceinline__ bool dequant_slab(const uint8_t* slab, bool have, int dw, int lane, uint8_t* sA, uint32_t bar_pempty_slot,
                                              uint32_t bar_aempty, uint32_t bar_afull, uint32_t& ai, volatile int* abort_flag) {
     constexpr int FB = frag_bytes(BITS);
-    constexpr uint32_t MAGIC = BF16 ? 0x43004300u : 0x64006400u;
+    constexpr uint32_t MAGIC = 0x64006400u;
     const int g = lane >> 2, t = lane & 3;
     LaneCodes<BITS> lc;
     uint32_t dmw[2][4];   // [row half][block]: half2 (scale, min)
@@ -202,12 +190,10 @@ __device__ __forceinline__ bool dequant_slab(const uint8_t* slab, bool have, int
 #pragma unroll
             for (int hi = 0; hi < 2; ++hi) {
                 const __half2 dm = *reinterpret_cast<const __half2*>(&dmw[hi][j]);
-                const float d = __low2float(dm);
-                const float mb = fmaf(-128.f, d, __high2float(dm));
                 const __half2 d2 = __low2half2(dm), m2 = __high2half2(dm);
                 uint32_t o[4];
 #pragma unroll
-                for (int i = 0; i < 4; ++i) o[i] = dequant_pair<BF16>(code_pair<BITS>(lc, j, hi, i, MAGIC), d, mb, d2, m2);
+                for (int i = 0; i < 4; ++i) o[i] = dequant_pair(code_pair<BITS>(lc, j, hi, i, MAGIC), d2, m2);
                 const int row = dw * 16 + g + 8 * hi;
                 const int chunk = (jj * 4 + t) ^ (row & 7);
                 *reinterpret_cast<uint4*>(At + (row >> 3) * 1024 + (row & 7) * 128 + chunk * 16) = make_uint4(o[0], o[1], o[2], o[3]);
@@ -220,7 +206,6 @@ __device__ __forceinline__ bool dequant_slab(const uint8_t* slab, bool have, int
     return true;
 }
 
-template <bool BF16>
 __global__ void __launch_bounds__(GM_THREADS, 1) gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ GemmOutMaps tmap_out, const GemmArgs a) {
     constexpr int P_BYTES = 8 * frag_bytes(4);                // packed fragments of one slab (largest width)
     extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -317,8 +302,7 @@ __global__ void __launch_bounds__(GM_THREADS, 1) gemm_kernel(const __grid_consta
                 uint32_t idesc[2];
                 for (int j = 0; j < 2; ++j) {
                     const uint32_t w = (j == 0) ? sg.w0 : sg.w1;
-                    idesc[j] = (1u << 4) | ((BF16 ? 1u : 0u) << 7) | ((BF16 ? 1u : 0u) << 10) | ((w >> 3) << 17) |
-                               ((uint32_t)(GM_ROWS >> 4) << 24);
+                    idesc[j] = (1u << 4) | ((w >> 3) << 17) | ((uint32_t)(GM_ROWS >> 4) << 24);   // f16 x f16 -> f32
                 }
                 for (int it = 2 * sg.s0; it < 2 * sg.s1 && ok; ++it) {
                     const uint32_t as = ai % GM_ASTAGES;
@@ -359,9 +343,9 @@ __global__ void __launch_bounds__(GM_THREADS, 1) gemm_kernel(const __grid_consta
                 if (!ok) break;
                 ++pi;
                 const uint8_t* slab = sP + ps * P_BYTES;
-                if (op.bits == 2) ok = dequant_slab<2, BF16>(slab, dw < n_rt, dw, lane, sA, bar_pempty + 8 * ps, bar_aempty, bar_afull, ai, abort_flag);
-                else if (op.bits == 3) ok = dequant_slab<3, BF16>(slab, dw < n_rt, dw, lane, sA, bar_pempty + 8 * ps, bar_aempty, bar_afull, ai, abort_flag);
-                else ok = dequant_slab<4, BF16>(slab, dw < n_rt, dw, lane, sA, bar_pempty + 8 * ps, bar_aempty, bar_afull, ai, abort_flag);
+                if (op.bits == 2) ok = dequant_slab<2>(slab, dw < n_rt, dw, lane, sA, bar_pempty + 8 * ps, bar_aempty, bar_afull, ai, abort_flag);
+                else if (op.bits == 3) ok = dequant_slab<3>(slab, dw < n_rt, dw, lane, sA, bar_pempty + 8 * ps, bar_aempty, bar_afull, ai, abort_flag);
+                else ok = dequant_slab<4>(slab, dw < n_rt, dw, lane, sA, bar_pempty + 8 * ps, bar_aempty, bar_afull, ai, abort_flag);
             }
             // epilogue: TMEM lane quarter (warp % 4) x this warp group's columns -> out[token][row]
             if (ok) ok = mbar_wait(bar_accum, segc & 1, abort_flag, 7);
@@ -400,6 +384,8 @@ __global__ void __launch_bounds__(GM_THREADS, 1) gemm_kernel(const __grid_consta
                 const int n0 = sg.rt * GM_ROWS + lq * 32;
                 const int64_t n = (int64_t)n0 + lane;
                 const int tok0 = sg.st * a.st_tokens + acc * GM_MAX_TN;
+                // token rows whose input was divided by a power of two get it back here (rare: a flag says whether any)
+                const bool scaled = a.scaled_flag != nullptr && __ldcg(a.scaled_flag) != 0;
                 if (a.tma_out) {
                     // the A ring is idle now (every MMA of the run has completed): two 4 KB chunks per warp
                     float* stg = reinterpret_cast<float*>(sA + dw * 8192);
@@ -411,6 +397,11 @@ __global__ void __launch_bounds__(GM_THREADS, 1) gemm_kernel(const __grid_consta
                         if (lane == 0) bulk_wait_read<1>();   // the copy that last read this chunk has left shared memory
                         __syncwarp();
                         float* chunk = stg + buf * 1024;      // [32 tokens][32 rows]
+                        if (scaled) {
+                            const float sc = __ldcg(a.tok_scale + min(tok0 + c0 + lane, a.M - 1));
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) * __shfl_sync(0xffffffffu, sc, j));
+                        }
 #pragma unroll
                         for (int j = 0; j < 32; ++j) chunk[j * 32 + lane] = __uint_as_float(v[j]);
                         fence_async_smem();
@@ -438,6 +429,7 @@ __global__ void __launch_bounds__(GM_THREADS, 1) gemm_kernel(const __grid_consta
                                 if (c0 + j < c_hi && tok < a.M) {
                                     const int64_t o = (int64_t)tok * op.ldo + n;
                                     float val = __uint_as_float(v[j]);
+                                    if (scaled) val *= __ldcg(a.tok_scale + tok);
                                     if (add_res) val += __ldg(op.res + o);
                                     if (whole) op.out[o] = val;
                                     else atomicAdd(op.out + o, val);
@@ -478,10 +470,9 @@ EncodeTiledFn tensor_map_encoder() {
     return fn;
 }
 
-template <bool BF16>
 static cudaError_t launch_one(const CUtensorMap& tm, const GemmOutMaps& tmo, const GemmArgs& a, int grid, cudaStream_t s) {
     constexpr int SMEM = 1024 + GM_ASTAGES * GM_A_BYTES + GM_BSLOTS * GM_B_BYTES + GM_PSTAGES * 8 * frag_bytes(4) + 256;
-    auto kern = gemm_kernel<BF16>;
+    auto kern = gemm_kernel;
     static PerDeviceOnce configured;
     {
         const int rc = configured.run(current_device(), [&] {
@@ -498,13 +489,15 @@ bool gemm_stores_first(const aq_handle_s* const* hs, int n, int M, cudaStream_t 
 
 // n (<= GM_MAX_OPS) matrices with the same K against one x: out[i] = (res[i]) + x W_i^T.
 // outs_ready: the caller has already put the residual (or zeros) into every output.
-cudaError_t launch_gemm_group(const aq_handle_s* const* hs, int n, const void* x, aq_dtype_t xdt, int M, float* const* outs,
-                              const int64_t* ldos, const float* const* ress, bool outs_ready, cudaStream_t s) {
+cudaError_t launch_gemm_group(const aq_handle_s* const* hs, int n, const void* x16, const float* tok_scale, const int* scaled_flag,
+                              int M, float* const* outs, const int64_t* ldos, const float* const* ress, bool outs_ready,
+                              cudaStream_t s) {
     EncodeTiledFn enc = tensor_map_encoder();
     if (!enc || n < 1 || n > GM_MAX_OPS) return cudaErrorNotSupported;
     GemmArgs a;
     memset(&a, 0, sizeof(a));
     a.n_ops = n; a.M = M; a.n_slabs = hs[0]->KP * 2;
+    a.tok_scale = tok_scale; a.scaled_flag = tok_scale ? scaled_flag : nullptr;
     for (int i = 0; i < n; ++i) {
         if (hs[i]->K != hs[0]->K) return cudaErrorInvalidValue;
         GemmOp& o = a.op[i];
@@ -527,8 +520,7 @@ cudaError_t launch_gemm_group(const aq_handle_s* const* hs, int n, const void* x
     const cuuint64_t strides[1] = {(cuuint64_t)hs[0]->K * 2};
     const cuuint32_t box[2] = {(cuuint32_t)GM_KSTAGE, (cuuint32_t)a.tn};
     const cuuint32_t estr[2] = {1, 1};
-    const CUresult r = enc(&tm, xdt == AQ_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2,
-                           const_cast<void*>(x), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+    const CUresult r = enc(&tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(x16), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
@@ -574,12 +566,76 @@ cudaError_t launch_gemm_group(const aq_handle_s* const* hs, int n, const void* x
             e = cudaMemset2DAsync(o.out, (size_t)o.ldo * sizeof(float), 0, (size_t)o.N * sizeof(float), (size_t)M, s);
         if (e != cudaSuccess) return e;
     }
-    return (xdt == AQ_BF16) ? launch_one<true>(tm, tmo, a, grid, s) : launch_one<false>(tm, tmo, a, grid, s);
+    return launch_one(tm, tmo, a, grid, s);
 }
 
-cudaError_t launch_gemm(const aq_handle_s* h, const void* x, aq_dtype_t xdt, int M, float* out, int64_t ldo,
-                        const float* res, cudaStream_t s) {
-    return launch_gemm_group(&h, 1, x, xdt, M, &out, &ldo, &res, false, s);
+cudaError_t launch_gemm(const aq_handle_s* h, const void* x16, const float* tok_scale, const int* scaled_flag, int M, float* out,
+                        int64_t ldo, const float* res, cudaStream_t s) {
+    return launch_gemm_group(&h, 1, x16, tok_scale, scaled_flag, M, &out, &ldo, &res, false, s);
+}
+
+// ---- bfloat16 activations -> binary16 operand ---------------------------------------------------------------
+// One CTA per token row.  A bfloat16 value has 8 significant bits, so it is a binary16 value whenever it is inside
+// binary16's range (magnitudes below 2^-17 land on the subnormal grid, an absolute error below 2^-25).  A row that
+// holds a magnitude of 2^15 or more is divided by the power of two that brings its largest one below 2^15 (exact for
+// everything that stays normal); scale[m] is that power of two, 1 otherwise, and *flag is raised when any row has one.
+__global__ void __launch_bounds__(256) rows_to_f16_kernel(const __nv_bfloat16* __restrict__ x, __half* __restrict__ x16,
+                                                          float* __restrict__ scale, int* __restrict__ flag, int64_t K) {
+    const int64_t m = blockIdx.x;
+    const __nv_bfloat16* xr = x + m * K;
+    __half* o = x16 + m * K;
+    float mx = 0.f;
+    for (int64_t k = threadIdx.x * 8; k < K; k += 256 * 8) {   // K is a multiple of 32
+        const uint4 v = *reinterpret_cast<const uint4*>(xr + k);
+        const __nv_bfloat162* b = reinterpret_cast<const __nv_bfloat162*>(&v);
+        uint4 r;
+        __half2* h = reinterpret_cast<__half2*>(&r);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float2 f = __bfloat1622float2(b[i]);
+            h[i] = __floats2half2_rn(f.x, f.y);
+            mx = fmaxf(mx, fmaxf(fabsf(f.x), fabsf(f.y)));
+        }
+        *reinterpret_cast<uint4*>(o + k) = r;
+    }
+    __shared__ float red[8];
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, d));
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = mx;
+    __syncthreads();
+    mx = red[0];
+#pragma unroll
+    for (int i = 1; i < 8; ++i) mx = fmaxf(mx, red[i]);
+    float sc = 1.f;
+    if (mx >= 32768.f && mx <= 3.0e38f) {   // (non-finite input stays non-finite: nothing to rescue)
+        int e;
+        frexpf(mx, &e);                       // mx = f 2^e, f in [0.5, 1)
+        sc = ldexpf(1.f, e - 15);             // mx / sc in [2^14, 2^15)
+        const float inv = 1.f / sc;
+        for (int64_t k = threadIdx.x * 8; k < K; k += 256 * 8) {
+            const uint4 v = *reinterpret_cast<const uint4*>(xr + k);
+            const __nv_bfloat162* b = reinterpret_cast<const __nv_bfloat162*>(&v);
+            uint4 r;
+            __half2* h = reinterpret_cast<__half2*>(&r);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float2 f = __bfloat1622float2(b[i]);
+                h[i] = __floats2half2_rn(f.x * inv, f.y * inv);
+            }
+            *reinterpret_cast<uint4*>(o + k) = r;
+        }
+        if (threadIdx.x == 0) *flag = 1;
+    }
+    if (threadIdx.x == 0) scale[m] = sc;
+}
+
+cudaError_t launch_rows_to_f16(const void* x_bf16, void* x16, float* scale, int* flag, int M, int64_t K, cudaStream_t s) {
+    cudaError_t e = cudaMemsetAsync(flag, 0, sizeof(int), s);
+    if (e != cudaSuccess) return e;
+    rows_to_f16_kernel<<<(unsigned)M, 256, 0, s>>>(reinterpret_cast<const __nv_bfloat16*>(x_bf16), reinterpret_cast<__half*>(x16), scale,
+                                                   flag, K);
+    count_launch();
+    return cudaGetLastError();
 }
 
 // True when outputs without a residual need no zeroing before launch_gemm_group (split tiles store first).

@@ -21,6 +21,9 @@ struct aq_handle_s {
     size_t dev_bytes;  // n_frags * frag_bytes
     uint8_t* frags;    // DEVICE: fragment layout
     float* acc;        // DEVICE: [AQ_DECODE_MAX_M][NT*16] accumulation scratch, zero between calls
+    uint8_t* big;      // DEVICE: scratch of aq_linear with M > AQ_DECODE_MAX_M (float32 sums, binary16 copy of bfloat16
+                       // activations, row scales), allocated when the handle first sees such a call and grown on demand
+    size_t big_bytes;
     int* flags;        // DEVICE: bit 0 = range error seen while packing
     cudaStream_t last_stream;
 };
@@ -46,14 +49,18 @@ cudaError_t launch_gemv(const aq_handle_s* h, const void* x, aq_dtype_t xdt, int
 cudaError_t launch_finalize(const float* acc_in, float* acc_zero, int64_t ldacc, void* y, aq_dtype_t ydt,
                             int M, int64_t N, cudaStream_t s);
 
-// prefill path: out[m][n] = (res ? res[m][n] : 0) + sum_k x[m][k] w[n][k]; out, res fp32 [M][ldo];
+// prefill path: out[m][n] = (res ? res[m][n] : 0) + tok_scale[m] sum_k x16[m][k] w[n][k]; x16 binary16 [M][K];
+// tok_scale (with its flag, see launch_rows_to_f16) or null; out, res fp32 [M][ldo];
 // out need not be initialised (the launcher zeroes it when tiles are split over CTAs)
-cudaError_t launch_gemm(const aq_handle_s* h, const void* x, aq_dtype_t xdt, int M, float* out,
+cudaError_t launch_gemm(const aq_handle_s* h, const void* x16, const float* tok_scale, const int* scaled_flag, int M, float* out,
                         int64_t ldo, const float* res, cudaStream_t s);
+// bfloat16 rows -> the binary16 operand of the GEMM, the per-row power of two they were divided by (1 unless a row
+// leaves binary16's range) and a flag that says whether any row has one
+cudaError_t launch_rows_to_f16(const void* x_bf16, void* x16, float* scale, int* flag, int M, int64_t K, cudaStream_t s);
 // the same for up to AQ_GEMM_MAX_GROUP matrices of one K that read the same x, as one launch
 #define AQ_GEMM_MAX_GROUP 4
-cudaError_t launch_gemm_group(const aq_handle_s* const* hs, int n, const void* x, aq_dtype_t xdt, int M,
-                              float* const* outs, const int64_t* ldos, const float* const* ress, bool outs_ready,
+cudaError_t launch_gemm_group(const aq_handle_s* const* hs, int n, const void* x16, const float* tok_scale, const int* scaled_flag,
+                              int M, float* const* outs, const int64_t* ldos, const float* const* ress, bool outs_ready,
                               cudaStream_t s);
 bool gemm_outputs_can_be_preset(float* const* outs, const int64_t* ldos, int n);
 bool gemm_stores_first(const aq_handle_s* const* hs, int n, int M, cudaStream_t s);   // then only residuals need presetting
@@ -65,6 +72,8 @@ struct StackPlan {
     std::vector<int> phase_first;   // first op of each phase (ops that share one input vector)
     std::vector<size_t> pk_off;     // per buffer (M <= AQ_DECODE_MAX_M only): its packed 64-bit sums [M][width]
     size_t pk_begin = 0, pk_end = 0;   // the packed sums' region: zero at the start of a decode pass
+    std::vector<size_t> x16_off;    // per op (bfloat16, M > AQ_DECODE_MAX_M only): its phase's binary16 operand [M][K] ...
+    std::vector<size_t> rs_off;     // ... and the row scales [M] float32, followed by the flag (int)
     size_t stage_off = 0;           // end of the float32 buffers
     size_t total = 0;
 };

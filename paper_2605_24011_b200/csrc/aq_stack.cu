@@ -58,6 +58,17 @@ static bool plan_stack(const aq_stack_t* p, int M, StackPlan& plan) {
         plan.in_off[i] = off;
         off += align_up((size_t)M * p->buf_width[p->ops[i].src] * 2, 256);
     }
+    if (M > AQ_DECODE_MAX_M) {   // bfloat16 activations reach the tensor cores as binary16: a second staged vector per phase
+        plan.x16_off.assign(p->n_ops, 0);
+        plan.rs_off.assign(p->n_ops, 0);
+        for (int i = 0; i < p->n_ops; ++i) {
+            if (i > 0 && same_input(p->ops[i], p->ops[i - 1])) { plan.x16_off[i] = plan.x16_off[i - 1]; plan.rs_off[i] = plan.rs_off[i - 1]; continue; }
+            plan.x16_off[i] = off;
+            off += align_up((size_t)M * p->buf_width[p->ops[i].src] * 2, 256);
+            plan.rs_off[i] = off;
+            off += align_up((size_t)M * sizeof(float) + 16, 256);
+        }
+    }
     if (M <= AQ_DECODE_MAX_M) {   // the whole-program decode kernel accumulates packed 64-bit sums, one per element
         plan.pk_off.assign(p->n_bufs, 0);
         plan.pk_begin = off;
@@ -163,6 +174,95 @@ __global__ void __launch_bounds__(256) stage_kernel(const float* __restrict__ sr
     }
 }
 
+// The same for bfloat16 activations on the tensor-core path, one CTA per token row: besides the rounded vector x
+// (kept for the caller) it writes the binary16 copy x16 the GEMM reads -- exact wherever a bfloat16 value lies
+// inside binary16's range; a row with a magnitude of 2^15 or more is divided by the power of two that brings its
+// largest one below 2^15, kept in scale[m] (1 otherwise) and undone by the GEMM's epilogue; *flag is raised then.
+// The flag must be zero when the kernel starts.
+__global__ void __launch_bounds__(256) stage_rows_bf16_kernel(const float* __restrict__ src, const float* __restrict__ src2, int in_op,
+                                                              int64_t K, __nv_bfloat16* __restrict__ x, __half* __restrict__ x16,
+                                                              float* __restrict__ scale, int* __restrict__ flag, const PresetList pre) {
+    pdl_wait();
+    pdl_launch_dependents();
+    for (int q = 0; q < pre.n; ++q) {
+        float4* d = pre.dst[q];
+        const float4* r = pre.src[q];
+        for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < pre.n4[q]; i += (int64_t)gridDim.x * 256)
+            d[i] = r ? r[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    const int64_t m = blockIdx.x;
+    const float4* s4 = reinterpret_cast<const float4*>(src + m * K);
+    const float4* t4 = src2 ? reinterpret_cast<const float4*>(src2 + m * K) : nullptr;
+    __nv_bfloat16* xr = x + m * K;
+    __half* hr = x16 + m * K;
+    const int64_t q4 = K >> 2;
+    __shared__ float red[8];
+    float rms = 1.f;
+    if (in_op == AQ_IN_RMSNORM) {
+        float ss = 0.f;
+        for (int64_t k = threadIdx.x; k < q4; k += 256) {
+            const float4 v = s4[k];
+            ss = fmaf(v.x, v.x, ss); ss = fmaf(v.y, v.y, ss); ss = fmaf(v.z, v.z, ss); ss = fmaf(v.w, v.w, ss);
+        }
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, d);
+        if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+        __syncthreads();
+        float tot = 0.f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) tot += red[i];
+        rms = rsqrtf(tot / (float)K + 1e-6f);
+        __syncthreads();
+    }
+    // the rounded vector, its binary16 copy as if no scaling were needed, and the row's largest magnitude
+    float mx = 0.f;
+    for (int64_t k = threadIdx.x; k < q4; k += 256) {
+        float4 v = s4[k];
+        if (in_op == AQ_IN_SILU_MUL) {
+            const float4 u = t4[k];
+            v.x = v.x / (1.f + expf(-v.x)) * u.x; v.y = v.y / (1.f + expf(-v.y)) * u.y;
+            v.z = v.z / (1.f + expf(-v.z)) * u.z; v.w = v.w / (1.f + expf(-v.w)) * u.w;
+        } else {
+            v.x *= rms; v.y *= rms; v.z *= rms; v.w *= rms;
+        }
+        const __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y), b = __floats2bfloat162_rn(v.z, v.w);
+        uint2 r;
+        r.x = *reinterpret_cast<const uint32_t*>(&a); r.y = *reinterpret_cast<const uint32_t*>(&b);
+        *reinterpret_cast<uint2*>(xr + 4 * k) = r;
+        const float2 fa = __bfloat1622float2(a), fb = __bfloat1622float2(b);
+        const __half2 ha = __floats2half2_rn(fa.x, fa.y), hb = __floats2half2_rn(fb.x, fb.y);
+        uint2 h;
+        h.x = *reinterpret_cast<const uint32_t*>(&ha); h.y = *reinterpret_cast<const uint32_t*>(&hb);
+        *reinterpret_cast<uint2*>(hr + 4 * k) = h;
+        mx = fmaxf(mx, fmaxf(fmaxf(fabsf(fa.x), fabsf(fa.y)), fmaxf(fabsf(fb.x), fabsf(fb.y))));
+    }
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, d));
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = mx;
+    __syncthreads();   // (also: this CTA's writes of x are visible to its own threads below)
+    mx = red[0];
+#pragma unroll
+    for (int i = 1; i < 8; ++i) mx = fmaxf(mx, red[i]);
+    float sc = 1.f;
+    if (mx >= 32768.f && mx <= 3.0e38f) {
+        int e;
+        frexpf(mx, &e);
+        sc = ldexpf(1.f, e - 15);
+        const float inv = 1.f / sc;
+        for (int64_t k = threadIdx.x; k < q4; k += 256) {
+            const uint2 r = *reinterpret_cast<const uint2*>(xr + 4 * k);
+            const float2 fa = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&r.x));
+            const float2 fb = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&r.y));
+            const __half2 ha = __floats2half2_rn(fa.x * inv, fa.y * inv), hb = __floats2half2_rn(fb.x * inv, fb.y * inv);
+            uint2 h;
+            h.x = *reinterpret_cast<const uint32_t*>(&ha); h.y = *reinterpret_cast<const uint32_t*>(&hb);
+            *reinterpret_cast<uint2*>(hr + 4 * k) = h;
+        }
+        if (threadIdx.x == 0) *flag = 1;
+    }
+    if (threadIdx.x == 0) scale[m] = sc;
+}
+
 template <typename T>
 static cudaError_t run_stack(const aq_stack_t* p, const StackPlan& plan, const T* x0, T* out, int out_buf, int M,
                              aq_dtype_t dt, uint8_t* ws, cudaStream_t s) {
@@ -173,6 +273,13 @@ static cudaError_t run_stack(const aq_stack_t* p, const StackPlan& plan, const T
         const int64_t n = (int64_t)M * p->buf_width[0];
         widen_kernel<T><<<(unsigned)((n + 255) / 256), 256, 0, s>>>(x0, buf(0), n);
         count_launch();
+    }
+    if (!decode && dt == AQ_BF16) {   // the "a row was scaled" flags of all phases start at zero
+        for (int k = 0; k < p->n_ops; ++k) {
+            if (k > 0 && plan.rs_off[k] == plan.rs_off[k - 1]) continue;
+            e = cudaMemsetAsync(ws + plan.rs_off[k] + (size_t)M * sizeof(float), 0, sizeof(int), s);
+            if (e != cudaSuccess) return e;
+        }
     }
     if (decode) {   // one persistent kernel for the whole program, when it fits
         const int r = launch_decode_stack(p, plan, M, dt, ws, s, &e);
@@ -232,7 +339,12 @@ static cudaError_t run_stack(const aq_stack_t* p, const StackPlan& plan, const T
             const unsigned g = (f.in_op == AQ_IN_RMSNORM) ? (unsigned)M : (unsigned)std::min<int64_t>((total4 + 255) / 256, 4 * 148);
             const float* s2 = (f.in_op == AQ_IN_SILU_MUL) ? buf(f.src2) : nullptr;
             if (decode) stage_kernel<T><<<g, 256, 0, s>>>(buf(f.src), s2, (int)f.in_op, K, total4, stage, pre);
-            else e = launch_pdl(stage_kernel<T>, dim3(g), dim3(256), 0, s, (const float*)buf(f.src), s2, (int)f.in_op, K, total4, stage, pre);
+            else if (dt == AQ_BF16) {
+                int* flag = reinterpret_cast<int*>(ws + plan.rs_off[i] + (size_t)M * sizeof(float));
+                e = launch_pdl(stage_rows_bf16_kernel, dim3((unsigned)M), dim3(256), 0, s, (const float*)buf(f.src), s2, (int)f.in_op, K,
+                               reinterpret_cast<__nv_bfloat16*>(stage), reinterpret_cast<__half*>(ws + plan.x16_off[i]),
+                               reinterpret_cast<float*>(ws + plan.rs_off[i]), flag, pre);
+            } else e = launch_pdl(stage_kernel<T>, dim3(g), dim3(256), 0, s, (const float*)buf(f.src), s2, (int)f.in_op, K, total4, stage, pre);
             if (e != cudaSuccess) return e;
         }
         count_launch();
@@ -262,7 +374,11 @@ static cudaError_t run_stack(const aq_stack_t* p, const StackPlan& plan, const T
                     o.w->last_stream = s;
                     ++n; ++j;
                 }
-                e = launch_gemm_group(hs, n, stage, dt, M, outs, ldos, ress, preset, s);
+                if (dt == AQ_BF16)
+                    e = launch_gemm_group(hs, n, ws + plan.x16_off[i], reinterpret_cast<const float*>(ws + plan.rs_off[i]),
+                                          reinterpret_cast<const int*>(ws + plan.rs_off[i] + (size_t)M * sizeof(float)), M, outs, ldos, ress,
+                                          preset, s);
+                else e = launch_gemm_group(hs, n, stage, nullptr, nullptr, M, outs, ldos, ress, preset, s);
                 if (e != cudaSuccess) return e;
             }
         }
