@@ -25,10 +25,11 @@ def _seed(*key) -> int:
     return int(np.random.SeedSequence(list(_flat(key))).generate_state(1)[0])
 
 
-def build_stack(layer_shapes, n_layers, bits, key, outliers=False, sample_rows=0, device="cuda"):
+def build_stack(layer_shapes, n_layers, bits, key, outliers=False, sample_rows=0, device="cuda", full_layers=()):
     """Pack n_layers blocks.  bits: one width per matrix, in order.
     Returns (layers, samples, stats): layers for programs.block_program;
-    samples[(layer, name)] = (row indices, float32 rows, bits) when sample_rows > 0."""
+    samples[(layer, name)] = (row indices, float32 rows, bits) when sample_rows > 0; for the layers
+    listed in full_layers every row is kept."""
     import torch
     layers, samples = [], {}
     weights = packed = device_bytes = 0
@@ -40,6 +41,8 @@ def build_stack(layer_shapes, n_layers, bits, key, outliers=False, sample_rows=0
             W = synth.weights_device(N, K, _seed(key, l, i), outliers=outliers, device=device)
             if sample_rows:
                 rows = np.sort(rs.choice(N, size=min(sample_rows, N), replace=False))
+                if l in full_layers:
+                    rows = np.arange(N)
                 samples[(l, name)] = (rows, W[torch.from_numpy(rows).to(device)].cpu().numpy(), bits[i])
             h = aq.aq_pack(bits[i], 32, W)
             torch.cuda.current_stream().synchronize()
@@ -55,13 +58,14 @@ def build_stack(layer_shapes, n_layers, bits, key, outliers=False, sample_rows=0
     return layers, samples, info
 
 
-def llama7b_decode_stack(n_layers=32, seed=0, sample_rows=0):
+def llama7b_decode_stack(n_layers=32, seed=0, sample_rows=0, full_layers=()):
     """The 7B-class decoder linear stack: per-matrix widths from {2,3,4} with a
     parameter-weighted mean of 2.5 bits, N(0,0.02) weights with 0.1 % x20 outliers."""
     shapes = synth.llama7b_layer()
     sizes = [N * K for (_, _, N, K) in synth.stack_shapes(shapes, n_layers)]
     bits = synth.draw_bits(sizes, 2.5, seed)
-    layers, samples, info = build_stack(shapes, n_layers, bits, (3, seed), outliers=True, sample_rows=sample_rows)
+    layers, samples, info = build_stack(shapes, n_layers, bits, (3, seed), outliers=True, sample_rows=sample_rows,
+                                        full_layers=full_layers)
     prog, out_buf, names = programs.block_program(layers)
     info["bits"] = bits
     info["layers"] = layers   # the packed matrices, for other wirings of the same stack (programs.independent_program)

@@ -60,9 +60,12 @@ def _run(aq, prog, out_buf, names, samples, M, dtype, width, key, kind="normal",
 
 
 def test_config3_full_7b_decode_stack(aq):
-    """32 layers x {q,k,v,o,gate,up,down}, per-matrix 2/3/4-bit (mean 2.5), 0.1% x20 outliers, M = 1, fp16."""
+    """32 layers x {q,k,v,o,gate,up,down}, per-matrix 2/3/4-bit (mean 2.5), 0.1% x20 outliers, M = 1 and 8, fp16.
+    Every output of the first and of the last layer is checked (all 4096 / 11008 rows of their matrices: a unit dealt
+    to the wrong CTA or op would show there), 48 sampled rows per matrix in between.  The oracle re-quantises
+    2 x 202 M weights for this: the test takes about twenty seconds."""
     from paper_2605_24011_b200 import workloads
-    prog, out_buf, names, samples, info = workloads.llama7b_decode_stack(n_layers=32, seed=0, sample_rows=48)
+    prog, out_buf, names, samples, info = workloads.llama7b_decode_stack(n_layers=32, seed=0, sample_rows=48, full_layers=(0, 31))
     assert abs(info["mean_code_bits"] - 2.5) <= 0.005
     assert info["weights"] == 6_476_005_376
     _run(aq, prog, out_buf, names, samples, 1, torch.float16, 4096, (3, 0))

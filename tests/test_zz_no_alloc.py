@@ -44,6 +44,37 @@ def test_noalloc_matches_aq_linear_twice(aq, bits, M, dtype):
     h.free()
 
 
+def test_noalloc_leaves_device_memory_alone_and_fills_the_scratch_to_its_edge(aq):
+    """The property the entry point exists for: after one warm-up call (which looks up the array's address) a burst of
+    calls changes neither the free device memory nor anything the caching allocator holds.  The shape is the largest
+    the fixed array takes: 8 tokens and N = 16380, padded to 16384 rows, so the last row of the last token is the
+    array's last element; the result must still agree with aq_linear's."""
+    N, K, M = 16380, 64, 8
+    W = synth.weights(N, K, 43, 2)
+    h = aq.aq_pack(3, 32, torch.from_numpy(W).cuda())
+    xt = torch.from_numpy(synth.activations(M, K, 43, 1)).to(torch.float16)
+    x = xt.cuda()
+    y = torch.full((M, N), float("nan"), dtype=torch.float16, device="cuda")
+    y_ref = torch.empty((M, N), dtype=torch.float16, device="cuda")
+    aq.aq_linear(h, x, y_ref)
+    aq.aq_linear_noalloc(h, x, y)                 # warm-up: first call on the device
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    reserved0 = torch.cuda.memory_reserved()
+    for _ in range(20):
+        aq.aq_linear_noalloc(h, x, y)
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0 and torch.cuda.memory_reserved() == reserved0
+    aq.aq_check()
+    d, m, q = O.quantize(W, 3)
+    yo, T = O.linear(d, m, q, xt.to(torch.float64).numpy())
+    a, b = y.double().cpu().numpy(), y_ref.double().cpu().numpy()
+    assert O.linear_excess(a, yo, T).max() <= 1.0
+    assert np.all(np.abs(a - b) <= 2 * (2e-3 * T + 1e-5))
+    h.free()
+
+
 def test_noalloc_rejects_what_the_fixed_scratch_cannot_hold(aq):
     lib = aq.raw_lib()
     W = torch.from_numpy(synth.weights(32, 64, 42)).cuda()
