@@ -54,7 +54,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-i", str(self.index), "-lms", "100"], stdout=subprocess.PIPE, text=True)
+                                          "-i", str(self.index), "-lms", "20"], stdout=subprocess.PIPE, text=True)
             self.t = threading.Thread(target=self._read, daemon=True)
             self.t.start()
         except Exception:
@@ -259,10 +259,17 @@ def run_micro(args):
 def run_configs(args):
     """The five workload configurations, one timing each (CUDA events, cold weights where a case fits in L2)."""
     import torch
-    from paper_2605_24011_b200 import aq, programs, synth, workloads
     torch.cuda.set_device(0)
-    peaks = _peaks()
+    print(json.dumps(configs_leg(_peaks(), torch, None, None, None)))
+
+
+def configs_leg(peaks, torch, prog7, out_buf7, info7):
+    """One timing per workload configuration other than the headline one, each with its roofline fraction (HBM bytes
+    for the decode-shaped ones, flops for the prefill-shaped ones).  prog7: the 7B-class stack when the caller has
+    built it already (else it is built here)."""
+    from paper_2605_24011_b200 import aq, programs, synth, workloads
     out = {"peaks": peaks}
+    hbm, tf_peak = peaks["hbm_gbs"], peaks["bf16_tflops"]
 
     def timed_us(fn, steps, warm=3):
         return 1e3 * _timed(fn, steps, warm, torch) / steps
@@ -285,7 +292,11 @@ def run_configs(args):
     pb = 4096 * 4096 * 5 // 8
     t_lc, t_lh = timed_us(lin_cold, 48), timed_us(lambda: aq.aq_linear(hs[0], x, y), 48)
     t_dc, t_dh = timed_us(deq_cold, 48), timed_us(lambda: aq.aq_dequant(hs[0], wf[0]), 48)
-    out["config1"] = {"linear_M1_us_cold": t_lc, "linear_M1_gbs_cold": pb / t_lc / 1e3, "linear_M1_us_l2hot": t_lh,
+    out["config1"] = {"roofline": {"bound": "hbm", "achieved": pb / t_lc / 1e3, "peak": hbm, "unit": "GB/s", "frac": pb / t_lc / 1e3 / hbm,
+                                   "what": "aq_linear M=1, 4096x4096 4-bit, cold L2 (24 packed copies in rotation)"},
+                      "dequant_roofline": {"bound": "hbm", "achieved": (pb + 2 * 4096 * 4096) / t_dc / 1e3, "peak": hbm, "unit": "GB/s",
+                                           "frac": (pb + 2 * 4096 * 4096) / t_dc / 1e3 / hbm},
+                      "linear_M1_us_cold": t_lc, "linear_M1_gbs_cold": pb / t_lc / 1e3, "linear_M1_us_l2hot": t_lh,
                       "linear_M1_gbs_l2hot": pb / t_lh / 1e3, "dequant_us_cold": t_dc,
                       "dequant_gbs_cold": (pb + 2 * 4096 * 4096) / t_dc / 1e3, "dequant_us_l2hot": t_dh,
                       "note": "one aq_linear call = streaming kernel + output cast (two launches)"}
@@ -314,21 +325,34 @@ def run_configs(args):
         t = timed_us(mlp, 36, 12)
         cfg2[f"M{M}_us"] = t
         cfg2[f"M{M}_gbs"] = 3 * 22_544_384 / t / 1e3
+        cfg2[f"M{M}_roofline"] = {"bound": "hbm", "achieved": 3 * 22_544_384 / t / 1e3, "peak": hbm, "unit": "GB/s",
+                                  "frac": 3 * 22_544_384 / t / 1e3 / hbm}
     out["config2"] = cfg2
     for st in sets:
         for h in st[3]:
             h.free()
     del sets
 
-    # 3 and 4: the 7B-class stack, M = 1 (fp16) and M = 512 (bf16)
-    prog, out_buf, names, _, info = workloads.llama7b_decode_stack(n_layers=32, seed=0)
-    for M, dt, key in ((1, torch.float16, "config3"), (8, torch.float16, "config3_M8"), (512, torch.bfloat16, "config4")):
+    # 3 and 4: the 7B-class stack, M = 1 (fp16) and M = 512 (bf16); only M = 8 when the caller times those two itself
+    if prog7 is None:
+        prog, out_buf, names, _, info = workloads.llama7b_decode_stack(n_layers=32, seed=0)
+        cases = ((1, torch.float16, "config3"), (8, torch.float16, "config3_M8"), (512, torch.bfloat16, "config4"))
+    else:
+        prog, out_buf, info = prog7, out_buf7, info7
+        cases = ((8, torch.float16, "config3_M8"),)
+    for M, dt, key in cases:
         ws = torch.empty(prog.workspace_bytes(M), dtype=torch.uint8, device="cuda")
         x0 = workloads.activations_device(M, 4096, dt, 3, M, kind="vision_text" if M == 512 else "normal")
         yo = torch.empty((M, 4096), dtype=dt, device="cuda")
         t = timed_us(lambda: aq.aq_stack_forward(prog, x0, yo, out_buf, M, ws), 20 if M <= 8 else 5)
         out[key] = {"us_per_pass": t, "gbs": info["packed_bytes"] / t / 1e3, "tflops": 2.0 * M * info["weights"] / t / 1e6,
                     "mean_code_bits": info["mean_code_bits"]}
+        if M <= 8:
+            out[key]["roofline"] = {"bound": "hbm", "achieved": info["packed_bytes"] / t / 1e3, "peak": hbm, "unit": "GB/s",
+                                    "frac": info["packed_bytes"] / t / 1e3 / hbm}
+        else:
+            out[key]["roofline"] = {"bound": "tensor", "achieved": 2.0 * M * info["weights"] / t / 1e6, "peak": tf_peak, "unit": "TFLOP/s",
+                                    "frac": 2.0 * M * info["weights"] / t / 1e6 / tf_peak}
         del ws
     del prog
 
@@ -340,7 +364,9 @@ def run_configs(args):
     yo = torch.empty((M, 2048), dtype=torch.bfloat16, device="cuda")
     t = timed_us(lambda: aq.aq_stack_forward(prog, x0, yo, out_buf, M, ws), 5)
     c5 = {"backbone_prefill_M768_us": t, "backbone_prefill_tflops": 2.0 * M * info["weights"] / t / 1e6,
-          "backbone_mean_code_bits": info["mean_code_bits"]}
+          "backbone_mean_code_bits": info["mean_code_bits"],
+          "backbone_roofline": {"bound": "tensor", "achieved": 2.0 * M * info["weights"] / t / 1e6, "peak": tf_peak, "unit": "TFLOP/s",
+                                "frac": 2.0 * M * info["weights"] / t / 1e6 / tf_peak}}
     del prog, ws
     prog, out_buf, names, _, info = workloads.expert_stack(n_layers=18, seed=0)
     M = 50
@@ -367,11 +393,15 @@ def run_configs(args):
             ten_steps()
     torch.cuda.synchronize()
     tg = timed_us(graph.replay, 5)
+    c5["expert_roofline"] = {"bound": "hbm", "achieved": 10 * info["packed_bytes"] / t / 1e3, "peak": hbm, "unit": "GB/s",
+                             "frac": 10 * info["packed_bytes"] / t / 1e3 / hbm,
+                             "what": "bytes = packed weights per flow-matching step (M = 50: 2 M flops per weight is far below the "
+                                     "tensor roofline, the step is bound by streaming the weights and by its 144 launches)"}
     c5.update({"expert_graph_10_steps_M50_us": tg, "expert_graph_us_per_step": tg / 10,
                "expert_graph_gbs": 10 * info["packed_bytes"] / tg / 1e3, "expert_graph_tflops": 10 * 2.0 * M * info["weights"] / tg / 1e6})
     out["config5"] = c5
     aq.aq_check()
-    print(json.dumps(out))
+    return out
 
 
 WORKLOAD = ("7B-class decoder linear stack, M=1 decode: 32 layers x {q,k,v,o 4096x4096; gate,up 11008x4096; "
@@ -382,7 +412,7 @@ WORKLOAD = ("7B-class decoder linear stack, M=1 decode: 32 layers x {q,k,v,o 409
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
     ap.add_argument("--layers", type=int, default=32, help="decoder layers (32 = the full workload)")
@@ -498,8 +528,10 @@ def main():
     }
 
     if world == 1 and rank == 0 and not args.no_extras:
-        line["prefill"] = prefill_leg(aq, workloads, prog, out_buf, info, peaks, torch)
+        line["prefill"] = prefill_leg(aq, workloads, prog, out_buf, info, peaks, torch, local)
         line["dequant"] = dequant_leg(aq, synth, peaks, torch)
+        if args.layers == 32:
+            line["configs"] = configs_leg(peaks, torch, prog, out_buf, info)
         cores = len(os.sched_getaffinity(0))
         mats = oracle_layer_sample()
         dt, nb = time_oracle(mats, repeats=7)
@@ -515,13 +547,15 @@ def main():
 
 # dram__bytes_read.sum + dram__bytes_write.sum of the decode kernel per stack pass, from the ncu
 # capture summarised under profiles/ (None until a capture has been taken).
-DECODE_TRAFFIC_BYTES = int((354.938e6 + 4.175e6) * 2833383424 / 354.17e6)
+DECODE_TRAFFIC_BYTES = None
 # gemm_kernel: 21.21 MB of DRAM traffic per 11008 x 4096 launch, scaled by weights to the 224 matrices of one pass
-PREFILL_TRAFFIC_BYTES = int(21.21e6 * 6476005376 / (11008 * 4096))
+PREFILL_TRAFFIC_BYTES = None
 
 
-def prefill_leg(aq, workloads, prog, out_buf, info, peaks, torch):
-    """Same stack, M = 512 prefill: 256 vision-like rows + 256 text rows, bf16."""
+def prefill_leg(aq, workloads, prog, out_buf, info, peaks, torch, gpu_index=0):
+    """Same stack, M = 512 prefill: 256 vision-like rows + 256 text rows, bf16.  The leg is a burst (a quarter of a
+    second), so its roofline fraction divides by the measured burst peak; the fraction of the sustained peak (what a
+    seconds-long GEMM loop holds under the power cap) is given beside it."""
     M = 512
     ws = torch.empty(prog.workspace_bytes(M), dtype=torch.uint8, device="cuda")
     x0 = workloads.activations_device(M, 4096, torch.bfloat16, 4, 0, kind="vision_text")
@@ -530,18 +564,26 @@ def prefill_leg(aq, workloads, prog, out_buf, info, peaks, torch):
     def step():
         aq.aq_stack_forward(prog, x0, out, out_buf, M, ws)
 
+    n_pass = 25
+    for _ in range(3):
+        step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(gpu_index)
+    sampler.start()
     l0 = aq.aq_kernel_launches()
-    ms = _timed(step, 5, 3, torch) / 5
-    launches = (aq.aq_kernel_launches() - l0) // 8
+    ms = _timed(step, n_pass, 0, torch) / n_pass
+    launches = (aq.aq_kernel_launches() - l0) // n_pass
+    clocks = sampler.stop()
     aq.aq_check()
     flops = 2.0 * M * info["weights"]
     tf = flops / (ms * 1e-3) / 1e12
     return {"workload": "same stack, M=512 (256 vision rows N(0,1)*U(0.5,2) + 256 text rows), bf16, dequant->tcgen05 GEMM",
             "ms_per_pass": ms, "tflops": tf, "pct_of_nominal_bf16": 100.0 * tf / NOMINAL_BF16_TFLOPS,
-            "gpu_launches_per_pass": int(launches),
-            "roofline": {"bound": "tensor", "achieved": tf, "peak": peaks["bf16_tflops_sustained"] or peaks["bf16_tflops"],
-                         "unit": "TFLOP/s", "frac": tf / (peaks["bf16_tflops_sustained"] or peaks["bf16_tflops"]),
-                         "traffic": PREFILL_TRAFFIC_BYTES, "peak_source": peaks["source"] + " (sustained: timed inside a long step)",
+            "gpu_launches_per_pass": int(launches), "passes_timed": n_pass, "clocks": clocks,
+            "roofline": {"bound": "tensor", "achieved": tf, "peak": peaks["bf16_tflops"],
+                         "unit": "TFLOP/s", "frac": tf / peaks["bf16_tflops"],
+                         "frac_of_sustained_peak": tf / (peaks["bf16_tflops_sustained"] or peaks["bf16_tflops"]),
+                         "traffic": PREFILL_TRAFFIC_BYTES, "peak_source": peaks["source"] + " (burst peak: the leg lasts about 0.2 s)",
                          "kernel": "gemm_kernel (128 grouped launches per pass; time = whole pass incl. staging kernels)"}}
 
 

@@ -73,7 +73,9 @@ struct StackPlan {
     std::vector<size_t> pk_off;     // per buffer (M <= AQ_DECODE_MAX_M only): its packed 64-bit sums [M][width]
     size_t pk_begin = 0, pk_end = 0;   // the packed sums' region: zero at the start of a decode pass
     std::vector<size_t> x16_off;    // per op (bfloat16, M > AQ_DECODE_MAX_M only): its phase's binary16 operand [M][K] ...
-    std::vector<size_t> rs_off;     // ... and the row scales [M] float32, followed by the flag (int)
+    std::vector<size_t> rs_off;     // ... the row scales [M] float32 ...
+    std::vector<size_t> flag_off;   // ... and the phase's "some row is scaled" flag (int), inside [flags_begin, flags_end)
+    size_t flags_begin = 0, flags_end = 0;
     size_t stage_off = 0;           // end of the float32 buffers
     size_t total = 0;
 };

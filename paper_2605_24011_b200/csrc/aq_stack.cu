@@ -61,12 +61,20 @@ static bool plan_stack(const aq_stack_t* p, int M, StackPlan& plan) {
     if (M > AQ_DECODE_MAX_M) {   // bfloat16 activations reach the tensor cores as binary16: a second staged vector per phase
         plan.x16_off.assign(p->n_ops, 0);
         plan.rs_off.assign(p->n_ops, 0);
+        plan.flag_off.assign(p->n_ops, 0);
+        plan.flags_begin = off;          // one int per phase, together: a single memset clears them
+        off += align_up((size_t)p->n_ops * sizeof(int), 256);
+        plan.flags_end = off;
         for (int i = 0; i < p->n_ops; ++i) {
-            if (i > 0 && same_input(p->ops[i], p->ops[i - 1])) { plan.x16_off[i] = plan.x16_off[i - 1]; plan.rs_off[i] = plan.rs_off[i - 1]; continue; }
+            if (i > 0 && same_input(p->ops[i], p->ops[i - 1])) {
+                plan.x16_off[i] = plan.x16_off[i - 1]; plan.rs_off[i] = plan.rs_off[i - 1]; plan.flag_off[i] = plan.flag_off[i - 1];
+                continue;
+            }
+            plan.flag_off[i] = plan.flags_begin + (size_t)i * sizeof(int);
             plan.x16_off[i] = off;
             off += align_up((size_t)M * p->buf_width[p->ops[i].src] * 2, 256);
             plan.rs_off[i] = off;
-            off += align_up((size_t)M * sizeof(float) + 16, 256);
+            off += align_up((size_t)M * sizeof(float), 256);
         }
     }
     if (M <= AQ_DECODE_MAX_M) {   // the whole-program decode kernel accumulates packed 64-bit sums, one per element
@@ -275,11 +283,8 @@ static cudaError_t run_stack(const aq_stack_t* p, const StackPlan& plan, const T
         count_launch();
     }
     if (!decode && dt == AQ_BF16) {   // the "a row was scaled" flags of all phases start at zero
-        for (int k = 0; k < p->n_ops; ++k) {
-            if (k > 0 && plan.rs_off[k] == plan.rs_off[k - 1]) continue;
-            e = cudaMemsetAsync(ws + plan.rs_off[k] + (size_t)M * sizeof(float), 0, sizeof(int), s);
-            if (e != cudaSuccess) return e;
-        }
+        e = cudaMemsetAsync(ws + plan.flags_begin, 0, plan.flags_end - plan.flags_begin, s);
+        if (e != cudaSuccess) return e;
     }
     if (decode) {   // one persistent kernel for the whole program, when it fits
         const int r = launch_decode_stack(p, plan, M, dt, ws, s, &e);
@@ -340,7 +345,7 @@ static cudaError_t run_stack(const aq_stack_t* p, const StackPlan& plan, const T
             const float* s2 = (f.in_op == AQ_IN_SILU_MUL) ? buf(f.src2) : nullptr;
             if (decode) stage_kernel<T><<<g, 256, 0, s>>>(buf(f.src), s2, (int)f.in_op, K, total4, stage, pre);
             else if (dt == AQ_BF16) {
-                int* flag = reinterpret_cast<int*>(ws + plan.rs_off[i] + (size_t)M * sizeof(float));
+                int* flag = reinterpret_cast<int*>(ws + plan.flag_off[i]);
                 e = launch_pdl(stage_rows_bf16_kernel, dim3((unsigned)M), dim3(256), 0, s, (const float*)buf(f.src), s2, (int)f.in_op, K,
                                reinterpret_cast<__nv_bfloat16*>(stage), reinterpret_cast<__half*>(ws + plan.x16_off[i]),
                                reinterpret_cast<float*>(ws + plan.rs_off[i]), flag, pre);
@@ -376,7 +381,7 @@ static cudaError_t run_stack(const aq_stack_t* p, const StackPlan& plan, const T
                 }
                 if (dt == AQ_BF16)
                     e = launch_gemm_group(hs, n, ws + plan.x16_off[i], reinterpret_cast<const float*>(ws + plan.rs_off[i]),
-                                          reinterpret_cast<const int*>(ws + plan.rs_off[i] + (size_t)M * sizeof(float)), M, outs, ldos, ress,
+                                          reinterpret_cast<const int*>(ws + plan.flag_off[i]), M, outs, ldos, ress,
                                           preset, s);
                 else e = launch_gemm_group(hs, n, stage, nullptr, nullptr, M, outs, ldos, ress, preset, s);
                 if (e != cudaSuccess) return e;
