@@ -698,8 +698,12 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArg
                         int sl = -1;
 #pragma unroll
                         for (int x = 0; x < DS_MAX_SLOTS; ++x) sl = (x < n_slots && slabs[x] == slab) ? x : sl;
-                        place(sl >= 0 ? sh.xs + (size_t)sl * slab_bytes : nullptr, 0, i4,
-                              make_float4(v[n].x * scale, v[n].y * scale, v[n].z * scale, v[n].w * scale), mine);
+                        // most of the row is read for its sum of squares only: a warp (its 32 groups are half a slab)
+                        // whose groups are neither staged nor part of this CTA's share of the caller's copy rounds nothing
+                        const int wg = i4 - lane;
+                        if (sl >= 0 || (wg < g1 && wg + 32 > g0))
+                            place(sl >= 0 ? sh.xs + (size_t)sl * slab_bytes : nullptr, 0, i4,
+                                  make_float4(v[n].x * scale, v[n].y * scale, v[n].z * scale, v[n].w * scale), mine);
                     }
                 }
             } else {
