@@ -378,3 +378,115 @@ def quantize_opt(W: np.ndarray, bits: int, F=None, rounds: int = 4):
     m = np.where(useB, mB, mA)
     q = np.where(useB[:, :, None], qB, qA)
     return d, m, q.astype(np.uint8).reshape(N, K)
+
+
+# --------------------------------------------------------------------------
+# Super-blocks: two-level block parameters [Section 3, "Weight quantization"]
+# --------------------------------------------------------------------------
+# The paper's format is a block / super-block hierarchy: S consecutive blocks form a super-block
+# whose own scale and zero point compress the per-block (s_b, z_b).  It prints neither S nor the
+# width of the compressed parameters.  Reading taken here: S = 8 blocks (256 weights); the block
+# scales and the block minima of a super-block are each coded with Eq. 1's rule one level up,
+# with 6-bit codes u_b, v_b in {0..63}:
+#     scale_b = D u_b                     (symmetric special case: zero point 0; D binary16)
+#     min_b   = Mn + Dm v_b               (asymmetric: Mn, Dm binary16; Mn plays the zero point)
+# and the decoded block parameters are rounded to binary16, so that a super-block matrix decodes
+# exactly like a plain one with those parameters: w_hat = f16(scale_b) q + f16(min_b).
+# Stored bits per weight: n + (3 * 16 + 8 * 12) / 256 = n + 0.5625 (against n + 1).
+SUPER = 8
+SUB_MAX = 63
+
+
+def sb_block_params(D, Dm, Mn, u, v):
+    """Decoded per-block (scale, min) as binary16 [N][K/32] from the super-block parameters
+    D, Dm, Mn [N][K/256] (binary16) and the 6-bit codes u, v [N][K/32].  One rounding each:
+    scale = f16(D u) (the product is exact in binary32), min = f16(fma(Dm, v, Mn))."""
+    D32 = np.repeat(np.asarray(D, dtype=np.float16).astype(np.float32), SUPER, axis=1)
+    Dm64 = np.repeat(np.asarray(Dm, dtype=np.float16).astype(np.float64), SUPER, axis=1)
+    Mn64 = np.repeat(np.asarray(Mn, dtype=np.float16).astype(np.float64), SUPER, axis=1)
+    with np.errstate(over="ignore", invalid="ignore"):
+        d = (D32 * u.astype(np.float32)).astype(np.float32).astype(np.float16)
+        # fused multiply-add: the exact value (float64 holds it) rounded once to binary32, then to binary16
+        m = (Dm64 * v.astype(np.float64) + Mn64).astype(np.float32).astype(np.float16)
+    return d, m
+
+
+def quantize_sb(W: np.ndarray, bits: int):
+    """Round-to-nearest quantiser with super-block parameters.  W float32 [N][K], K % 256 == 0.
+    Returns (D, Dm, Mn, u, v, q).  Every step is one correctly rounded binary32 operation:
+        per block:        s = (max - min) / L,  mn = min                         (as quantize(), before binary16)
+        per super-block:  D  = f16(max_b s / 63);              u_b = clamp(rint(s_b / D), 0, 63)   (0 when D = 0)
+                          Mn = f16(min_b mn_b);  Dm = f16(max(0, max_b mn_b - Mn) / 63)
+                          v_b = clamp(rint((mn_b - Mn) / Dm), 0, 63)                               (0 when Dm = 0)
+        codes:            q = clamp(rint((w - min_b) / scale_b), 0, L) with the DECODED block parameters
+                          (sb_block_params), 0 everywhere when scale_b = 0."""
+    W = np.ascontiguousarray(W, dtype=np.float32)
+    N, K = W.shape
+    if K % (BLOCK * SUPER):
+        raise ValueError("K must be a multiple of 256")
+    f32 = np.float32
+    L = f32(code_max(bits))
+    Wb = W.reshape(N, K // BLOCK, BLOCK)
+    mn, mx = Wb.min(axis=2), Wb.max(axis=2)
+    s = ((mx - mn).astype(f32) / L).astype(f32)
+    sS, mnS = s.reshape(N, -1, SUPER), mn.reshape(N, -1, SUPER)
+    with np.errstate(divide="ignore", invalid="ignore", over="ignore"):
+        D = (sS.max(axis=2) / f32(SUB_MAX)).astype(f32).astype(np.float16)
+        D32 = D.astype(f32)[:, :, None]
+        u = np.where(D32 == 0, f32(0), np.clip(np.rint((sS / D32).astype(f32)), 0, SUB_MAX))
+        Mn = mnS.min(axis=2).astype(np.float16)
+        Mn32 = Mn.astype(f32)
+        Dm = (np.maximum((mnS.max(axis=2) - Mn32).astype(f32), f32(0)) / f32(SUB_MAX)).astype(f32).astype(np.float16)
+        Dm32 = Dm.astype(f32)[:, :, None]
+        t = ((mnS - Mn32[:, :, None]).astype(f32) / Dm32).astype(f32)
+        v = np.where(Dm32 == 0, f32(0), np.clip(np.rint(t), 0, SUB_MAX))
+    u = np.nan_to_num(u).astype(np.uint8).reshape(N, K // BLOCK)
+    v = np.nan_to_num(v).astype(np.uint8).reshape(N, K // BLOCK)
+    d, m = sb_block_params(D, Dm, Mn, u, v)
+    d32, m32 = d.astype(f32)[:, :, None], m.astype(f32)[:, :, None]
+    with np.errstate(divide="ignore", invalid="ignore", over="ignore"):
+        tq = ((Wb - m32).astype(f32) / d32).astype(f32)
+    tq = np.where(d32 == 0, f32(0), tq)
+    q = np.clip(np.rint(tq), 0, L)
+    return D, Dm, Mn, u, v, q.astype(np.uint8).reshape(N, K)
+
+
+def packed_nbytes_sb(N: int, K: int, bits: int) -> int:
+    """Closed form: per super-block 6 + 12 + 8 * 4n bytes, i.e. n + 0.5625 bits per weight."""
+    return N * (K // (BLOCK * SUPER)) * (18 + 32 * bits)
+
+
+def pack_sb(D, Dm, Mn, u, v, q, bits: int) -> np.ndarray:
+    """Canonical bytes of a super-block matrix: super-blocks in row-major order over (row, super-block); a record is
+    [D f16 LE][Dm f16 LE][Mn f16 LE][12 bytes: one little-endian integer of 96 bits in which block b's u sits at bits
+    [12 b, 12 b + 6) and its v at [12 b + 6, 12 b + 12)][codes of the 8 blocks: 8 x 4n bytes, each block as in pack()]."""
+    N, ns = D.shape
+    nb = ns * SUPER
+    assert u.shape == (N, nb) and v.shape == (N, nb) and q.shape == (N, nb * BLOCK)
+    assert int(u.max(initial=0)) <= SUB_MAX and int(v.max(initial=0)) <= SUB_MAX and int(q.max(initial=0)) <= code_max(bits)
+    rec = np.empty((N, ns, 18 + 32 * bits), dtype=np.uint8)
+    for a, off in ((D, 0), (Dm, 2), (Mn, 4)):
+        rec[:, :, off:off + 2] = np.asarray(a).astype("<f2").view(np.uint8).reshape(N, ns, 2)
+    uv = u.astype(np.uint16) | (v.astype(np.uint16) << 6)                      # 12 bits per block
+    uvbits = np.unpackbits(uv.reshape(N, ns, SUPER, 1).view(np.uint8), axis=3, bitorder="little")[..., :12]
+    rec[:, :, 6:18] = np.packbits(uvbits.reshape(N, ns, SUPER * 12), axis=2, bitorder="little")
+    codebits = np.unpackbits(q.reshape(N, ns, SUPER * BLOCK, 1), axis=3, bitorder="little")[..., :bits]
+    rec[:, :, 18:] = np.packbits(codebits.reshape(N, ns, SUPER * BLOCK * bits), axis=2, bitorder="little")
+    return rec.reshape(-1)
+
+
+def unpack_sb(buf: np.ndarray, bits: int, N: int, K: int):
+    """Inverse of pack_sb(): canonical bytes -> (D, Dm, Mn, u, v, q)."""
+    ns = K // (BLOCK * SUPER)
+    buf = np.asarray(buf, dtype=np.uint8)
+    assert buf.size == packed_nbytes_sb(N, K, bits)
+    rec = buf.reshape(N, ns, 18 + 32 * bits)
+    f = lambda off: np.ascontiguousarray(rec[:, :, off:off + 2]).view("<f2").reshape(N, ns).astype(np.float16)
+    D, Dm, Mn = f(0), f(2), f(4)
+    uvbits = np.unpackbits(np.ascontiguousarray(rec[:, :, 6:18]), axis=2, bitorder="little").reshape(N, ns, SUPER, 12)
+    w6 = (1 << np.arange(6)).astype(np.uint8)
+    u = (uvbits[..., :6] * w6).sum(axis=3).astype(np.uint8).reshape(N, ns * SUPER)
+    v = (uvbits[..., 6:] * w6).sum(axis=3).astype(np.uint8).reshape(N, ns * SUPER)
+    cb = np.unpackbits(np.ascontiguousarray(rec[:, :, 18:]), axis=2, bitorder="little").reshape(N, ns, SUPER * BLOCK, bits)
+    q = (cb * (1 << np.arange(bits)).astype(np.uint8)).sum(axis=3).astype(np.uint8).reshape(N, K)
+    return D, Dm, Mn, u, v, q
