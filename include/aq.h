@@ -144,6 +144,31 @@ aq_status_t aq_allocate_bits(const double* S, const int64_t* numel, const int32_
                              double* objective_out);
 
 /*
+ * aq_pack_sb / aq_import_sb / aq_export_sb -- the two-level (super-block) form of the format (Section 3, "Weight
+ * quantization": every S consecutive blocks form a super-block with its own scale and zero point that compress the
+ * per-block parameters).  The paper prints neither S nor the width of the compressed parameters; this library takes
+ * S = 8 blocks (256 weights) and, per super-block, three binary16 values D, Dm, Mn and per block two 6-bit codes
+ * u, v in {0 .. 63}:      scale_b = f16(D u_b),      min_b = f16(fma(Dm, v_b, Mn)),
+ * Eq. 1's rule one level up (zero point 0 for the scales, Mn for the minima), the decoded block parameters rounded
+ * to binary16; codes q as in aq_pack with those parameters.  K % 256 == 0; sblock must be 8.
+ * Canonical bytes: super-blocks in row-major order over (row, super-block); a record is
+ *     [D][Dm][Mn] (binary16 LE) [12 bytes: a little-endian integer of 96 bits, block b's u at bits [12 b, 12 b + 6),
+ *     its v at [12 b + 6, 12 b + 12)] [codes of the 8 blocks, each as in the plain record]
+ * i.e. n + 0.5625 bits per weight instead of n + 1 (aq_info's packed_bytes).  Quantiser, in binary32 with one
+ * rounding per operation: s_b = (max - min) / (2^n - 1) and mn_b = min per block; D = f16(max_b s_b / 63),
+ * u_b = clamp(rint(s_b / D)); Mn = f16(min_b mn_b), Dm = f16(max(0, max_b mn_b - Mn) / 63), v_b = clamp(rint((mn_b -
+ * Mn) / Dm)) (codes 0 where a divisor is 0).  On the device the handle keeps the decoded block parameters in the
+ * ordinary layout, so aq_dequant, aq_linear and aq_stack_forward take it like any other handle (its device memory is
+ * that of a plain handle plus 32 bytes per super-block; the saving is the container's).  aq_export on such a handle
+ * gives the plain record form with the decoded parameters.  Errors as aq_pack / aq_import / aq_export.
+ */
+aq_status_t aq_pack_sb(int bits, int block, int sblock, const float* W_dev, int64_t N, int64_t K, aq_stream_t stream,
+                       aq_handle_t* out);
+aq_status_t aq_import_sb(int bits, int block, int sblock, int64_t N, int64_t K, const void* canon_host, size_t nbytes,
+                         aq_stream_t stream, aq_handle_t* out);
+aq_status_t aq_export_sb(aq_handle_t h, void* canon_host, size_t cap, size_t* nbytes);
+
+/*
  * aq_import -- build a handle from canonical bytes (Appendix D container).
  *   canon_host : HOST, nbytes == N*K*(bits+1)/8 bytes in the layout above
  * Synchronises `stream` before returning (the host buffer may be reused).

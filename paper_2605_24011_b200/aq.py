@@ -25,7 +25,7 @@ AQ_IN_PLAIN, AQ_IN_RMSNORM, AQ_IN_SILU_MUL = 0, 1, 2
 AQ_OUT_STORE, AQ_OUT_ADD = 0, 1
 AQ_MAX_M, AQ_DECODE_MAX_M = 4096, 8
 
-SYMBOLS = ("aq_pack", "aq_pack_opt", "aq_import", "aq_export", "aq_info", "aq_dequant", "aq_linear", "aq_linear_f32out", "aq_linear_noalloc",
+SYMBOLS = ("aq_pack", "aq_pack_opt", "aq_pack_sb", "aq_import_sb", "aq_export_sb", "aq_import", "aq_export", "aq_info", "aq_dequant", "aq_linear", "aq_linear_f32out", "aq_linear_noalloc",
            "aq_rbf_gram", "aq_hsic", "aq_sensitivity", "aq_allocate_bits",
            "aq_stack_workspace_bytes", "aq_stack_forward", "aq_stack_buffer_offset", "aq_stack_input_offset", "aq_check", "aq_free",
            "aq_set_wait_limit_ns", "aq_debug_decode_hold", "aq_status_string", "aq_last_cuda_error", "aq_kernel_launches")
@@ -56,6 +56,12 @@ _lib.aq_allocate_bits.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64,
                                   C.POINTER(C.c_double)]
 _lib.aq_allocate_bits.restype = C.c_int
 _lib.aq_import.argtypes = [C.c_int, C.c_int, C.c_int64, C.c_int64, C.c_void_p, C.c_size_t, C.c_void_p, C.POINTER(_H)]
+_lib.aq_pack_sb.argtypes = [C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.POINTER(_H)]
+_lib.aq_pack_sb.restype = C.c_int
+_lib.aq_import_sb.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int64, C.c_int64, C.c_void_p, C.c_size_t, C.c_void_p, C.POINTER(_H)]
+_lib.aq_import_sb.restype = C.c_int
+_lib.aq_export_sb.argtypes = [_H, C.c_void_p, C.c_size_t, C.POINTER(C.c_size_t)]
+_lib.aq_export_sb.restype = C.c_int
 _lib.aq_export.argtypes = [_H, C.c_void_p, C.c_size_t, C.POINTER(C.c_size_t)]
 _lib.aq_info.argtypes = [_H, C.POINTER(C.c_int), C.POINTER(C.c_int), C.POINTER(C.c_int64), C.POINTER(C.c_int64),
                          C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
@@ -238,6 +244,36 @@ def aq_import(bits: int, block: int, N: int, K: int, canon, stream=None) -> Hand
     h = _H()
     _check(_lib.aq_import(bits, block, N, K, buf.ctypes.data, buf.size, _stream(stream), C.byref(h)), "aq_import")
     return Handle(h.value)
+
+
+def aq_pack_sb(bits: int, W, block: int = 32, sblock: int = 8, stream=None) -> Handle:
+    """Super-block form: W CUDA float32 [N][K] (contiguous), K % 256 == 0."""
+    N, K = W.shape
+    h = _H()
+    _check(_lib.aq_pack_sb(bits, block, sblock, _ptr(W), N, K, _stream(stream), C.byref(h)), "aq_pack_sb")
+    return Handle(h.value)
+
+
+def aq_import_sb(bits: int, N: int, K: int, canon, block: int = 32, sblock: int = 8, stream=None) -> Handle:
+    """canon: host bytes / numpy uint8 array holding the canonical super-block stream."""
+    import numpy as np
+    buf = np.ascontiguousarray(np.frombuffer(canon, dtype=np.uint8) if isinstance(canon, (bytes, bytearray)) else canon,
+                               dtype=np.uint8)
+    h = _H()
+    _check(_lib.aq_import_sb(bits, block, sblock, N, K, buf.ctypes.data, buf.size, _stream(stream), C.byref(h)), "aq_import_sb")
+    return Handle(h.value)
+
+
+def aq_export_sb(h: Handle, allow_range_error: bool = False):
+    """Canonical super-block bytes as a numpy uint8 array."""
+    import numpy as np
+    n = C.c_size_t()
+    _check(_lib.aq_export_sb(h.raw, None, 0, C.byref(n)), "aq_export_sb(size)")
+    out = np.empty(n.value, dtype=np.uint8)
+    st = _lib.aq_export_sb(h.raw, out.ctypes.data, out.size, C.byref(n))
+    if not (allow_range_error and st == AQ_ERR_RANGE):
+        _check(st, "aq_export_sb")
+    return out
 
 
 def aq_export(h: Handle, allow_range_error: bool = False):

@@ -71,7 +71,7 @@ static aq_status_t new_handle(int bits, int block, int64_t N, int64_t K, aq_hand
     h->n_frags = (int64_t)h->NT * h->KP * 2;
     h->dev_bytes = (size_t)h->n_frags * frag_bytes(bits);
     h->frags = nullptr; h->acc = nullptr; h->flags = nullptr; h->last_stream = nullptr;
-    h->big = nullptr; h->big_bytes = 0;
+    h->big = nullptr; h->big_bytes = 0; h->sb = nullptr;
     const size_t acc_bytes = (size_t)AQ_DECODE_MAX_M * h->NT * 16 * sizeof(float);
     if (cudaMalloc(&h->frags, h->dev_bytes) != cudaSuccess || cudaMalloc(&h->acc, acc_bytes) != cudaSuccess ||
         cudaMalloc(&h->flags, 256) != cudaSuccess) {
@@ -85,7 +85,7 @@ static aq_status_t new_handle(int bits, int block, int64_t N, int64_t K, aq_hand
 }
 
 static void destroy(aq_handle_s* h) {
-    cudaFree(h->frags); cudaFree(h->acc); cudaFree(h->flags); cudaFree(h->big);
+    cudaFree(h->frags); cudaFree(h->acc); cudaFree(h->flags); cudaFree(h->big); cudaFree(h->sb);
     h->magic = 0;
     delete h;
 }
@@ -126,6 +126,66 @@ aq_status_t aq_pack_opt(int bits, int block, const float* W_dev, const float* F_
     cudaError_t e = cudaMemsetAsync(h->acc, 0, (size_t)AQ_DECODE_MAX_M * h->NT * 16 * sizeof(float), s);
     if (e == cudaSuccess) e = cudaMemsetAsync(h->flags, 0, 256, s);
     if (e == cudaSuccess) e = launch_pack_opt(h, W_dev, F_dev, rounds, s);
+    if (e != cudaSuccess) { destroy(h); return cuda_fail(e); }
+    h->last_stream = s;
+    *out = h;
+    return AQ_OK;
+}
+
+static size_t sb_nbytes(int bits, int64_t N, int64_t K) { return (size_t)N * (size_t)(K / 256) * (size_t)(18 + 32 * bits); }
+
+static aq_status_t new_sb_handle(int bits, int block, int sblock, int64_t N, int64_t K, aq_handle_t* out) {
+    if (!out) return AQ_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (sblock != 8) return AQ_ERR_UNSUPPORTED;
+    if (K < 256 || K % 256 != 0) return AQ_ERR_INVALID_ARG;
+    aq_handle_t h = nullptr;
+    aq_status_t st = new_handle(bits, block, N, K, &h);
+    if (st != AQ_OK) return st;
+    if (cudaMalloc(&h->sb, (size_t)N * (size_t)(K / 256) * 32) != cudaSuccess) { cudaGetLastError(); destroy(h); return AQ_ERR_ALLOC; }
+    *out = h;
+    return AQ_OK;
+}
+
+aq_status_t aq_pack_sb(int bits, int block, int sblock, const float* W_dev, int64_t N, int64_t K, aq_stream_t stream,
+                       aq_handle_t* out) {
+    if (!out) return AQ_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!W_dev || !aligned16(W_dev)) return AQ_ERR_INVALID_ARG;
+    aq_handle_t h = nullptr;
+    aq_status_t st = new_sb_handle(bits, block, sblock, N, K, &h);
+    if (st != AQ_OK) return st;
+    cudaStream_t s = (cudaStream_t)stream;
+    cudaError_t e = cudaMemsetAsync(h->acc, 0, (size_t)AQ_DECODE_MAX_M * h->NT * 16 * sizeof(float), s);
+    if (e == cudaSuccess) e = cudaMemsetAsync(h->flags, 0, 256, s);
+    if (e == cudaSuccess) e = launch_pack_sb(h, W_dev, s);
+    if (e != cudaSuccess) { destroy(h); return cuda_fail(e); }
+    h->last_stream = s;
+    *out = h;
+    return AQ_OK;
+}
+
+aq_status_t aq_import_sb(int bits, int block, int sblock, int64_t N, int64_t K, const void* canon_host, size_t nbytes,
+                         aq_stream_t stream, aq_handle_t* out) {
+    if (!out) return AQ_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!canon_host) return AQ_ERR_INVALID_ARG;
+    aq_handle_t h = nullptr;
+    aq_status_t st = new_sb_handle(bits, block, sblock, N, K, &h);
+    if (st != AQ_OK) return st;
+    if (nbytes != sb_nbytes(bits, N, K)) { destroy(h); return AQ_ERR_INVALID_ARG; }
+    cudaStream_t s = (cudaStream_t)stream;
+    const size_t plain_bytes = (size_t)N * (size_t)(K / 32) * (size_t)(4 + 4 * bits);
+    const size_t plain_at = (nbytes + 255) / 256 * 256;
+    uint8_t* tmp = nullptr;
+    if (cudaMalloc(&tmp, plain_at + plain_bytes) != cudaSuccess) { cudaGetLastError(); destroy(h); return AQ_ERR_ALLOC; }
+    cudaError_t e = cudaMemcpyAsync(tmp, canon_host, nbytes, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaMemsetAsync(h->acc, 0, (size_t)AQ_DECODE_MAX_M * h->NT * 16 * sizeof(float), s);
+    if (e == cudaSuccess) e = cudaMemsetAsync(h->flags, 0, 256, s);
+    if (e == cudaSuccess) e = launch_sb_records(h, tmp, tmp + plain_at, true, s);
+    if (e == cudaSuccess) e = launch_import(h, tmp + plain_at, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    cudaFree(tmp);
     if (e != cudaSuccess) { destroy(h); return cuda_fail(e); }
     h->last_stream = s;
     *out = h;
@@ -181,6 +241,26 @@ aq_status_t aq_export(aq_handle_t h, void* canon_host, size_t cap, size_t* nbyte
     return range_status(h);
 }
 
+aq_status_t aq_export_sb(aq_handle_t h, void* canon_host, size_t cap, size_t* nbytes) {
+    if (!handle_ok(h) || !h->sb) return AQ_ERR_INVALID_ARG;
+    const size_t need = sb_nbytes(h->bits, h->N, h->K);
+    if (nbytes) *nbytes = need;
+    if (!canon_host) return nbytes ? AQ_OK : AQ_ERR_INVALID_ARG;
+    if (cap < need) return AQ_ERR_INVALID_ARG;
+    const size_t plain_bytes = (size_t)h->N * (size_t)(h->K / 32) * (size_t)(4 + 4 * h->bits);
+    const size_t plain_at = (need + 255) / 256 * 256;
+    uint8_t* tmp = nullptr;
+    if (cudaMalloc(&tmp, plain_at + plain_bytes) != cudaSuccess) { cudaGetLastError(); return AQ_ERR_ALLOC; }
+    cudaStream_t s = h->last_stream;
+    cudaError_t e = launch_export(h, tmp + plain_at, s);
+    if (e == cudaSuccess) e = launch_sb_records(h, tmp, tmp + plain_at, false, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(canon_host, tmp, need, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    cudaFree(tmp);
+    if (e != cudaSuccess) return cuda_fail(e);
+    return range_status(h);
+}
+
 aq_status_t aq_info(aq_handle_t h, int* bits, int* block, int64_t* N, int64_t* K, size_t* packed_bytes,
                     size_t* device_bytes) {
     if (!handle_ok(h)) return AQ_ERR_INVALID_ARG;
@@ -188,8 +268,8 @@ aq_status_t aq_info(aq_handle_t h, int* bits, int* block, int64_t* N, int64_t* K
     if (block) *block = 32;
     if (N) *N = h->N;
     if (K) *K = h->K;
-    if (packed_bytes) *packed_bytes = (size_t)h->N * (size_t)(h->K / 32) * (size_t)(4 + 4 * h->bits);
-    if (device_bytes) *device_bytes = h->dev_bytes;
+    if (packed_bytes) *packed_bytes = h->sb ? sb_nbytes(h->bits, h->N, h->K) : (size_t)h->N * (size_t)(h->K / 32) * (size_t)(4 + 4 * h->bits);
+    if (device_bytes) *device_bytes = h->dev_bytes + (h->sb ? (size_t)h->N * (size_t)(h->K / 256) * 32 : 0);
     return range_status(h);
 }
 

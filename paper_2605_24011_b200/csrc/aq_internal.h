@@ -21,6 +21,8 @@ struct aq_handle_s {
     size_t dev_bytes;  // n_frags * frag_bytes
     uint8_t* frags;    // DEVICE: fragment layout
     float* acc;        // DEVICE: [AQ_DECODE_MAX_M][NT*16] accumulation scratch, zero between calls
+    uint8_t* sb;       // DEVICE: super-block parameters (32 bytes per row and super-block) of a handle made by aq_pack_sb /
+                       // aq_import_sb, else null
     uint8_t* big;      // DEVICE: scratch of aq_linear with M > AQ_DECODE_MAX_M (float32 sums, binary16 copy of bfloat16
                        // activations, row scales), allocated when the handle first sees such a call and grown on demand
     size_t big_bytes;
@@ -40,6 +42,10 @@ cudaError_t launch_pack_opt(const aq_handle_s* h, const float* W, const float* F
 cudaError_t launch_import(const aq_handle_s* h, const uint8_t* canon_dev, cudaStream_t s);
 cudaError_t launch_export(const aq_handle_s* h, uint8_t* canon_dev, cudaStream_t s);
 cudaError_t launch_dequant(const aq_handle_s* h, void* out, aq_dtype_t dt, cudaStream_t s);
+// super-block format (aq_superblock.cu): quantise into fragments + side entries; canonical super-block bytes <-> plain
+// canonical records carrying the decoded block parameters (to_plain also fills the side entries)
+cudaError_t launch_pack_sb(const aq_handle_s* h, const float* W, cudaStream_t s);
+cudaError_t launch_sb_records(const aq_handle_s* h, uint8_t* sbcanon_dev, uint8_t* plain_dev, bool to_plain, cudaStream_t s);
 
 // decode path: accumulate x W^T into acc (fp32 [M][ldacc]); x is [M][K] of xdt.  With y_fused the kernel's last CTA
 // also writes y[m][n] = cast(acc[m][n]) (row-major [M][N] of ydt) and leaves acc zero again: acc must be the handle's own
