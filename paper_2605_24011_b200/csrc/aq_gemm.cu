@@ -18,9 +18,10 @@
 //   D[128 lanes][tokens] fp32 in TMEM: two accumulators of up to 256 tokens, so
 //                       a weight is dequantised once per 512 tokens.
 // One persistent CTA per SM.  The work -- (row tile, token super-tile, 128-k
-// slab) triples, weighted by their accumulators -- is cut into equal contiguous
-// runs, one per CTA; a run that covers a tile's whole K stores its sums, any
-// other run adds them with red.add (the launcher zeroes the output first).
+// slab) triples, weighted by their accumulators -- is cut into contiguous
+// runs, one per CTA, balanced for MMA work plus a fixed cost per piece of a
+// tile; a run that covers a tile's whole K stores its sums, any other run
+// adds them (reduce-add copies; see the store-first protocol below).
 // Warp roles: 0..7 = dequantise then epilogue, 8 = token-tile TMA producer
 // (+ TMEM allocation), 9 = MMA issue, 10 = packed-fragment bulk-copy producer.
 // Epilogue: TMEM -> registers -> 32 x 32 fp32 chunks in shared memory (the idle
@@ -59,6 +60,10 @@ constexpr int GM_MAX_TILES = 8192;
 __device__ uint32_t g_tile_flags[GM_FLAG_SLOTS][GM_MAX_TILES];
 
 constexpr int GM_MAX_OPS = 4;      // matrices that share one input (q|k|v, gate|up) run as one launch
+constexpr int GM_MAX_GRID = 192;   // CTAs of one launch (one per SM)
+// What ending one piece of a tile costs a CTA (accumulator drain, epilogue, refilling the pipeline), in units of one
+// slab-accumulator of MMA work (measured: about 8 us against 0.88 us); the runs are cut so that work + pieces balance.
+constexpr int GM_SEG_COST = 9;
 
 struct GemmOp {
     const uint8_t* frags;
@@ -87,6 +92,7 @@ struct GemmArgs {
     uint32_t epoch;
     const float* tok_scale;    // per token: the power of two its row of x was divided by, or null
     const int* scaled_flag;    // nonzero when some entry of tok_scale is not 1 (null: none is)
+    int bounds[GM_MAX_GRID + 1];   // CTA c works on slab-accumulators [bounds[c], bounds[c + 1]) (even numbers)
 };
 
 struct GemmOutMaps { CUtensorMap m[GM_MAX_OPS]; };
@@ -245,9 +251,7 @@ __global__ void __launch_bounds__(GM_THREADS, 1) gemm_kernel(const __grid_consta
     pdl_launch_dependents();
 
     // this CTA's run, in slab-accumulators (even bounds)
-    const long long total = (long long)a.n_slabs * a.Rtot * (2LL * a.n2 + (a.n_st - a.n2));
-    const long long run_lo = ((total * blockIdx.x) / gridDim.x) & ~1LL;
-    const long long run_hi = (blockIdx.x + 1 == gridDim.x) ? total : (((total * (blockIdx.x + 1)) / gridDim.x) & ~1LL);
+    const long long run_lo = a.bounds[blockIdx.x], run_hi = a.bounds[blockIdx.x + 1];
     GemmSeg sg;
     long long pos = run_lo;
 
@@ -389,11 +393,11 @@ __global__ void __launch_bounds__(GM_THREADS, 1) gemm_kernel(const __grid_consta
                 if (a.tma_out) {
                     // the A ring is idle now (every MMA of the run has completed): two 4 KB chunks per warp
                     float* stg = reinterpret_cast<float*>(sA + dw * 8192);
-                    int buf = 0;
-                    for (int c0 = c_lo; c0 < c_hi; c0 += 32, buf ^= 1) {
-                        uint32_t v[32];
-                        tmem_ld32(tmem_base + ((uint32_t)(lq * 32) << 16) + (uint32_t)(acc * GM_MAX_TN + c0), v);
-                        tmem_ld_wait();
+                    // two register sets: the TMEM load of the next 32 columns is in flight while this one is staged
+                    const uint32_t t_addr = tmem_base + ((uint32_t)(lq * 32) << 16) + (uint32_t)(acc * GM_MAX_TN);
+                    auto emit = [&](uint32_t (&v)[32], int c0, int buf) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) asm volatile("" : "+r"(v[j]));   // (read only after the wait above)
                         if (lane == 0) bulk_wait_read<1>();   // the copy that last read this chunk has left shared memory
                         __syncwarp();
                         float* chunk = stg + buf * 1024;      // [32 tokens][32 rows]
@@ -410,6 +414,19 @@ __global__ void __launch_bounds__(GM_THREADS, 1) gemm_kernel(const __grid_consta
                             if (whole) tma_store_2d(tmo, smem_u32(chunk), n0, tok0 + c0);
                             else tma_reduce_add_2d(tmo, smem_u32(chunk), n0, tok0 + c0);
                             bulk_commit();
+                        }
+                    };
+                    uint32_t va[32], vb[32];
+                    int n_chunks = 0;   // (the two staging chunks alternate; the copies are drained at the end of the piece)
+                    if (c_lo < c_hi) tmem_ld32(t_addr + (uint32_t)c_lo, va);
+                    for (int c0 = c_lo; c0 < c_hi; c0 += 64) {
+                        tmem_ld_wait();
+                        if (c0 + 32 < c_hi) tmem_ld32(t_addr + (uint32_t)(c0 + 32), vb);
+                        emit(va, c0, n_chunks++ & 1);
+                        if (c0 + 32 < c_hi) {
+                            tmem_ld_wait();
+                            if (c0 + 64 < c_hi) tmem_ld32(t_addr + (uint32_t)(c0 + 64), va);
+                            emit(vb, c0 + 32, n_chunks++ & 1);
                         }
                     }
                     if (lane == 0) {
@@ -470,6 +487,39 @@ EncodeTiledFn tensor_map_encoder() {
     return fn;
 }
 
+// Cuts [0, total) into `grid` contiguous runs with even bounds.  A run costs its slab-accumulators plus GM_SEG_COST per
+// tile it touches; the smallest budget under which a greedy walk places everything is found by bisection.  Tiles:
+// n_two of c2 units first, then tiles of c1 units.
+static void cut_runs(long long total, long long n_two, long long c2, long long c1, int grid, int* bounds) {
+    auto tile_end = [&](long long pos) {
+        const long long reg2 = n_two * c2;
+        return pos < reg2 ? (pos / c2 + 1) * c2 : reg2 + ((pos - reg2) / c1 + 1) * c1;
+    };
+    auto walk = [&](long long budget, int* out) {
+        long long pos = 0;
+        for (int c = 0; c < grid; ++c) {
+            if (out) out[c] = (int)pos;
+            long long left = budget;
+            while (pos < total) {
+                const long long te = tile_end(pos), need = GM_SEG_COST + (te - pos);
+                if (need <= left) { pos = te; left -= need; continue; }
+                const long long take = (left - GM_SEG_COST) & ~1LL;
+                if (take >= 2) pos += take;
+                break;
+            }
+        }
+        if (out) out[grid] = (int)total;
+        return pos >= total;
+    };
+    long long lo = total / grid, hi = total / grid + c2 + 4 * GM_SEG_COST + 2;
+    while (!walk(hi, nullptr)) hi *= 2;
+    while (lo < hi) {
+        const long long mid = (lo + hi) / 2;
+        if (walk(mid, nullptr)) hi = mid; else lo = mid + 1;
+    }
+    walk(hi, bounds);   // (a tail of CTAs may be left without work: their runs are empty)
+}
+
 static cudaError_t launch_one(const CUtensorMap& tm, const GemmOutMaps& tmo, const GemmArgs& a, int grid, cudaStream_t s) {
     constexpr int SMEM = 1024 + GM_ASTAGES * GM_A_BYTES + GM_BSLOTS * GM_B_BYTES + GM_PSTAGES * 8 * frag_bytes(4) + 256;
     auto kern = gemm_kernel;
@@ -513,8 +563,10 @@ cudaError_t launch_gemm_group(const aq_handle_s* const* hs, int n, const void* x
         a.tn = ((M + 15) / 16) * 16; a.st_tokens = a.tn; a.n_st = 1; a.n2 = 0;
     }
     const long long total = (long long)a.n_slabs * a.Rtot * (2LL * a.n2 + (a.n_st - a.n2));
-    int grid = sm_count();
+    int grid = sm_count() < GM_MAX_GRID ? sm_count() : GM_MAX_GRID;
     if (total / 2 < grid) grid = (int)(total / 2);
+    if (total > 0x7fffffffLL) return cudaErrorInvalidValue;
+    cut_runs(total, (long long)a.n2 * a.Rtot, 2LL * a.n_slabs, a.n_slabs, grid, a.bounds);
     CUtensorMap tm;
     const cuuint64_t dims[2] = {(cuuint64_t)hs[0]->K, (cuuint64_t)M};
     const cuuint64_t strides[1] = {(cuuint64_t)hs[0]->K * 2};
@@ -544,7 +596,7 @@ cudaError_t launch_gemm_group(const aq_handle_s* const* hs, int n, const void* x
     {
         const long long c2 = 2LL * a.n_slabs, reg2 = c2 * a.n2 * a.Rtot;
         for (int c = 1; c < grid && all_whole; ++c) {
-            const long long b = ((total * c) / grid) & ~1LL;
+            const long long b = a.bounds[c];
             all_whole = (b <= reg2) ? (b % c2 == 0) : ((b - reg2) % a.n_slabs == 0);
         }
     }
