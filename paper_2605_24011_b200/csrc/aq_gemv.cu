@@ -148,8 +148,90 @@ static cudaError_t launch_one(const GemvArgs& a, cudaStream_t s) {
     return cudaGetLastError();
 }
 
+// Small matrices (a few MB: the launch, not HBM, is what counts): one CTA per 16-row tile, its warps share the tile's
+// k-slabs, sum in registers along k and meet in shared memory, and the tile's outputs are cast and written by the CTA
+// itself: no global atomics, no ticket, no second pass over the sums.
+constexpr int ROWS_STAGES = 2;
+
+template <int BITS, int MT, bool BF16>
+__global__ void __launch_bounds__(GEMV_WARPS * 32) gemv_rows_kernel(const GemvArgs a) {
+    constexpr int UB = 2 * frag_bytes(BITS);
+    constexpr int PIECES = UB / 16 / 32;
+    extern __shared__ __align__(128) uint8_t smem[];
+    __shared__ float sums[8 * 16];   // [token][row of the tile]
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int R = blockIdx.x;
+    const int KP = (int)(a.n_units / a.NT);
+    uint8_t* ring = smem + (size_t)warp * ROWS_STAGES * UB;
+    const uint32_t ring_s = (uint32_t)__cvta_generic_to_shared(ring);
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    auto issue = [&](int P, int slot) {
+        const uint8_t* src = a.frags + ((int64_t)P * a.NT + R) * UB;
+        const uint32_t dst = ring_s + slot * UB;
+#pragma unroll
+        for (int p = 0; p < PIECES; ++p) cp_async16(dst + (p * 32 + lane) * 16, src + (p * 32 + lane) * 16, pol);
+    };
+#pragma unroll
+    for (int i = 0; i < ROWS_STAGES; ++i) {
+        if (warp + GEMV_WARPS * i < KP) issue(warp + GEMV_WARPS * i, i);
+        cp_async_commit();
+    }
+    if (threadIdx.x < 8 * 16) sums[threadIdx.x] = 0.f;
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    int slot = 0;
+    for (int P = warp; P < KP; P += GEMV_WARPS) {
+        XOperand<MT> xo;
+        load_x_operand<MT, BF16>(xo, a.x, a.K, a.M, P, lane);
+        cp_async_wait<ROWS_STAGES - 1>();
+        __syncwarp();
+        unit_mac<BITS, MT, BF16>(ring + slot * UB, xo, lane, acc);
+        __syncwarp();   // every lane has read the slot
+        if (P + GEMV_WARPS * ROWS_STAGES < KP) issue(P + GEMV_WARPS * ROWS_STAGES, slot);
+        cp_async_commit();
+        slot ^= 1;
+    }
+    cp_async_wait<0>();
+    __syncthreads();   // sums are zero
+    if (warp < KP) unit_commit<MT>(acc, sums, 16, 0, 16, a.M, lane);
+    __syncthreads();
+    if (threadIdx.x < 16 * a.M) {
+        const int m = threadIdx.x >> 4, r = threadIdx.x & 15;
+        const int64_t row = (int64_t)R * 16 + r;
+        if (row < a.N) {
+            const float v = sums[m * 16 + r];
+            const int64_t i = (int64_t)m * a.N + row;
+            if (a.ydt == AQ_F32) reinterpret_cast<float*>(a.y)[i] = v;
+            else if (a.ydt == AQ_F16) reinterpret_cast<__half*>(a.y)[i] = __float2half_rn(v);
+            else reinterpret_cast<__nv_bfloat16*>(a.y)[i] = __float2bfloat16_rn(v);
+        }
+    }
+}
+
+template <int BITS, int MT, bool BF16>
+static cudaError_t launch_rows(const GemvArgs& a, cudaStream_t s) {
+    constexpr int SMEM = GEMV_WARPS * ROWS_STAGES * 2 * frag_bytes(BITS);
+    static_assert(SMEM <= 48 * 1024, "fits the default dynamic shared memory limit");
+    gemv_rows_kernel<BITS, MT, BF16><<<a.NT, GEMV_WARPS * 32, SMEM, s>>>(a);
+    count_launch();
+    return cudaGetLastError();
+}
+
+// True when the row-tile kernel above is the better choice: outputs written by the kernel, one wave of CTAs, every
+// warp with a short run along k.
+static bool rows_kernel_fits(const GemvArgs& a) {
+    const int64_t KP = a.n_units / a.NT;
+    return a.y != nullptr && a.NT <= 4 * sm_count() && KP >= 2 && KP <= 8 * GEMV_WARPS;
+}
+
 template <int BITS, bool BF16>
 static cudaError_t launch_mt(const GemvArgs& a, cudaStream_t s) {
+    if (rows_kernel_fits(a)) {
+        if (a.M == 1) return launch_rows<BITS, 1, BF16>(a, s);
+        if (a.M == 2) return launch_rows<BITS, 2, BF16>(a, s);
+        if (a.M <= 4) return launch_rows<BITS, 4, BF16>(a, s);
+        return launch_rows<BITS, 8, BF16>(a, s);
+    }
     if (a.M == 1) return launch_one<BITS, 1, BF16>(a, s);
     if (a.M == 2) return launch_one<BITS, 2, BF16>(a, s);
     if (a.M <= 4) return launch_one<BITS, 4, BF16>(a, s);
