@@ -191,18 +191,27 @@ __device__ __forceinline__ bool dequant_slab(const uint8_t* slab, bool have, int
         ++ai;
         uint8_t* At = sA + as * GM_A_BYTES;
 #pragma unroll
-        for (int jj = 0; jj < 2; ++jj) {
-            const int j = 2 * h + jj;
+        for (int hi = 0; hi < 2; ++hi) {
+            // the two 16-byte chunks of this lane (blocks 2h and 2h + 1 of the row)
+            uint32_t o[2][4];
 #pragma unroll
-            for (int hi = 0; hi < 2; ++hi) {
+            for (int jj = 0; jj < 2; ++jj) {
+                const int j = 2 * h + jj;
                 const __half2 dm = *reinterpret_cast<const __half2*>(&dmw[hi][j]);
                 const __half2 d2 = __low2half2(dm), m2 = __high2half2(dm);
-                uint32_t o[4];
 #pragma unroll
-                for (int i = 0; i < 4; ++i) o[i] = dequant_pair(code_pair<BITS>(lc, j, hi, i, MAGIC), d2, m2);
-                const int row = dw * 16 + g + 8 * hi;
-                const int chunk = (jj * 4 + t) ^ (row & 7);
-                *reinterpret_cast<uint4*>(At + (row >> 3) * 1024 + (row & 7) * 128 + chunk * 16) = make_uint4(o[0], o[1], o[2], o[3]);
+                for (int i = 0; i < 4; ++i) o[jj][i] = dequant_pair(code_pair<BITS>(lc, j, hi, i, MAGIC), d2, m2);
+            }
+            // Rows with odd g store block 2h + 1 first: the eight lanes that a 16-byte store serves together (g = 2q,
+            // 2q + 1; t = 0..3) then hit eight different chunks of the swizzle atom instead of four twice.
+            const int row = dw * 16 + g + 8 * hi;
+            const bool odd = (g & 1) != 0;
+            uint8_t* rp = At + (row >> 3) * 1024 + (row & 7) * 128;
+#pragma unroll
+            for (int st = 0; st < 2; ++st) {
+                const int jj = odd ? 1 - st : st;
+                const uint4 v = (st == 0) == !odd ? make_uint4(o[0][0], o[0][1], o[0][2], o[0][3]) : make_uint4(o[1][0], o[1][1], o[1][2], o[1][3]);
+                *reinterpret_cast<uint4*>(rp + (((jj * 4 + t) ^ (row & 7)) * 16)) = v;
             }
         }
         fence_async_smem();
