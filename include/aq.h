@@ -303,6 +303,14 @@ size_t aq_stack_workspace_bytes(const aq_stack_t* prog, int M);
  *                   afterwards buffer b is float32 [M][width[b]] at byte
  *                   offset aq_stack_buffer_offset(prog, M, b): every op's
  *                   input and output stay readable for per-op checks
+ * CUDA graphs: the call may be recorded into a graph (stream capture) and
+ * replayed.  For M <= AQ_DECODE_MAX_M make one eager call with the same
+ * program, M, dtype and workspace on that device first: it builds the device
+ * tables of the one-launch kernel, which allocates, and a capture forbids
+ * allocation (without that call the capture records the slower form, one
+ * launch per linear).  Tables used under a capture stay until a handle of the
+ * program is freed.  aq_free of any handle of the program releases them and
+ * invalidates every graph recorded with it: destroy those graphs first.
  */
 aq_status_t aq_stack_forward(const aq_stack_t* prog, const void* x0_dev, void* out_dev, int out_buf,
                              int M, aq_dtype_t dtype, void* workspace_dev, size_t ws_bytes,
