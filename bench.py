@@ -574,11 +574,14 @@ def main():
         dist.destroy_process_group()
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum of the decode kernel per stack pass, from the ncu
-# capture summarised under profiles/ (None until a capture has been taken).
-DECODE_TRAFFIC_BYTES = None
-# gemm_kernel: 21.21 MB of DRAM traffic per 11008 x 4096 launch, scaled by weights to the 224 matrices of one pass
-PREFILL_TRAFFIC_BYTES = None
+# dram__bytes_read.sum + dram__bytes_write.sum of the decode kernel per stack pass, from the ncu capture summarised in
+# profiles/decode_stack_kernel_7b_4layers_M1.md: 355,753,984 + 4,211,456 bytes for the first 4 layers (354,172,928
+# packed bytes), times 8 for the 32 layers (every byte is read once, so traffic grows with the packed bytes).
+# Set to None whenever the kernel changes, until the capture has been taken again.
+DECODE_TRAFFIC_BYTES = 8 * (355_753_984 + 4_211_456)
+# gemm_kernel (profiles/gemm_kernel_11008x4096_M512_2bit.md): 21,212,160 + 19,456 bytes of DRAM traffic for one 11008 x 4096
+# 2-bit launch (16,908,288 packed bytes), scaled by packed bytes to the 224 matrices of one pass
+PREFILL_TRAFFIC_BYTES = round(2_833_383_424 * (21_212_160 + 19_456) / 16_908_288)
 
 
 def prefill_leg(aq, workloads, prog, out_buf, info, peaks, torch, gpu_index=0):
@@ -612,7 +615,8 @@ def prefill_leg(aq, workloads, prog, out_buf, info, peaks, torch, gpu_index=0):
             "roofline": {"bound": "tensor", "achieved": tf, "peak": peaks["bf16_tflops"],
                          "unit": "TFLOP/s", "frac": tf / peaks["bf16_tflops"],
                          "frac_of_sustained_peak": tf / (peaks["bf16_tflops_sustained"] or peaks["bf16_tflops"]),
-                         "traffic": PREFILL_TRAFFIC_BYTES, "peak_source": peaks["source"] + " (burst peak: the leg lasts about 0.2 s)",
+                         "traffic": PREFILL_TRAFFIC_BYTES, "traffic_note": "dram bytes of the one-launch ncu capture (11008 x 4096) scaled by packed bytes to the pass",
+                         "peak_source": peaks["source"] + " (burst peak: the leg lasts about 0.2 s)",
                          "kernel": "gemm_kernel (128 grouped launches per pass; time = whole pass incl. staging kernels)"}}
 
 
