@@ -105,6 +105,9 @@ struct DsPhase {
     uint32_t expect;       // contributions that complete an element of src
     uint32_t expect2;
     int32_t pad_[1];
+    u64* norm;             // [CTAs][M] (sum of squares over the CTA's share of the row | 1 << 32), zero before the
+                           // pass; null: every CTA reads whole rows for the norm itself
+    u64 pad2_;
     DsOp ops[DS_MAX_PHASE_OPS];
 };
 static_assert(sizeof(DsOp) == 48, "DsOp layout");
@@ -707,7 +710,47 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArg
                     }
                 }
             } else {
-                if (P.in_op == AQ_IN_RMSNORM) {
+                bool normed = false;
+                if constexpr (MT > 1) {
+                if (P.in_op == AQ_IN_RMSNORM && P.norm != nullptr) {
+                    // Row norms from shares: this CTA sums the squares of its share of every token row (one group of
+                    // four per thread, one trip to L2), publishes the M partial sums as (float | 1 << 32) words, and
+                    // gathers every CTA's words; all sums run in a fixed order, so every CTA gets the same norms.
+                    float* part = &sh.red[0][0];
+                    float* gathered = reinterpret_cast<float*>(sh.xs);   // [CTA][M]: the slab area is not in use yet
+                    const int share = g1 - g0, n_items = share * M;      // (the host made sure n_items fits sh.red)
+                    if ((int)threadIdx.x < n_items) {
+                        const int m = (int)threadIdx.x / share, i4 = g0 + (int)threadIdx.x - m * share;
+                        const float4 v = source4(P.src, P.src_f, expect, m, i4);
+                        part[threadIdx.x] = fmaf(v.x, v.x, fmaf(v.y, v.y, fmaf(v.z, v.z, v.w * v.w)));
+                    }
+                    ds_consumer_sync();
+                    if ((int)threadIdx.x < M) {
+                        float ss = 0.f;
+                        for (int j = 0; j < share; ++j) ss += part[threadIdx.x * share + j];
+                        const u64 w = (u64)__float_as_uint(ss) | (1ull << 32);
+                        asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(P.norm + (size_t)blockIdx.x * M + threadIdx.x), "l"(w) : "memory");
+                    }
+                    const int n_words = (int)gridDim.x * M;
+                    for (int it = threadIdx.x; it < n_words; it += DS_CTHREADS) {
+                        u64 w;
+                        for (;;) {
+                            w = ds_ld1(P.norm + it);
+                            if ((w >> 32) != 0 || give_up()) break;
+                        }
+                        gathered[it] = __uint_as_float((uint32_t)w);
+                    }
+                    ds_consumer_sync();
+                    if ((int)threadIdx.x < M) {
+                        float tot = 0.f;
+                        for (int c = 0; c < (int)gridDim.x; ++c) tot += gathered[c * M + threadIdx.x];
+                        sh.scale[threadIdx.x] = rsqrtf(tot / (float)P.K + 1e-6f);
+                    }
+                    ds_consumer_sync();
+                    normed = true;
+                }
+                }
+                if (P.in_op == AQ_IN_RMSNORM && !normed) {
                     for (int m = 0; m < M; ++m) {
                         float ss = 0.f;
                         for (int i = threadIdx.x; i < q4; i += DS_CTHREADS) {
@@ -977,6 +1020,13 @@ bool build_decode_tables(const aq_stack_t* p, const StackPlan& plan, int M, int 
             if (f.in_op == AQ_IN_RMSNORM) whole[f.src] = 1;
             P.stage = ws + plan.in_off[first];
             P.K = (int32_t)K; P.in_op = f.in_op; P.op_count = count;
+            // several tokens: the row norms come from per-CTA partial sums exchanged through the workspace (whole
+            // rows read by every CTA are 8 M K bytes per CTA from the same lines of L2); the partial sums of a CTA's
+            // share are added up through sh.red, hence the bound on the share
+            P.norm = nullptr;
+            if (f.in_op == AQ_IN_RMSNORM && M >= 3 && !plan.nm_off.empty() && plan.nm_off[pfirst] != 0 && n_cta <= AQ_NORM_MAX_CTAS &&
+                (int64_t)M * ((K / 4 + n_cta - 1) / n_cta + 1) <= (int64_t)AQ_DECODE_MAX_M * DS_WARPS)
+                P.norm = reinterpret_cast<u64*>(ws + plan.nm_off[pfirst]);
             for (int i = first; i < last; ++i) {
                 const aq_stack_op_t& o = p->ops[i];
                 DsOp& d = P.ops[i - first];

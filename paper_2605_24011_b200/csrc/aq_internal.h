@@ -71,6 +71,9 @@ cudaError_t launch_gemm_group(const aq_handle_s* const* hs, int n, const void* x
 bool gemm_outputs_can_be_preset(float* const* outs, const int64_t* ldos, int n);
 bool gemm_stores_first(const aq_handle_s* const* hs, int n, int M, cudaStream_t s);   // then only residuals need presetting
 
+// CTAs the whole-program decode kernel may have when it exchanges row norms through the workspace (one per SM).
+constexpr int AQ_NORM_MAX_CTAS = 192;
+
 // Where a program's buffers and staged inputs sit in the caller's workspace (aq_stack.cu).
 struct StackPlan {
     std::vector<size_t> buf_off;    // per buffer: float32 [M][width]
@@ -78,6 +81,8 @@ struct StackPlan {
     std::vector<int> phase_first;   // first op of each phase (ops that share one input vector)
     std::vector<size_t> pk_off;     // per buffer (M <= AQ_DECODE_MAX_M only): its packed 64-bit sums [M][width]
     size_t pk_begin = 0, pk_end = 0;   // the packed sums' region: zero at the start of a decode pass
+    std::vector<size_t> nm_off;     // per op that opens an RMS-normalised phase (3 <= M <= AQ_DECODE_MAX_M): the CTAs'
+                                    // partial sums of squares [AQ_NORM_MAX_CTAS][M] of 8 bytes, inside the region above; else 0
     std::vector<size_t> x16_off;    // per op (bfloat16, M > AQ_DECODE_MAX_M only): its phase's binary16 operand [M][K] ...
     std::vector<size_t> rs_off;     // ... the row scales [M] float32 ...
     std::vector<size_t> flag_off;   // ... and the phase's "some row is scaled" flag (int), inside [flags_begin, flags_end)

@@ -84,6 +84,12 @@ static bool plan_stack(const aq_stack_t* p, int M, StackPlan& plan) {
             plan.pk_off[b] = off;
             off += align_up((size_t)M * p->buf_width[b] * 8, 256);
         }
+        plan.nm_off.assign(p->n_ops, 0);
+        for (int i = 0; i < p->n_ops && M >= 3; ++i) {
+            if (p->ops[i].in_op != AQ_IN_RMSNORM || (i > 0 && same_input(p->ops[i], p->ops[i - 1]))) continue;
+            plan.nm_off[i] = off;
+            off += align_up((size_t)AQ_NORM_MAX_CTAS * M * 8, 256);
+        }
         plan.pk_end = off;
     }
     plan.total = off;
