@@ -163,6 +163,10 @@ struct DsArgs {
     int n_mini_ops;
     int n_tails;
     int M;
+    // the caller's rounded output: the tail chunks that convert [out_src, out_src + out_n) also write it (null: nobody does)
+    void* out;
+    const u64* out_src;
+    int64_t out_n;
 };
 
 // ---- small PTX wrappers ---------------------------------------------------------
@@ -881,7 +885,15 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_stack_kernel(const DsArg
                 DsQuad q;
                 ds_ld_quad(T.src + i, q);
                 if (!ds_quad_complete(T.src + i, q, T.expect, wait_ns, &sh.abort_flag)) ok = false;
-                else *reinterpret_cast<float4*>(T.out + i) = ds_quad_value(q);
+                else {
+                    const float4 v = ds_quad_value(q);
+                    *reinterpret_cast<float4*>(T.out + i) = v;
+                    if (a.out != nullptr) {
+                        const int64_t o = (T.src - a.out_src) + i;
+                        float unused;
+                        if (o >= 0 && o < a.out_n) *reinterpret_cast<uint2*>(reinterpret_cast<uint16_t*>(a.out) + o) = ds_round4<BF16>(v, &unused);
+                    }
+                }
             }
         }
     }
@@ -903,6 +915,7 @@ struct DecodePlan {
     int n_tails = 0;
     int device = 0;
     bool pinned = false;          // recorded into a CUDA graph: its device tables must outlive the plan cache's turnover
+    std::vector<char> in_tails;   // per buffer: the tail chunks convert it (no phase reads it)
     uint64_t stamp = 0;
 };
 
@@ -929,7 +942,8 @@ template <typename T> void key_put(std::vector<uint8_t>& k, const T& v) {
 // read the same input vector) and the list of buffers nobody reads.  False when the program
 // does not fit this kernel.
 bool build_decode_tables(const aq_stack_t* p, const StackPlan& plan, int M, int n_cta, uint8_t* ws,
-                         std::vector<DsPhase>& phases, std::vector<DsTail>& tails, std::vector<DsCtaPhase>& ctab) {
+                         std::vector<DsPhase>& phases, std::vector<DsTail>& tails, std::vector<DsCtaPhase>& ctab,
+                         std::vector<char>& in_tails) {
     if (M < 1 || M > AQ_DECODE_MAX_M || p->n_ops > 32000 || plan.pk_off.empty()) return false;
     phases.clear();
     tails.clear();
@@ -1049,10 +1063,12 @@ bool build_decode_tables(const aq_stack_t* p, const StackPlan& plan, int M, int 
         }
     }
     // what no phase has copied out for the caller
+    in_tails.assign(p->n_bufs, 0);
     for (int b = 1; b < p->n_bufs; ++b) {
         if (writer[b] < 0 || recorded[b]) continue;
         const int64_t n = (int64_t)M * p->buf_width[b];
         if (n % 4) return false;
+        in_tails[b] = 1;
         for (int64_t i = 0; i < n; i += DS_TAIL_CHUNK) {
             DsTail t;
             memset(&t, 0, sizeof(t));
@@ -1089,8 +1105,9 @@ static cudaError_t launch_ds(const DsArgs& a, int grid, cudaStream_t s) {
 }
 
 int launch_decode_stack(const aq_stack_t* p, const StackPlan& plan, int M, aq_dtype_t dt, uint8_t* ws, cudaStream_t s,
-                        cudaError_t* err) {
+                        cudaError_t* err, void* out, int out_buf, bool* wrote_out) {
     *err = cudaSuccess;
+    *wrote_out = false;
     const int grid = sm_count();
     const int dev = current_device();
     cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
@@ -1116,7 +1133,8 @@ int launch_decode_stack(const aq_stack_t* p, const StackPlan& plan, int M, aq_dt
         std::vector<DsPhase> phases;
         std::vector<DsTail> tails;
         std::vector<DsCtaPhase> ctab;
-        if (!build_decode_tables(p, plan, M, grid, ws, phases, tails, ctab)) return 1;
+        std::vector<char> in_tails;
+        if (!build_decode_tables(p, plan, M, grid, ws, phases, tails, ctab, in_tails)) return 1;
         if (g_plans.size() >= MAX_PLANS) {   // make room: the oldest plan no graph refers to
             size_t oldest = g_plans.size();
             for (size_t i = 0; i < g_plans.size(); ++i)
@@ -1129,6 +1147,7 @@ int launch_decode_stack(const aq_stack_t* p, const StackPlan& plan, int M, aq_dt
         dp->key = key;
         dp->device = dev;
         for (int i = 0; i < p->n_ops; ++i) dp->handles.push_back(p->ops[i].w);
+        dp->in_tails = in_tails;
         dp->phases_bytes = (phases.size() * sizeof(DsPhase) + 255) / 256 * 256;
         std::vector<uint8_t> mini(phases.size() * sizeof(DsMiniPhase));
         for (size_t i = 0; i < phases.size(); ++i) {
@@ -1179,6 +1198,14 @@ int launch_decode_stack(const aq_stack_t* p, const StackPlan& plan, int M, aq_dt
     a.n_tails = dp->n_tails;
     a.M = M;
     a.wait_ns = g_wait_ns;
+    a.out = nullptr; a.out_src = nullptr; a.out_n = 0;
+    if (out != nullptr && out_buf >= 1 && out_buf < p->n_bufs && dp->in_tails[out_buf] &&
+        (reinterpret_cast<uintptr_t>(out) & 7u) == 0) {
+        a.out = out;
+        a.out_src = reinterpret_cast<const u64*>(ws + plan.pk_off[out_buf]);
+        a.out_n = (int64_t)M * p->buf_width[out_buf];
+        *wrote_out = true;
+    }
     // the packed sums start from zero
     cudaError_t e = cudaMemsetAsync(ws + plan.pk_begin, 0, plan.pk_end - plan.pk_begin, s);
     if (e == cudaSuccess) {

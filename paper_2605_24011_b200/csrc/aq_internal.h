@@ -93,8 +93,9 @@ struct StackPlan {
 
 // whole-program decode (M <= AQ_DECODE_MAX_M) in one persistent kernel: 0 = launched,
 // 1 = the program does not fit that kernel (nothing launched), -1 = CUDA error in *err
+// (out: the caller's rounded copy of buffer out_buf, or null; *wrote_out: the kernel itself writes it)
 int launch_decode_stack(const aq_stack_t* p, const StackPlan& plan, int M, aq_dtype_t dt, uint8_t* ws, cudaStream_t s,
-                        cudaError_t* err);
+                        cudaError_t* err, void* out, int out_buf, bool* wrote_out);
 void decode_stack_forget(aq_handle_t h);   // drops cached device tables that name h
 int read_decode_status(bool clear);        // nonzero: a bounded wait in the decode-stack kernel ran out
 void set_decode_wait_ns(unsigned long long ns);   // limit of every wait in that kernel (0: the default, two seconds)

@@ -293,12 +293,13 @@ static cudaError_t run_stack(const aq_stack_t* p, const StackPlan& plan, const T
         if (e != cudaSuccess) return e;
     }
     if (decode) {   // one persistent kernel for the whole program, when it fits
-        const int r = launch_decode_stack(p, plan, M, dt, ws, s, &e);
+        bool wrote_out = false;
+        const int r = launch_decode_stack(p, plan, M, dt, ws, s, &e, out, out_buf, &wrote_out);
         if (r < 0) return e;
         if (r == 0) {
             for (int k = 0; k < p->n_ops; ++k) p->ops[k].w->last_stream = s;
         }
-        if (r == 0 && out) {
+        if (r == 0 && out && !wrote_out) {
             const int64_t n = (int64_t)M * p->buf_width[out_buf];
             narrow_kernel<T><<<(unsigned)((n + 255) / 256), 256, 0, s>>>(buf(out_buf), out, n);
             count_launch();
