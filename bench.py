@@ -575,10 +575,10 @@ def main():
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum of the decode kernel per stack pass, from the ncu capture summarised in
-# profiles/decode_stack_kernel_7b_4layers_M1.md: 355,753,984 + 4,211,456 bytes for the first 4 layers (354,172,928
+# profiles/decode_stack_kernel_7b_4layers_M1.md: 355,754,752 + 3,822,848 bytes for the first 4 layers (354,172,928
 # packed bytes), times 8 for the 32 layers (every byte is read once, so traffic grows with the packed bytes).
 # Set to None whenever the kernel changes, until the capture has been taken again.
-DECODE_TRAFFIC_BYTES = 8 * (355_753_984 + 4_211_456)
+DECODE_TRAFFIC_BYTES = 8 * (355_754_752 + 3_822_848)
 # gemm_kernel (profiles/gemm_kernel_11008x4096_M512_2bit.md): 21,212,160 + 19,456 bytes of DRAM traffic for one 11008 x 4096
 # 2-bit launch (16,908,288 packed bytes), scaled by packed bytes to the 224 matrices of one pass
 PREFILL_TRAFFIC_BYTES = round(2_833_383_424 * (21_212_160 + 19_456) / 16_908_288)
