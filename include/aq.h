@@ -144,6 +144,35 @@ aq_status_t aq_allocate_bits(const double* S, const int64_t* numel, const int32_
                              double* objective_out);
 
 /*
+ * Attention of one decoded token over a key/value cache, with rotary position embedding: the step between the
+ * projections W_Q, W_K, W_V and W_O of a decoder block (Section 2, "Vision-Language-Action models", names the
+ * projections of every transformer block; the operation between them is the textbook scaled-dot-product attention
+ * and rotary embedding of the LLaMA-style backbone, which the paper does not restate).  Head dimension 128 only.
+ *
+ * Caches are DEVICE arrays [n_kv_heads][L_max][128] of `dtype` (AQ_F16 / AQ_BF16), head-major, owned by the caller.
+ *
+ * aq_rope       rotates, in place, one token's heads x_dev [n_heads][head_dim] (AQ_F16 / AQ_BF16 / AQ_F32; head_dim even):
+ *               pair (i, i + head_dim/2) of every head by the angle pos * theta^(-2 i / head_dim).
+ * aq_kv_append  cache[h][pos][:] = row[h][:] for keys and values (k_dev, v_dev [n_kv_heads][128]; pos < L_max).
+ * aq_attn_decode  out[h] = softmax_p(scale * q[h] . K[h / G][p]) V[h / G][p] over positions p < L, G = n_heads /
+ *               n_kv_heads (1 <= G <= 16) query heads sharing a key/value head.  q_dev [n_heads][128] of `dtype`;
+ *               out_dev [n_heads][128] of out_dtype (any of the three); scale <= 0 means 1/sqrt(128).
+ *               scratch_dev: DEVICE, 256-byte aligned, aq_attn_scratch_bytes(n_kv_heads) bytes, contents irrelevant
+ *               before and after; calls that share it must be ordered on one stream.
+ * Scores and sums are binary32; the softmax weights enter the second product rounded to `dtype`, so against the exact
+ * result an output is off by at most about 2^-10 (AQ_F16; 2^-7 for AQ_BF16) of sum_p softmax_p |V[p]|.
+ * Errors: AQ_ERR_INVALID_ARG (null / misaligned pointer, L not in 1..L_max, n_heads not a multiple of n_kv_heads),
+ * AQ_ERR_UNSUPPORTED (head_dim != 128, G > 16, n_kv_heads > 64, dtype), AQ_ERR_ARCH, AQ_ERR_CUDA.
+ */
+size_t aq_attn_scratch_bytes(int n_kv_heads);
+aq_status_t aq_rope(void* x_dev, int n_heads, int head_dim, int64_t pos, float theta, aq_dtype_t dtype, aq_stream_t stream);
+aq_status_t aq_kv_append(void* k_cache_dev, void* v_cache_dev, const void* k_dev, const void* v_dev, int n_kv_heads,
+                         int head_dim, int64_t pos, int64_t L_max, aq_dtype_t dtype, aq_stream_t stream);
+aq_status_t aq_attn_decode(const void* q_dev, const void* k_cache_dev, const void* v_cache_dev, void* out_dev, int n_heads,
+                           int n_kv_heads, int head_dim, int64_t L, int64_t L_max, float scale, aq_dtype_t dtype,
+                           aq_dtype_t out_dtype, void* scratch_dev, size_t scratch_bytes, aq_stream_t stream);
+
+/*
  * aq_pack_sb / aq_import_sb / aq_export_sb -- the two-level (super-block) form of the format (Section 3, "Weight
  * quantization": every S consecutive blocks form a super-block with its own scale and zero point that compress the
  * per-block parameters).  The paper prints neither S nor the width of the compressed parameters; this library takes

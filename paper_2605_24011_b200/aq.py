@@ -27,6 +27,7 @@ AQ_MAX_M, AQ_DECODE_MAX_M = 4096, 8
 
 SYMBOLS = ("aq_pack", "aq_pack_opt", "aq_pack_sb", "aq_import_sb", "aq_export_sb", "aq_import", "aq_export", "aq_info", "aq_dequant", "aq_linear", "aq_linear_f32out", "aq_linear_noalloc",
            "aq_rbf_gram", "aq_hsic", "aq_sensitivity", "aq_allocate_bits",
+           "aq_attn_scratch_bytes", "aq_rope", "aq_kv_append", "aq_attn_decode",
            "aq_stack_workspace_bytes", "aq_stack_forward", "aq_stack_buffer_offset", "aq_stack_input_offset", "aq_check", "aq_free",
            "aq_set_wait_limit_ns", "aq_debug_decode_hold", "aq_status_string", "aq_last_cuda_error", "aq_kernel_launches")
 
@@ -48,6 +49,15 @@ _lib.aq_pack_opt.argtypes = [C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_int, 
 _lib.aq_pack_opt.restype = C.c_int
 _lib.aq_rbf_gram.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_float, C.c_void_p, C.c_int64, C.c_void_p]
 _lib.aq_rbf_gram.restype = C.c_int
+_lib.aq_attn_scratch_bytes.argtypes = [C.c_int]
+_lib.aq_attn_scratch_bytes.restype = C.c_size_t
+_lib.aq_rope.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int64, C.c_float, C.c_int, C.c_void_p]
+_lib.aq_rope.restype = C.c_int
+_lib.aq_kv_append.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int64, C.c_int64, C.c_int, C.c_void_p]
+_lib.aq_kv_append.restype = C.c_int
+_lib.aq_attn_decode.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int64, C.c_int64,
+                                C.c_float, C.c_int, C.c_int, C.c_void_p, C.c_size_t, C.c_void_p]
+_lib.aq_attn_decode.restype = C.c_int
 _lib.aq_hsic.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p]
 _lib.aq_hsic.restype = C.c_int
 _lib.aq_sensitivity.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_double, C.c_double, C.c_void_p, C.c_void_p]
@@ -185,6 +195,35 @@ def aq_rbf_gram(A, sigma: float, G=None, stream=None):
         G = torch.empty((K, K), dtype=torch.float32, device=A.device)
     _check(_lib.aq_rbf_gram(_ptr(A), dtype_code(A), K, d, float(sigma), _ptr(G), G.stride(0), _stream(stream)), "aq_rbf_gram")
     return G
+
+
+def aq_attn_scratch_bytes(n_kv_heads: int) -> int:
+    return int(_lib.aq_attn_scratch_bytes(int(n_kv_heads)))
+
+
+def aq_rope(x, pos: int, theta: float = 10000.0, stream=None):
+    """x: CUDA [n_heads][head_dim] (float16 / bfloat16 / float32), rotated in place for position pos."""
+    H, D = x.shape
+    _check(_lib.aq_rope(_ptr(x), H, D, int(pos), float(theta), dtype_code(x), _stream(stream)), "aq_rope")
+    return x
+
+
+def aq_kv_append(k_cache, v_cache, k, v, pos: int, stream=None):
+    """k_cache, v_cache: CUDA [n_kv_heads][L_max][head_dim]; k, v: CUDA [n_kv_heads][head_dim] of the same type."""
+    Hkv, Lmax, D = k_cache.shape
+    _check(_lib.aq_kv_append(_ptr(k_cache), _ptr(v_cache), _ptr(k), _ptr(v), Hkv, D, int(pos), Lmax, dtype_code(k_cache),
+                             _stream(stream)), "aq_kv_append")
+
+
+def aq_attn_decode(q, k_cache, v_cache, L: int, out, scratch, scale: float = 0.0, stream=None):
+    """q: CUDA [n_heads][head_dim]; caches [n_kv_heads][L_max][head_dim]; out: CUDA [n_heads][head_dim] (any of the three
+    types); scratch: CUDA uint8 tensor of at least aq_attn_scratch_bytes(n_kv_heads) bytes."""
+    H, D = q.shape
+    Hkv, Lmax, _ = k_cache.shape
+    _check(_lib.aq_attn_decode(_ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(out), H, Hkv, D, int(L), Lmax, float(scale),
+                               dtype_code(q), dtype_code(out), _ptr(scratch), scratch.numel() * scratch.element_size(),
+                               _stream(stream)), "aq_attn_decode")
+    return out
 
 
 def aq_hsic(KA, KB, out=None, stream=None):
