@@ -209,6 +209,23 @@ def run_micro(args):
             fn = lambda i: aq.aq_hsic(Gs[2 * (i % n_copies)], Gs[2 * (i % n_copies) + 1], out=res)
             work, unit = 2.0 * K * K * 4, "GB/s"
         out.update({"K_samples": K, "d": d})
+    elif args.micro == "attn_decode":
+        # one decoded token of a 7B-class block (32 heads of 128) against --K cached positions; HBM-bound on the cache:
+        # 2 (keys, values) x heads x positions x 128 x 2 bytes per call; caches rotate so that L2 does not hold them
+        H, L = 32, args.K or 4096
+        Hkv = args.N or 32                      # (--N: key/value heads, for grouped queries)
+        per = 2 * Hkv * L * 128 * 2
+        n_copies = max(1, int(600e6 // per))
+        g = torch.Generator(device="cuda")
+        g.manual_seed(11)
+        caches = [(torch.randn((Hkv, L, 128), generator=g, device="cuda", dtype=torch.float16),
+                   torch.randn((Hkv, L, 128), generator=g, device="cuda", dtype=torch.float16)) for _ in range(n_copies)]
+        q = torch.randn((H, 128), generator=g, device="cuda", dtype=torch.float16)
+        y = torch.empty((H, 128), dtype=torch.float16, device="cuda")
+        scratch = torch.empty(aq.aq_attn_scratch_bytes(Hkv), dtype=torch.uint8, device="cuda")
+        fn = lambda i: aq.aq_attn_decode(q, caches[i % n_copies][0], caches[i % n_copies][1], L, y, scratch)
+        work, unit = per, "GB/s"
+        out.update({"heads": H, "kv_heads": Hkv, "L": L, "copies": n_copies})
     elif args.micro in ("decode_linear", "prefill_linear", "dequant"):
         decode = args.micro == "decode_linear"
         M = args.M or (1 if decode else 512)
@@ -253,6 +270,28 @@ def run_micro(args):
     aq.aq_check()
     ms = e0.elapsed_time(e1) / args.steps
     out.update({"us_per_call": 1e3 * ms, "value": work / (ms * 1e-3) / (1e9 if unit == "GB/s" else 1e12), "unit": unit})
+    if args.micro == "attn_decode":
+        # the same calls recorded once into a CUDA graph and replayed: device time without the host's per-call cost
+        n = max(16, min(args.steps, 64))
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(graph, stream=side):
+                for i in range(n):
+                    fn(i)
+        torch.cuda.synchronize()
+        for _ in range(3):
+            graph.replay()
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(10):
+            graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        aq.aq_check()
+        msg = e0.elapsed_time(e1) / (10 * n)
+        out.update({"us_per_call_graph": 1e3 * msg, "value_graph": work / (msg * 1e-3) / 1e9})
     print(json.dumps(out))
 
 
@@ -446,7 +485,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
     ap.add_argument("--layers", type=int, default=32, help="decoder layers (32 = the full workload)")
     ap.add_argument("--no-extras", action="store_true", help="skip prefill / dequant / oracle legs")
-    ap.add_argument("--micro", choices=("decode_linear", "prefill_linear", "dequant", "decode_stack", "prefill_stack", "pack", "pack_opt", "rbf_gram", "hsic"),
+    ap.add_argument("--micro", choices=("decode_linear", "prefill_linear", "dequant", "decode_stack", "prefill_stack", "pack", "pack_opt", "rbf_gram", "hsic", "attn_decode"),
                     help="time one kernel on a small case (the command ncu captures are taken from) instead of the benchmark")
     ap.add_argument("--configs", action="store_true",
                     help="time all five workload configurations once each and print one JSON object (not the benchmark line)")

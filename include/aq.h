@@ -158,7 +158,8 @@ aq_status_t aq_allocate_bits(const double* S, const int64_t* numel, const int32_
  *               n_kv_heads (1 <= G <= 16) query heads sharing a key/value head.  q_dev [n_heads][128] of `dtype`;
  *               out_dev [n_heads][128] of out_dtype (any of the three); scale <= 0 means 1/sqrt(128).
  *               scratch_dev: DEVICE, 256-byte aligned, aq_attn_scratch_bytes(n_kv_heads) bytes, contents irrelevant
- *               before and after; calls that share it must be ordered on one stream.
+ *               before and after.  Calls on one device must not overlap in time (they share a small static ticket
+ *               array besides the scratch): keep them on one stream, or order the streams.
  * Scores and sums are binary32; the softmax weights enter the second product rounded to `dtype`, so against the exact
  * result an output is off by at most about 2^-10 (AQ_F16; 2^-7 for AQ_BF16) of sum_p softmax_p |V[p]|.
  * Errors: AQ_ERR_INVALID_ARG (null / misaligned pointer, L not in 1..L_max, n_heads not a multiple of n_kv_heads),

@@ -31,12 +31,15 @@ constexpr int AT_TILE_BYTES = AT_TILE * AT_ROW_BYTES;                  // 8 KB
 constexpr int AT_SMEM = AT_WARPS * AT_STAGES * 2 * AT_TILE_BYTES;      // 192 KB
 constexpr int AT_MAX_SPLITS = 64;
 
+// One ticket per key/value head: zero when the module is loaded, and put back to zero by the CTA that takes the last
+// one, so no launch has to clear them.  Shared by every call on the device: calls must not overlap (one stream at a time).
+__device__ unsigned int g_attn_tickets[64];
+
 struct AttnArgs {
     const void* q;          // [H][D]
     const void* kc;         // [Hkv][Lmax][D]
     const void* vc;
     void* out;              // [H][D]
-    unsigned int* tickets;  // [Hkv], zero before the launch
     float* ml;              // [Hkv][splits][16][2]: running maximum (log2 domain) and sum
     float* part;            // [Hkv][splits][16][D]: unnormalised output
     int64_t L, Lmax;
@@ -93,20 +96,6 @@ __global__ void __launch_bounds__(AT_WARPS * 32, 1) attn_decode_kernel(const Att
     const uint8_t* kc = reinterpret_cast<const uint8_t*>(a.kc) + (int64_t)hk * a.Lmax * AT_ROW_BYTES;
     const uint8_t* vc = reinterpret_cast<const uint8_t*>(a.vc) + (int64_t)hk * a.Lmax * AT_ROW_BYTES;
 
-    // the query heads of this key/value head as the A operand: row r = head hk G + r, rows >= G are zero
-    uint32_t qf[AT_D / 16][4];
-    {
-        const uint16_t* q = reinterpret_cast<const uint16_t*>(a.q) + (int64_t)hk * a.G * AT_D;
-#pragma unroll
-        for (int ks = 0; ks < AT_D / 16; ++ks) {
-            const int d0 = 16 * ks + 2 * t;
-            qf[ks][0] = g < a.G ? *reinterpret_cast<const uint32_t*>(q + g * AT_D + d0) : 0u;
-            qf[ks][1] = g + 8 < a.G ? *reinterpret_cast<const uint32_t*>(q + (g + 8) * AT_D + d0) : 0u;
-            qf[ks][2] = g < a.G ? *reinterpret_cast<const uint32_t*>(q + g * AT_D + d0 + 8) : 0u;
-            qf[ks][3] = g + 8 < a.G ? *reinterpret_cast<const uint32_t*>(q + (g + 8) * AT_D + d0 + 8) : 0u;
-        }
-    }
-
     // copies tile j of this warp (positions pt .. pt + 31) into stage s; rows at or past L are filled with zeros
     auto issue = [&](int j, int s) {
         const int64_t pt = p0 + (int64_t)(warp + AT_WARPS * j) * AT_TILE;
@@ -135,6 +124,21 @@ __global__ void __launch_bounds__(AT_WARPS * 32, 1) attn_decode_kernel(const Att
         if (s < my_tiles) issue(s, s);
         at_commit();
     }
+    // (while the first tiles are on their way) the query heads of this key/value head as the A operand: row r = head
+    // hk G + r, rows >= G are zero
+    uint32_t qf[AT_D / 16][4];
+    {
+        const uint16_t* q = reinterpret_cast<const uint16_t*>(a.q) + (int64_t)hk * a.G * AT_D;
+#pragma unroll
+        for (int ks = 0; ks < AT_D / 16; ++ks) {
+            const int d0 = 16 * ks + 2 * t;
+            qf[ks][0] = g < a.G ? *reinterpret_cast<const uint32_t*>(q + g * AT_D + d0) : 0u;
+            qf[ks][1] = g + 8 < a.G ? *reinterpret_cast<const uint32_t*>(q + (g + 8) * AT_D + d0) : 0u;
+            qf[ks][2] = g < a.G ? *reinterpret_cast<const uint32_t*>(q + g * AT_D + d0 + 8) : 0u;
+            qf[ks][3] = g + 8 < a.G ? *reinterpret_cast<const uint32_t*>(q + (g + 8) * AT_D + d0 + 8) : 0u;
+        }
+    }
+
     for (int j = 0; j < my_tiles; ++j) {
         at_wait<AT_STAGES - 2>();
         __syncwarp();   // every lane's copies of tile j have landed, and every lane is through with tile j - 1
@@ -248,27 +252,46 @@ __global__ void __launch_bounds__(AT_WARPS * 32, 1) attn_decode_kernel(const Att
     __shared__ int is_last;
     __threadfence();
     __syncthreads();
-    if (threadIdx.x == 0) is_last = (atomicAdd(a.tickets + hk, 1u) == (unsigned)n_sp - 1u) ? 1 : 0;
+    if (threadIdx.x == 0) is_last = (atomicAdd(g_attn_tickets + hk, 1u) == (unsigned)n_sp - 1u) ? 1 : 0;
     __syncthreads();
     if (!is_last) return;
     __threadfence();
-    for (int r = 0; r < a.G; ++r) {
+    // all (max, sum) pairs of the head first, in one round of loads; then the partial outputs, eight loads in flight
+    float* s_ml = reinterpret_cast<float*>(smem);   // [split][16][2]
+    for (int i = threadIdx.x; i < n_sp * 32; i += AT_WARPS * 32) s_ml[i] = __ldcg(a.ml + (size_t)hk * n_sp * 32 + i);
+    __syncthreads();
+    // one warp per row (rows warp, warp + 4, ...), four output dimensions per lane
+    for (int r = warp; r < a.G; r += AT_WARPS) {
         float M = -INFINITY;
-        for (int s = 0; s < n_sp; ++s) M = fmaxf(M, __ldcg(a.ml + (((size_t)hk * n_sp + s) * 16 + r) * 2));
-        float acc = 0.f, ls = 0.f;
-        for (int s = 0; s < n_sp; ++s) {
-            const size_t sl = (size_t)hk * n_sp + s;
-            const float wgt = exp2f(__ldcg(a.ml + (sl * 16 + r) * 2) - M);
-            acc = fmaf(wgt, __ldcg(a.part + (sl * 16 + r) * AT_D + d), acc);
-            ls = fmaf(wgt, __ldcg(a.ml + (sl * 16 + r) * 2 + 1), ls);
+        for (int s = 0; s < n_sp; ++s) M = fmaxf(M, s_ml[(s * 16 + r) * 2]);
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        float ls = 0.f;
+        const float4* pr = reinterpret_cast<const float4*>(a.part + ((size_t)hk * n_sp * 16 + r) * AT_D) + lane;
+        for (int s0 = 0; s0 < n_sp; s0 += 8) {
+            float4 v[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) v[i] = (s0 + i < n_sp) ? __ldcg(pr + (size_t)(s0 + i) * 16 * (AT_D / 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                if (s0 + i < n_sp) {
+                    const float wgt = exp2f(s_ml[((s0 + i) * 16 + r) * 2] - M);
+                    acc.x = fmaf(wgt, v[i].x, acc.x); acc.y = fmaf(wgt, v[i].y, acc.y);
+                    acc.z = fmaf(wgt, v[i].z, acc.z); acc.w = fmaf(wgt, v[i].w, acc.w);
+                    ls = fmaf(wgt, s_ml[((s0 + i) * 16 + r) * 2 + 1], ls);
+                }
+            }
         }
-        const float v = acc / ls;
-        const size_t oi = ((size_t)hk * a.G + r) * AT_D + d;
-        if (a.out_dtype == AQ_F32) reinterpret_cast<float*>(a.out)[oi] = v;
-        else if (a.out_dtype == AQ_F16) reinterpret_cast<__half*>(a.out)[oi] = __float2half_rn(v);
-        else reinterpret_cast<__nv_bfloat16*>(a.out)[oi] = __float2bfloat16_rn(v);
+        const float inv = 1.f / ls;
+        const float o4[4] = {acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv};
+        const size_t oi = ((size_t)hk * a.G + r) * AT_D + 4 * lane;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            if (a.out_dtype == AQ_F32) reinterpret_cast<float*>(a.out)[oi + i] = o4[i];
+            else if (a.out_dtype == AQ_F16) reinterpret_cast<__half*>(a.out)[oi + i] = __float2half_rn(o4[i]);
+            else reinterpret_cast<__nv_bfloat16*>(a.out)[oi + i] = __float2bfloat16_rn(o4[i]);
+        }
     }
-    if (threadIdx.x == 0) a.tickets[hk] = 0u;
+    if (threadIdx.x == 0) g_attn_tickets[hk] = 0u;
 }
 
 // ---- rotary embedding and cache append -----------------------------------------------------------------------
@@ -307,8 +330,9 @@ __global__ void kv_append_kernel(uint4* kc, uint4* vc, const uint4* k, const uin
 
 // ---- host ---------------------------------------------------------------------------------------------------
 static int attn_max_splits(int n_kv) {
-    // about two CTAs per SM over all heads
-    int want = (2 * sm_count() + n_kv - 1) / n_kv;
+    // one CTA per SM fits (its rings take most of the shared memory), so one wave: as many splits as keep the grid
+    // inside the SM count
+    int want = sm_count() / n_kv;
     if (want < 1) want = 1;
     return want > AT_MAX_SPLITS ? AT_MAX_SPLITS : want;
 }
@@ -334,13 +358,10 @@ cudaError_t launch_attn_decode(const void* q, const void* kc, const void* vc, vo
     AttnArgs a;
     a.q = q; a.kc = kc; a.vc = vc; a.out = out;
     uint8_t* sc = reinterpret_cast<uint8_t*>(scratch);
-    a.tickets = reinterpret_cast<unsigned int*>(sc);                                  // (n_kv <= 64: inside the first 256 bytes)
     a.ml = reinterpret_cast<float*>(sc + 256);
     a.part = reinterpret_cast<float*>(sc + 256 + (size_t)n_kv * AT_MAX_SPLITS * 16 * 2 * sizeof(float));
     a.L = L; a.Lmax = Lmax; a.G = n_heads / n_kv; a.chunk = chunk; a.out_dtype = (int)out_dt;
     a.scale_log2 = scale * 1.4426950408889634f;
-    cudaError_t e = cudaMemsetAsync(a.tickets, 0, 256, s);
-    if (e != cudaSuccess) return e;
     const bool bf = (dt == AQ_BF16);
     static PerDeviceOnce configured[2];
     {
