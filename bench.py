@@ -598,6 +598,7 @@ def main():
     if world == 1 and rank == 0 and not args.no_extras:
         line["prefill"] = prefill_leg(aq, workloads, prog, out_buf, info, peaks, torch, local)
         line["dequant"] = dequant_leg(aq, synth, peaks, torch)
+        line["attn_decode"] = attn_leg(aq, peaks, torch)
         if args.layers == 32:
             line["configs"] = configs_leg(peaks, torch, prog, out_buf, info)
         cores = len(os.sched_getaffinity(0))
@@ -657,6 +658,45 @@ def prefill_leg(aq, workloads, prog, out_buf, info, peaks, torch, gpu_index=0):
                          "traffic": PREFILL_TRAFFIC_BYTES, "traffic_note": "dram bytes of the one-launch ncu capture (11008 x 4096) scaled by packed bytes to the pass",
                          "peak_source": peaks["source"] + " (burst peak: the leg lasts about 0.2 s)",
                          "kernel": "gemm_kernel (128 grouped launches per pass; time = whole pass incl. staging kernels)"}}
+
+
+def attn_leg(aq, peaks, torch):
+    """One decoded token's attention over a key/value cache (32 heads of 128, fp16) at 4096 and 16384 positions: HBM-bound
+    on the cache bytes; the calls are replayed from a CUDA graph (device time), caches rotate past L2."""
+    g = torch.Generator(device="cuda")
+    g.manual_seed(11)
+    H = 32
+    q = torch.randn((H, 128), generator=g, device="cuda", dtype=torch.float16)
+    y = torch.empty((H, 128), dtype=torch.float16, device="cuda")
+    scratch = torch.empty(aq.aq_attn_scratch_bytes(H), dtype=torch.uint8, device="cuda")
+    out = {"workload": "aq_attn_decode, 32 heads of 128, fp16, one token against L cached positions, caches cold (in rotation)"}
+    for L in (4096, 16384):
+        per = 2 * H * L * 128 * 2
+        n = max(2, int(600e6 // per))
+        caches = [(torch.randn((H, L, 128), generator=g, device="cuda", dtype=torch.float16),
+                   torch.randn((H, L, 128), generator=g, device="cuda", dtype=torch.float16)) for _ in range(n)]
+        calls = 4 * n
+        fn = lambda i: aq.aq_attn_decode(q, caches[i % n][0], caches[i % n][1], L, y, scratch)
+        for i in range(n):
+            fn(i)
+        torch.cuda.synchronize()
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(graph, stream=side):
+                for i in range(calls):
+                    fn(i)
+        torch.cuda.synchronize()
+        us = 1e3 * _timed(graph.replay, 10, 3, torch) / (10 * calls)
+        aq.aq_check()
+        gbs = per / us / 1e3
+        out[f"L{L}"] = {"us_per_call": us, "gbs": gbs,
+                        "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
+                                     "traffic": 67_174_656 + 485_376 if L == 4096 else None, "peak_source": peaks["source"],
+                                     "kernel": "attn_decode_kernel"}}
+        del caches
+    return out
 
 
 def dequant_leg(aq, synth, peaks, torch):
