@@ -71,3 +71,18 @@ def attn_bound(q: np.ndarray, K: np.ndarray, V: np.ndarray, L: int, scale: float
     P = _scores(q, K, L, scale, G)
     V = np.abs(np.asarray(V, dtype=np.float64))
     return np.stack([P[h] @ V[h // G, :L, :] for h in range(H)])
+
+
+def attn_decode_tokens(q: np.ndarray, K: np.ndarray, V: np.ndarray, L: int, scale: float | None = None) -> np.ndarray:
+    """Several new tokens at once (the last M of the L cached positions are theirs): q [M][H][D]; token m sees positions
+    0 .. L - M + m (itself and everything before it: causal attention).  Returns float64 [M][H][D]."""
+    q = np.asarray(q)
+    M = q.shape[0]
+    assert 1 <= M <= L
+    return np.stack([attn_decode(q[m], K, V, L - (M - 1 - m), scale) for m in range(M)])
+
+
+def attn_bound_tokens(q: np.ndarray, K: np.ndarray, V: np.ndarray, L: int, scale: float | None = None) -> np.ndarray:
+    q = np.asarray(q)
+    M = q.shape[0]
+    return np.stack([attn_bound(q[m], K, V, L - (M - 1 - m), scale) for m in range(M)])

@@ -139,3 +139,30 @@ def test_attention_bound():
     T = A.attn_bound(q, K, V, 6)
     assert np.all(T >= np.abs(A.attn_decode(q, K, V, 6)) - 1e-15)
     assert np.allclose(A.attn_bound(q, K, np.abs(V), 6), A.attn_decode(q, K, np.abs(V), 6))
+
+
+def test_attention_of_several_new_tokens_is_causal():
+    g = _rng(7)
+    M, H, Hkv, D, Lmax, L = 3, 4, 2, 6, 12, 9
+    q = g.standard_normal((M, H, D))
+    K = g.standard_normal((Hkv, Lmax, D))
+    V = g.standard_normal((Hkv, Lmax, D))
+    out = A.attn_decode_tokens(q, K, V, L)
+    assert out.shape == (M, H, D)
+    # brute force: token m sees positions 0 .. L - M + m
+    for m in range(M):
+        ref = _brute(q[m].tolist(), K.tolist(), V.tolist(), L - (M - 1 - m), 1.0 / math.sqrt(D))
+        assert np.allclose(out[m], np.array(ref), atol=1e-13)
+    # the last token is the single-token case; the first one sees M - 1 positions fewer
+    assert np.array_equal(out[M - 1], A.attn_decode(q[M - 1], K, V, L))
+    assert np.array_equal(out[0], A.attn_decode(q[0], K, V, L - M + 1))
+    # what comes after a token does not reach it: changing the last position changes the last token only
+    K2, V2 = K.copy(), V.copy()
+    K2[:, L - 1] += 1.0
+    V2[:, L - 1] -= 2.0
+    out2 = A.attn_decode_tokens(q, K2, V2, L)
+    assert np.array_equal(out2[: M - 1], out[: M - 1]) and not np.allclose(out2[M - 1], out[M - 1])
+    # one token: the plain function
+    assert np.array_equal(A.attn_decode_tokens(q[:1], K, V, L)[0], A.attn_decode(q[0], K, V, L))
+    T = A.attn_bound_tokens(q, K, V, L)
+    assert T.shape == out.shape and np.all(T >= np.abs(out) - 1e-15)
