@@ -154,22 +154,25 @@ aq_status_t aq_allocate_bits(const double* S, const int64_t* numel, const int32_
  * aq_rope       rotates, in place, one token's heads x_dev [n_heads][head_dim] (AQ_F16 / AQ_BF16 / AQ_F32; head_dim even):
  *               pair (i, i + head_dim/2) of every head by the angle pos * theta^(-2 i / head_dim).
  * aq_kv_append  cache[h][pos][:] = row[h][:] for keys and values (k_dev, v_dev [n_kv_heads][128]; pos < L_max).
- * aq_attn_decode  out[h] = softmax_p(scale * q[h] . K[h / G][p]) V[h / G][p] over positions p < L, G = n_heads /
- *               n_kv_heads (1 <= G <= 16) query heads sharing a key/value head.  q_dev [n_heads][128] of `dtype`;
- *               out_dev [n_heads][128] of out_dtype (any of the three); scale <= 0 means 1/sqrt(128).
+ * aq_attn_decode  out[m][h] = softmax_p(scale * q[m][h] . K[h / G][p]) V[h / G][p] for M new tokens whose keys and
+ *               values are the last M of the L cached positions: token m sees positions p <= L - M + m (itself and
+ *               everything before it).  G = n_heads / n_kv_heads query heads share a key/value head; G * M <= 16
+ *               (with 32 heads of their own: 1 <= M <= 16; AQ_DECODE_MAX_M tokens need G <= 2).  q_dev
+ *               [M][n_heads][128] of `dtype`; out_dev [M][n_heads][128] of out_dtype (any of the three); scale <= 0
+ *               means 1/sqrt(128).
  *               scratch_dev: DEVICE, 256-byte aligned, aq_attn_scratch_bytes(n_kv_heads) bytes, contents irrelevant
  *               before and after.  Calls on one device must not overlap in time (they share a small static ticket
  *               array besides the scratch): keep them on one stream, or order the streams.
  * Scores and sums are binary32; the softmax weights enter the second product rounded to `dtype`, so against the exact
  * result an output is off by at most about 2^-10 (AQ_F16; 2^-7 for AQ_BF16) of sum_p softmax_p |V[p]|.
- * Errors: AQ_ERR_INVALID_ARG (null / misaligned pointer, L not in 1..L_max, n_heads not a multiple of n_kv_heads),
- * AQ_ERR_UNSUPPORTED (head_dim != 128, G > 16, n_kv_heads > 64, dtype), AQ_ERR_ARCH, AQ_ERR_CUDA.
+ * Errors: AQ_ERR_INVALID_ARG (null / misaligned pointer, M < 1, L not in M..L_max, n_heads not a multiple of
+ * n_kv_heads), AQ_ERR_UNSUPPORTED (head_dim != 128, G * M > 16, n_kv_heads > 64, dtype), AQ_ERR_ARCH, AQ_ERR_CUDA.
  */
 size_t aq_attn_scratch_bytes(int n_kv_heads);
 aq_status_t aq_rope(void* x_dev, int n_heads, int head_dim, int64_t pos, float theta, aq_dtype_t dtype, aq_stream_t stream);
 aq_status_t aq_kv_append(void* k_cache_dev, void* v_cache_dev, const void* k_dev, const void* v_dev, int n_kv_heads,
                          int head_dim, int64_t pos, int64_t L_max, aq_dtype_t dtype, aq_stream_t stream);
-aq_status_t aq_attn_decode(const void* q_dev, const void* k_cache_dev, const void* v_cache_dev, void* out_dev, int n_heads,
+aq_status_t aq_attn_decode(const void* q_dev, const void* k_cache_dev, const void* v_cache_dev, void* out_dev, int M, int n_heads,
                            int n_kv_heads, int head_dim, int64_t L, int64_t L_max, float scale, aq_dtype_t dtype,
                            aq_dtype_t out_dtype, void* scratch_dev, size_t scratch_bytes, aq_stream_t stream);
 

@@ -55,7 +55,7 @@ _lib.aq_rope.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int64, C.c_float, C.c
 _lib.aq_rope.restype = C.c_int
 _lib.aq_kv_append.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int64, C.c_int64, C.c_int, C.c_void_p]
 _lib.aq_kv_append.restype = C.c_int
-_lib.aq_attn_decode.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int64, C.c_int64,
+_lib.aq_attn_decode.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int64, C.c_int64,
                                 C.c_float, C.c_int, C.c_int, C.c_void_p, C.c_size_t, C.c_void_p]
 _lib.aq_attn_decode.restype = C.c_int
 _lib.aq_hsic.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p]
@@ -216,11 +216,13 @@ def aq_kv_append(k_cache, v_cache, k, v, pos: int, stream=None):
 
 
 def aq_attn_decode(q, k_cache, v_cache, L: int, out, scratch, scale: float = 0.0, stream=None):
-    """q: CUDA [n_heads][head_dim]; caches [n_kv_heads][L_max][head_dim]; out: CUDA [n_heads][head_dim] (any of the three
-    types); scratch: CUDA uint8 tensor of at least aq_attn_scratch_bytes(n_kv_heads) bytes."""
-    H, D = q.shape
+    """q: CUDA [n_heads][head_dim] (one new token) or [M][n_heads][head_dim] (M new tokens, the last M of the L cached
+    positions, each seeing the positions up to its own); caches [n_kv_heads][L_max][head_dim]; out: CUDA, the shape of
+    q, any of the three types; scratch: CUDA uint8 tensor of at least aq_attn_scratch_bytes(n_kv_heads) bytes."""
+    M = 1 if q.dim() == 2 else q.shape[0]
+    H, D = q.shape[-2], q.shape[-1]
     Hkv, Lmax, _ = k_cache.shape
-    _check(_lib.aq_attn_decode(_ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(out), H, Hkv, D, int(L), Lmax, float(scale),
+    _check(_lib.aq_attn_decode(_ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(out), M, H, Hkv, D, int(L), Lmax, float(scale),
                                dtype_code(q), dtype_code(out), _ptr(scratch), scratch.numel() * scratch.element_size(),
                                _stream(stream)), "aq_attn_decode")
     return out

@@ -405,23 +405,23 @@ aq_status_t aq_kv_append(void* k_cache_dev, void* v_cache_dev, const void* k_dev
     return e == cudaSuccess ? AQ_OK : cuda_fail(e);
 }
 
-aq_status_t aq_attn_decode(const void* q_dev, const void* k_cache_dev, const void* v_cache_dev, void* out_dev, int n_heads,
+aq_status_t aq_attn_decode(const void* q_dev, const void* k_cache_dev, const void* v_cache_dev, void* out_dev, int M, int n_heads,
                            int n_kv_heads, int head_dim, int64_t L, int64_t L_max, float scale, aq_dtype_t dtype,
                            aq_dtype_t out_dtype, void* scratch_dev, size_t scratch_bytes, aq_stream_t stream) {
     if (!q_dev || !k_cache_dev || !v_cache_dev || !out_dev || !scratch_dev || !aligned16(q_dev) || !aligned16(k_cache_dev) ||
         !aligned16(v_cache_dev) || !aligned16(out_dev) || (reinterpret_cast<uintptr_t>(scratch_dev) & 255u))
         return AQ_ERR_INVALID_ARG;
-    if (n_heads < 1 || n_kv_heads < 1 || n_heads % n_kv_heads != 0 || L < 1 || L > L_max || L_max > ((int64_t)1 << 31) ||
+    if (M < 1 || n_heads < 1 || n_kv_heads < 1 || n_heads % n_kv_heads != 0 || L < M || L > L_max || L_max > ((int64_t)1 << 31) ||
         !std::isfinite(scale))
         return AQ_ERR_INVALID_ARG;
     if (dtype != AQ_F16 && dtype != AQ_BF16) return (dtype == AQ_F32) ? AQ_ERR_UNSUPPORTED : AQ_ERR_INVALID_ARG;
     if (out_dtype != AQ_F16 && out_dtype != AQ_BF16 && out_dtype != AQ_F32) return AQ_ERR_INVALID_ARG;
-    if (head_dim != 128 || n_heads / n_kv_heads > 16 || n_kv_heads > 64) return AQ_ERR_UNSUPPORTED;
+    if (head_dim != 128 || (int64_t)(n_heads / n_kv_heads) * M > 16 || n_kv_heads > 64) return AQ_ERR_UNSUPPORTED;
     aq_status_t st = check_arch(nullptr);
     if (st != AQ_OK) return st;
     if (scratch_bytes < attn_scratch_bytes(n_kv_heads)) return AQ_ERR_INVALID_ARG;
     if (!(scale > 0.f)) scale = 0.08838834764831845f;   // 1 / sqrt(128)
-    const cudaError_t e = launch_attn_decode(q_dev, k_cache_dev, v_cache_dev, out_dev, n_heads, n_kv_heads, L, L_max, scale, dtype,
+    const cudaError_t e = launch_attn_decode(q_dev, k_cache_dev, v_cache_dev, out_dev, M, n_heads, n_kv_heads, L, L_max, scale, dtype,
                                              out_dtype, scratch_dev, (cudaStream_t)stream);
     return e == cudaSuccess ? AQ_OK : cuda_fail(e);
 }

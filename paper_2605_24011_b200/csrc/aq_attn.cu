@@ -36,14 +36,16 @@ constexpr int AT_MAX_SPLITS = 64;
 __device__ unsigned int g_attn_tickets[64];
 
 struct AttnArgs {
-    const void* q;          // [H][D]
+    const void* q;          // [M][H][D]
     const void* kc;         // [Hkv][Lmax][D]
     const void* vc;
-    void* out;              // [H][D]
+    void* out;              // [M][H][D]
     float* ml;              // [Hkv][splits][16][2]: running maximum (log2 domain) and sum
     float* part;            // [Hkv][splits][16][D]: unnormalised output
     int64_t L, Lmax;
     int G;                  // query heads per key/value head
+    int M;                  // new tokens (the last M of the L positions are theirs); G * M <= 16 rows
+    int H;                  // query heads in all (row pitch of q and out)
     int chunk;              // positions per split (a multiple of AT_TILE)
     int out_dtype;          // aq_dtype_t of out
     float scale_log2;       // scale * log2(e)
@@ -126,19 +128,25 @@ __global__ void __launch_bounds__(AT_WARPS * 32, 1) attn_decode_kernel(const Att
     }
     // (while the first tiles are on their way) the query heads of this key/value head as the A operand: row r = head
     // hk G + r, rows >= G are zero
+    // row r = token r / G, head hk G + r % G of that token; rows >= G M are zero
+    const int R = a.G * a.M;
+    const int tok0 = g / a.G, tok1 = (g + 8) / a.G;
     uint32_t qf[AT_D / 16][4];
     {
-        const uint16_t* q = reinterpret_cast<const uint16_t*>(a.q) + (int64_t)hk * a.G * AT_D;
+        const uint16_t* q = reinterpret_cast<const uint16_t*>(a.q);
+        const uint16_t* q0 = q + ((int64_t)tok0 * a.H + (int64_t)hk * a.G + (g - tok0 * a.G)) * AT_D;
+        const uint16_t* q1 = q + ((int64_t)tok1 * a.H + (int64_t)hk * a.G + (g + 8 - tok1 * a.G)) * AT_D;
 #pragma unroll
         for (int ks = 0; ks < AT_D / 16; ++ks) {
             const int d0 = 16 * ks + 2 * t;
-            qf[ks][0] = g < a.G ? *reinterpret_cast<const uint32_t*>(q + g * AT_D + d0) : 0u;
-            qf[ks][1] = g + 8 < a.G ? *reinterpret_cast<const uint32_t*>(q + (g + 8) * AT_D + d0) : 0u;
-            qf[ks][2] = g < a.G ? *reinterpret_cast<const uint32_t*>(q + g * AT_D + d0 + 8) : 0u;
-            qf[ks][3] = g + 8 < a.G ? *reinterpret_cast<const uint32_t*>(q + (g + 8) * AT_D + d0 + 8) : 0u;
+            qf[ks][0] = g < R ? *reinterpret_cast<const uint32_t*>(q0 + d0) : 0u;
+            qf[ks][1] = g + 8 < R ? *reinterpret_cast<const uint32_t*>(q1 + d0) : 0u;
+            qf[ks][2] = g < R ? *reinterpret_cast<const uint32_t*>(q0 + d0 + 8) : 0u;
+            qf[ks][3] = g + 8 < R ? *reinterpret_cast<const uint32_t*>(q1 + d0 + 8) : 0u;
         }
     }
-
+    // a token sees the positions up to its own: token m of M up to L - M + m (rows past the last one: any limit will do)
+    const int64_t lim0 = a.L - (a.M - 1 - min(tok0, a.M - 1)), lim1 = a.L - (a.M - 1 - min(tok1, a.M - 1));
     for (int j = 0; j < my_tiles; ++j) {
         at_wait<AT_STAGES - 2>();
         __syncwarp();   // every lane's copies of tile j have landed, and every lane is through with tile j - 1
@@ -166,24 +174,26 @@ __global__ void __launch_bounds__(AT_WARPS * 32, 1) attn_decode_kernel(const Att
 #pragma unroll
         for (int nt = 0; nt < 4; ++nt) {
             const int64_t pc = pt + 8 * nt + 2 * t;
-            const bool v0 = pc < a.L, v1 = pc + 1 < a.L;
-            sc[nt][0] = v0 ? sc[nt][0] * a.scale_log2 : -INFINITY;
-            sc[nt][1] = v1 ? sc[nt][1] * a.scale_log2 : -INFINITY;
-            sc[nt][2] = v0 ? sc[nt][2] * a.scale_log2 : -INFINITY;
-            sc[nt][3] = v1 ? sc[nt][3] * a.scale_log2 : -INFINITY;
+            sc[nt][0] = pc < lim0 ? sc[nt][0] * a.scale_log2 : -INFINITY;
+            sc[nt][1] = pc + 1 < lim0 ? sc[nt][1] * a.scale_log2 : -INFINITY;
+            sc[nt][2] = pc < lim1 ? sc[nt][2] * a.scale_log2 : -INFINITY;
+            sc[nt][3] = pc + 1 < lim1 ? sc[nt][3] * a.scale_log2 : -INFINITY;
             mx0 = fmaxf(mx0, fmaxf(sc[nt][0], sc[nt][1]));
             mx1 = fmaxf(mx1, fmaxf(sc[nt][2], sc[nt][3]));
         }
         mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1)); mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
         mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1)); mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
-        const float n0 = fmaxf(m0, mx0), n1 = fmaxf(m1, mx1);   // finite: the tile's first position is inside L
-        const float a0 = exp2f(m0 - n0), a1 = exp2f(m1 - n1);
+        // (a row that has seen nothing yet, its limit lying before this warp's first tiles, keeps -inf: the exponentials
+        // below are then taken against 0 and come out as 0)
+        const float n0 = fmaxf(m0, mx0), n1 = fmaxf(m1, mx1);
+        const float b0 = n0 == -INFINITY ? 0.f : n0, b1 = n1 == -INFINITY ? 0.f : n1;
+        const float a0 = exp2f(m0 - b0), a1 = exp2f(m1 - b1);
         m0 = n0; m1 = n1;
         float s0 = 0.f, s1 = 0.f;
 #pragma unroll
         for (int nt = 0; nt < 4; ++nt) {
-            sc[nt][0] = exp2f(sc[nt][0] - n0); sc[nt][1] = exp2f(sc[nt][1] - n0);
-            sc[nt][2] = exp2f(sc[nt][2] - n1); sc[nt][3] = exp2f(sc[nt][3] - n1);
+            sc[nt][0] = exp2f(sc[nt][0] - b0); sc[nt][1] = exp2f(sc[nt][1] - b0);
+            sc[nt][2] = exp2f(sc[nt][2] - b1); sc[nt][3] = exp2f(sc[nt][3] - b1);
             s0 += sc[nt][0] + sc[nt][1];
             s1 += sc[nt][2] + sc[nt][3];
         }
@@ -233,14 +243,15 @@ __global__ void __launch_bounds__(AT_WARPS * 32, 1) attn_decode_kernel(const Att
     __syncthreads();
     const int d = threadIdx.x;   // 128 threads: one output dimension each
     const size_t slot = (size_t)hk * n_sp + sp;
-    for (int r = 0; r < a.G; ++r) {
+    for (int r = 0; r < R; ++r) {
         float M = -INFINITY;
 #pragma unroll
         for (int w = 0; w < AT_WARPS; ++w) M = fmaxf(M, sm_m[w * 16 + r]);
+        const float Mb = M == -INFINITY ? 0.f : M;   // (a row that saw nothing in this split: all weights 0)
         float acc = 0.f, ls = 0.f;
 #pragma unroll
         for (int w = 0; w < AT_WARPS; ++w) {   // (a warp without tiles has maximum -inf and weight 0)
-            const float wgt = exp2f(sm_m[w * 16 + r] - M);
+            const float wgt = exp2f(sm_m[w * 16 + r] - Mb);
             acc = fmaf(wgt, sm_o[((size_t)w * 16 + r) * AT_D + d], acc);
             ls = fmaf(wgt, sm_l[w * 16 + r], ls);
         }
@@ -261,8 +272,8 @@ __global__ void __launch_bounds__(AT_WARPS * 32, 1) attn_decode_kernel(const Att
     for (int i = threadIdx.x; i < n_sp * 32; i += AT_WARPS * 32) s_ml[i] = __ldcg(a.ml + (size_t)hk * n_sp * 32 + i);
     __syncthreads();
     // one warp per row (rows warp, warp + 4, ...), four output dimensions per lane
-    for (int r = warp; r < a.G; r += AT_WARPS) {
-        float M = -INFINITY;
+    for (int r = warp; r < R; r += AT_WARPS) {
+        float M = -INFINITY;   // finite in the end: every token sees position 0, which the first split holds
         for (int s = 0; s < n_sp; ++s) M = fmaxf(M, s_ml[(s * 16 + r) * 2]);
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         float ls = 0.f;
@@ -283,7 +294,8 @@ __global__ void __launch_bounds__(AT_WARPS * 32, 1) attn_decode_kernel(const Att
         }
         const float inv = 1.f / ls;
         const float o4[4] = {acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv};
-        const size_t oi = ((size_t)hk * a.G + r) * AT_D + 4 * lane;
+        const int tok = r / a.G;
+        const size_t oi = ((size_t)tok * a.H + (size_t)hk * a.G + (r - tok * a.G)) * AT_D + 4 * lane;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             if (a.out_dtype == AQ_F32) reinterpret_cast<float*>(a.out)[oi + i] = o4[i];
@@ -351,7 +363,7 @@ size_t attn_scratch_bytes(int n_kv) {
     return 256 + (size_t)n_kv * AT_MAX_SPLITS * 16 * 2 * sizeof(float) + (size_t)n_kv * attn_max_splits(n_kv) * 16 * AT_D * sizeof(float) + 256;
 }
 
-cudaError_t launch_attn_decode(const void* q, const void* kc, const void* vc, void* out, int n_heads, int n_kv, int64_t L,
+cudaError_t launch_attn_decode(const void* q, const void* kc, const void* vc, void* out, int M, int n_heads, int n_kv, int64_t L,
                                int64_t Lmax, float scale, aq_dtype_t dt, aq_dtype_t out_dt, void* scratch, cudaStream_t s) {
     int splits, chunk;
     attn_geometry(n_kv, L, &splits, &chunk);
@@ -360,7 +372,7 @@ cudaError_t launch_attn_decode(const void* q, const void* kc, const void* vc, vo
     uint8_t* sc = reinterpret_cast<uint8_t*>(scratch);
     a.ml = reinterpret_cast<float*>(sc + 256);
     a.part = reinterpret_cast<float*>(sc + 256 + (size_t)n_kv * AT_MAX_SPLITS * 16 * 2 * sizeof(float));
-    a.L = L; a.Lmax = Lmax; a.G = n_heads / n_kv; a.chunk = chunk; a.out_dtype = (int)out_dt;
+    a.L = L; a.Lmax = Lmax; a.G = n_heads / n_kv; a.M = M; a.H = n_heads; a.chunk = chunk; a.out_dtype = (int)out_dt;
     a.scale_log2 = scale * 1.4426950408889634f;
     const bool bf = (dt == AQ_BF16);
     static PerDeviceOnce configured[2];

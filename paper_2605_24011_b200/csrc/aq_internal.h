@@ -132,7 +132,7 @@ int read_stage1_status(bool clear);
 
 // single-token attention over a key/value cache (aq_attn.cu); head dimension 128
 size_t attn_scratch_bytes(int n_kv);
-cudaError_t launch_attn_decode(const void* q, const void* kc, const void* vc, void* out, int n_heads, int n_kv, int64_t L,
+cudaError_t launch_attn_decode(const void* q, const void* kc, const void* vc, void* out, int M, int n_heads, int n_kv, int64_t L,
                                int64_t Lmax, float scale, aq_dtype_t dt, aq_dtype_t out_dt, void* scratch, cudaStream_t s);
 cudaError_t launch_rope(void* x, int n_heads, int D, int64_t pos, float theta, aq_dtype_t dt, cudaStream_t s);
 cudaError_t launch_kv_append(void* kc, void* vc, const void* k, const void* v, int n_kv, int D, int64_t pos, int64_t Lmax, cudaStream_t s);

@@ -132,14 +132,16 @@ def test_attention_rejects_bad_arguments(aq):
     kc = torch.zeros((32, 64, 128), dtype=torch.float16, device="cuda")
     out = torch.zeros((32, 128), dtype=torch.float32, device="cuda")
     sc = torch.zeros(aq.aq_attn_scratch_bytes(32), dtype=torch.uint8, device="cuda")
-    def call(H=32, Hkv=32, D=128, L=10, Lmax=64, dt=aq.AQ_F16, odt=aq.AQ_F32, nbytes=None, qp=None):
-        return lib.aq_attn_decode(qp if qp is not None else q.data_ptr(), kc.data_ptr(), kc.data_ptr(), out.data_ptr(), H, Hkv, D, L, Lmax,
+    def call(H=32, Hkv=32, D=128, L=10, Lmax=64, dt=aq.AQ_F16, odt=aq.AQ_F32, nbytes=None, qp=None, M=1):
+        return lib.aq_attn_decode(qp if qp is not None else q.data_ptr(), kc.data_ptr(), kc.data_ptr(), out.data_ptr(), M, H, Hkv, D, L, Lmax,
                                   0.0, dt, odt, sc.data_ptr(), sc.numel() if nbytes is None else nbytes, None)
     assert call() == aq.AQ_OK
     assert call(L=0) == aq.AQ_ERR_INVALID_ARG and call(L=65) == aq.AQ_ERR_INVALID_ARG
     assert call(H=33) == aq.AQ_ERR_INVALID_ARG                  # not a multiple of the key/value heads
     assert call(D=64) == aq.AQ_ERR_UNSUPPORTED
     assert call(H=34, Hkv=2) == aq.AQ_ERR_UNSUPPORTED           # 17 query heads per key/value head
+    assert call(H=8, Hkv=4, M=9) == aq.AQ_ERR_UNSUPPORTED       # 2 x 9 rows
+    assert call(M=0) == aq.AQ_ERR_INVALID_ARG and call(M=4, L=3) == aq.AQ_ERR_INVALID_ARG
     assert call(dt=aq.AQ_F32) == aq.AQ_ERR_UNSUPPORTED
     assert call(nbytes=1024) == aq.AQ_ERR_INVALID_ARG
     assert call(qp=q.data_ptr() + 2) == aq.AQ_ERR_INVALID_ARG
@@ -147,3 +149,26 @@ def test_attention_rejects_bad_arguments(aq):
     assert lib.aq_rope(q.data_ptr(), 32, 127, 3, 10000.0, aq.AQ_F16, None) == aq.AQ_ERR_INVALID_ARG
     torch.cuda.synchronize()
     aq.aq_check()
+
+
+@pytest.mark.parametrize("name", ("f16", "bf16"))
+def test_attention_of_several_new_tokens(aq, name):
+    """M new tokens in one call (the decode path's 1..8, and up to 16 rows of heads x tokens): each sees the positions up
+    to its own.  Includes contexts shorter than a tile, so that some rows see nothing in some warps' tiles."""
+    for M, H, Hkv, L, Lmax in ((8, 32, 32, 1000, 1024), (16, 32, 32, 4096, 4096), (8, 16, 8, 333, 512), (4, 32, 8, 2049, 4096),
+                               (3, 8, 8, 3, 64), (8, 8, 8, 9, 64), (2, 64, 8, 130, 256), (5, 6, 2, 37, 40)):
+        g = np.random.default_rng(50 + M + L)
+        tdt = TD[name]
+        q = torch.from_numpy(g.standard_normal((M, H, 128)).astype(np.float32)).to(tdt)
+        K = torch.from_numpy(g.standard_normal((Hkv, Lmax, 128)).astype(np.float32)).to(tdt)
+        V = torch.from_numpy(g.standard_normal((Hkv, Lmax, 128)).astype(np.float32)).to(tdt)
+        scratch = torch.empty(aq.aq_attn_scratch_bytes(Hkv), dtype=torch.uint8, device="cuda")
+        out = torch.full((M, H, 128), float("nan"), dtype=torch.float32, device="cuda")
+        aq.aq_attn_decode(q.cuda(), K.cuda(), V.cuda(), L, out, scratch)
+        aq.aq_check()
+        qn, Kn, Vn = q.double().numpy(), K.double().numpy(), V.double().numpy()
+        ref, T = A.attn_decode_tokens(qn, Kn, Vn, L), A.attn_bound_tokens(qn, Kn, Vn, L)
+        got = out.double().cpu().numpy()
+        assert np.all(np.isfinite(got))
+        tol = (U[name] + 2.0 ** -16) * T + 1e-6
+        assert np.all(np.abs(got - ref) <= tol), f"M={M} H={H} Hkv={Hkv} L={L} {name}: worst {np.max(np.abs(got - ref) / tol):.3f}"
