@@ -55,6 +55,17 @@ def test_host_side_argument_checks_need_no_gpu():
     n = C.c_size_t()
     assert lib.aq_export(None, None, 0, C.byref(n)) == aq.AQ_ERR_INVALID_ARG
     lib.aq_free(None)   # no-op
+    # attention entry points: the same order of checks (arguments first, the device last)
+    assert lib.aq_attn_scratch_bytes(0) == 0 and lib.aq_attn_scratch_bytes(65) == 0
+    big = 0x10000
+    assert lib.aq_attn_decode(None, big, big, big, 1, 32, 32, 128, 10, 64, 0.0, 0, 2, big, 1 << 30, None) == aq.AQ_ERR_INVALID_ARG
+    assert lib.aq_attn_decode(big, big, big, big, 1, 32, 32, 64, 10, 64, 0.0, 0, 2, big, 1 << 30, None) == aq.AQ_ERR_UNSUPPORTED
+    assert lib.aq_attn_decode(big, big, big, big, 9, 32, 16, 128, 10, 64, 0.0, 0, 2, big, 1 << 30, None) == aq.AQ_ERR_UNSUPPORTED
+    assert lib.aq_attn_decode(big, big, big, big, 1, 32, 32, 128, 65, 64, 0.0, 0, 2, big, 1 << 30, None) == aq.AQ_ERR_INVALID_ARG
+    assert lib.aq_rope(None, 32, 128, 0, 10000.0, 0, None) == aq.AQ_ERR_INVALID_ARG
+    assert lib.aq_rope(big, 32, 128, 0, 0.5, 0, None) == aq.AQ_ERR_INVALID_ARG          # theta must exceed 1
+    assert lib.aq_kv_append(big, big, big, big, 32, 128, 64, 64, 0, None) == aq.AQ_ERR_INVALID_ARG   # pos == L_max
+    assert lib.aq_kv_append(big, big, big, big, 32, 64, 0, 64, 0, None) == aq.AQ_ERR_UNSUPPORTED
 
 
 def test_binding_has_no_fallback():
