@@ -349,6 +349,40 @@ aq_status_t aq_stack_forward(const aq_stack_t* prog, const void* x0_dev, void* o
                              int M, aq_dtype_t dtype, void* workspace_dev, size_t ws_bytes,
                              aq_stream_t stream);
 
+/*
+ * aq_stack_forward_attn -- aq_stack_forward for M <= AQ_DECODE_MAX_M new tokens with attention over a key/value cache
+ * between the linears (Section 2: W_Q, W_K, W_V feed the attention whose output W_O reads; the attention itself is
+ * the textbook operation, see aq_attn_decode).
+ *
+ * A buffer of the program that no op writes and that is not buffer 0 is an input filled by somebody else (float32
+ * [M][width] in the workspace).  Each aq_stack_attn_t says: after op `after_op` (the last op of a phase; its q, k, v
+ * buffers are complete then) rotate q and k for positions pos .. pos + M - 1 (aq_rope's rule), append the rounded k
+ * and v to rows pos .. pos + M - 1 of the caches, and write softmax attention of the M tokens over the L = pos + M
+ * cached positions (token m sees positions up to pos + m), scale 1/sqrt(128), as float32 into buffer dst_buf, which no
+ * op writes and which later ops (W_O) read.  Entries ascend in after_op.  Head dimension 128; (n_heads / n_kv_heads) *
+ * M <= 16; widths: q_buf and dst_buf n_heads * 128, k_buf and v_buf n_kv_heads * 128.
+ *   attn_scratch_dev : DEVICE, 256-byte aligned, aq_stack_attn_scratch_bytes(n_heads, n_kv_heads, M) bytes (the largest
+ *                      over the entries); contents irrelevant
+ * The linears between two attention steps run as one launch each of the whole-program decode kernel; a program that
+ * kernel cannot take returns AQ_ERR_UNSUPPORTED (the outputs are undefined then).  Other arguments, the workspace and what it
+ * holds afterwards as in aq_stack_forward; calls on one device must not overlap (see aq_attn_decode).
+ */
+typedef struct {
+    int32_t after_op;
+    int32_t q_buf, k_buf, v_buf, dst_buf;
+    int32_t n_heads, n_kv_heads;
+    int32_t pad_;
+    void* k_cache_dev;        /* DEVICE [n_kv_heads][L_max][128] of the activation dtype */
+    void* v_cache_dev;
+    int64_t L_max;
+} aq_stack_attn_t;
+
+size_t aq_stack_attn_scratch_bytes(int n_heads, int n_kv_heads, int M);
+aq_status_t aq_stack_forward_attn(const aq_stack_t* prog, const aq_stack_attn_t* attn, int n_attn, int64_t pos, float theta,
+                                  const void* x0_dev, void* out_dev, int out_buf, int M, aq_dtype_t dtype,
+                                  void* workspace_dev, size_t ws_bytes, void* attn_scratch_dev, size_t attn_scratch_bytes,
+                                  aq_stream_t stream);
+
 /* Byte offset of buffer b inside the workspace ((size_t)-1 on a bad argument). */
 size_t aq_stack_buffer_offset(const aq_stack_t* prog, int M, int b);
 

@@ -27,7 +27,7 @@ AQ_MAX_M, AQ_DECODE_MAX_M = 4096, 8
 
 SYMBOLS = ("aq_pack", "aq_pack_opt", "aq_pack_sb", "aq_import_sb", "aq_export_sb", "aq_import", "aq_export", "aq_info", "aq_dequant", "aq_linear", "aq_linear_f32out", "aq_linear_noalloc",
            "aq_rbf_gram", "aq_hsic", "aq_sensitivity", "aq_allocate_bits",
-           "aq_attn_scratch_bytes", "aq_rope", "aq_kv_append", "aq_attn_decode",
+           "aq_attn_scratch_bytes", "aq_rope", "aq_kv_append", "aq_attn_decode", "aq_stack_attn_scratch_bytes", "aq_stack_forward_attn",
            "aq_stack_workspace_bytes", "aq_stack_forward", "aq_stack_buffer_offset", "aq_stack_input_offset", "aq_check", "aq_free",
            "aq_set_wait_limit_ns", "aq_debug_decode_hold", "aq_status_string", "aq_last_cuda_error", "aq_kernel_launches")
 
@@ -401,6 +401,36 @@ def aq_stack_forward(prog: Program, x0, out, out_buf: int, M: int, workspace, st
     workspace: CUDA uint8 tensor of at least workspace_bytes(M)."""
     _check(_lib.aq_stack_forward(C.byref(prog.c), _ptr(x0), _ptr(out), out_buf, M, dtype_code(x0), _ptr(workspace),
                                  workspace.numel() * workspace.element_size(), _stream(stream)), "aq_stack_forward")
+    return out
+
+
+class StackAttn(C.Structure):
+    _fields_ = [("after_op", C.c_int32), ("q_buf", C.c_int32), ("k_buf", C.c_int32), ("v_buf", C.c_int32), ("dst_buf", C.c_int32),
+                ("n_heads", C.c_int32), ("n_kv_heads", C.c_int32), ("pad_", C.c_int32),
+                ("k_cache_dev", C.c_void_p), ("v_cache_dev", C.c_void_p), ("L_max", C.c_int64)]
+
+
+def aq_stack_attn_scratch_bytes(n_heads: int, n_kv_heads: int, M: int) -> int:
+    _lib.aq_stack_attn_scratch_bytes.argtypes = [C.c_int, C.c_int, C.c_int]
+    _lib.aq_stack_attn_scratch_bytes.restype = C.c_size_t
+    return int(_lib.aq_stack_attn_scratch_bytes(n_heads, n_kv_heads, M))
+
+
+def aq_stack_forward_attn(prog: Program, attn, pos: int, x0, out, out_buf: int, M: int, workspace, scratch, theta: float = 10000.0,
+                          stream=None):
+    """aq_stack_forward with attention over key/value caches between the linears.  attn: list of dicts with keys
+    after_op, q_buf, k_buf, v_buf, dst_buf, n_heads, n_kv_heads, k_cache, v_cache (CUDA [n_kv_heads][L_max][128] of x0's
+    type); pos: position of the first of the M new tokens; scratch: CUDA uint8 tensor (aq_stack_attn_scratch_bytes)."""
+    arr = (StackAttn * max(1, len(attn)))()
+    for i, t in enumerate(attn):
+        arr[i] = StackAttn(t["after_op"], t["q_buf"], t["k_buf"], t["v_buf"], t["dst_buf"], t["n_heads"], t["n_kv_heads"], 0,
+                           _ptr(t["k_cache"]), _ptr(t["v_cache"]), t["k_cache"].shape[1])
+    _lib.aq_stack_forward_attn.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_float, C.c_void_p, C.c_void_p, C.c_int, C.c_int,
+                                           C.c_int, C.c_void_p, C.c_size_t, C.c_void_p, C.c_size_t, C.c_void_p]
+    _lib.aq_stack_forward_attn.restype = C.c_int
+    _check(_lib.aq_stack_forward_attn(C.byref(prog.c), arr, len(attn), int(pos), float(theta), _ptr(x0), _ptr(out), out_buf, M,
+                                      dtype_code(x0), _ptr(workspace), workspace.numel() * workspace.element_size(), _ptr(scratch),
+                                      scratch.numel() * scratch.element_size(), _stream(stream)), "aq_stack_forward_attn")
     return out
 
 

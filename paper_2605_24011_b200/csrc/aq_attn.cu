@@ -340,6 +340,52 @@ __global__ void kv_append_kernel(uint4* kc, uint4* vc, const uint4* k, const uin
     vc[o] = v[idx];
 }
 
+// What a stack program's attention step does with the float32 q, k, v rows of its M new tokens before the attention
+// itself: rotates q and k for their positions, rounds q to the activation type into a staging array [M][H][D], and puts
+// the rounded k and v into rows pos .. pos + M - 1 of the caches.  One CTA of D/2 threads per (token, head).
+template <typename T>
+__global__ void attn_prepare_kernel(const float* __restrict__ q, const float* __restrict__ k, const float* __restrict__ v, T* __restrict__ q16,
+                                    T* __restrict__ kc, T* __restrict__ vc, int H, int Hkv, int D, int64_t pos, int64_t Lmax, double log2_theta) {
+    const int m = blockIdx.y, hh = blockIdx.x, i = threadIdx.x, half = D / 2;
+    auto cast = [](float x) -> T {
+        if constexpr (std::is_same<T, __half>::value) return __float2half_rn(x);
+        else return __float2bfloat16_rn(x);
+    };
+    if (hh >= H + Hkv) {   // a value head: rounded as it is
+        const int hk = hh - H - Hkv;
+        const float* src = v + ((size_t)m * Hkv + hk) * D;
+        T* dst = vc + ((size_t)hk * Lmax + pos + m) * D;
+        dst[i] = cast(src[i]);
+        dst[i + half] = cast(src[i + half]);
+        return;
+    }
+    const double ang = (double)(pos + m) * exp2(-2.0 * (double)i / (double)D * log2_theta);
+    double sn, cs;
+    sincos(ang, &sn, &cs);
+    const float fc = (float)cs, fs = (float)sn;
+    const bool is_q = hh < H;
+    const float* src = is_q ? q + ((size_t)m * H + hh) * D : k + ((size_t)m * Hkv + (hh - H)) * D;
+    T* dst = is_q ? q16 + ((size_t)m * H + hh) * D : kc + ((size_t)(hh - H) * Lmax + pos + m) * D;
+    const float a = src[i], b = src[i + half];
+    dst[i] = cast(fmaf(a, fc, -b * fs));
+    dst[i + half] = cast(fmaf(b, fc, a * fs));
+}
+
+cudaError_t launch_attn_prepare(const float* q, const float* k, const float* v, void* q16, void* kc, void* vc, int M, int H, int Hkv,
+                                int64_t pos, int64_t Lmax, float theta, aq_dtype_t dt, cudaStream_t s) {
+    const dim3 grid((unsigned)(H + 2 * Hkv), (unsigned)M);
+    const double l2t = log2((double)theta);
+    if (dt == AQ_F16)
+        attn_prepare_kernel<__half><<<grid, AT_D / 2, 0, s>>>(q, k, v, reinterpret_cast<__half*>(q16), reinterpret_cast<__half*>(kc),
+                                                             reinterpret_cast<__half*>(vc), H, Hkv, AT_D, pos, Lmax, l2t);
+    else
+        attn_prepare_kernel<__nv_bfloat16><<<grid, AT_D / 2, 0, s>>>(q, k, v, reinterpret_cast<__nv_bfloat16*>(q16),
+                                                                    reinterpret_cast<__nv_bfloat16*>(kc), reinterpret_cast<__nv_bfloat16*>(vc), H,
+                                                                    Hkv, AT_D, pos, Lmax, l2t);
+    count_launch();
+    return cudaGetLastError();
+}
+
 // ---- host ---------------------------------------------------------------------------------------------------
 static int attn_max_splits(int n_kv) {
     // one CTA per SM fits (its rings take most of the shared memory), so one wave: as many splits as keep the grid

@@ -922,7 +922,7 @@ struct DecodePlan {
 std::mutex g_plan_mutex;
 std::vector<DecodePlan*> g_plans;
 uint64_t g_plan_clock = 0;
-constexpr size_t MAX_PLANS = 16;
+constexpr size_t MAX_PLANS = 256;   // (a program with attention between its linears is one plan per stretch of linears)
 u64 g_wait_ns = DS_WAIT_NS_DEFAULT;
 bool g_hold = false;          // testing: the first packed input of a program expects one contribution too many
 
@@ -943,7 +943,7 @@ template <typename T> void key_put(std::vector<uint8_t>& k, const T& v) {
 // does not fit this kernel.
 bool build_decode_tables(const aq_stack_t* p, const StackPlan& plan, int M, int n_cta, uint8_t* ws,
                          std::vector<DsPhase>& phases, std::vector<DsTail>& tails, std::vector<DsCtaPhase>& ctab,
-                         std::vector<char>& in_tails) {
+                         std::vector<char>& in_tails, int op_first, int op_end) {
     if (M < 1 || M > AQ_DECODE_MAX_M || p->n_ops > 32000 || plan.pk_off.empty()) return false;
     phases.clear();
     tails.clear();
@@ -954,12 +954,21 @@ bool build_decode_tables(const aq_stack_t* p, const StackPlan& plan, int M, int 
     auto packed = [&](int b) { return reinterpret_cast<u64*>(ws + plan.pk_off[b]); };
     auto plain = [&](int b) { return reinterpret_cast<float*>(ws + plan.buf_off[b]); };
     auto expect_of = [&](int b) { return (uint32_t)p->ops[writer[b]].w->KP; };
+    // a launch that runs ops [op_first, op_end) of the program: what earlier launches of the pass wrote is complete (as
+    // packed sums and as the caller's float32 copy) before this one starts
+    for (int i = 0; i < op_first; ++i) {
+        writer[p->ops[i].dst] = i;
+        whole[p->ops[i].dst] = 1;
+        recorded[p->ops[i].dst] = 1;
+    }
     int rot = 0;   // where the next op's odd units start
     bool hold = g_hold;
     const int n_ph = (int)plan.phase_first.size();
     for (int ph = 0; ph < n_ph; ++ph) {
         const int pfirst = plan.phase_first[ph];
         const int plast = (ph + 1 < n_ph) ? plan.phase_first[ph + 1] : p->n_ops;
+        if (pfirst < op_first || pfirst >= op_end) continue;
+        if (plast > op_end) return false;   // (a launch ends where a phase ends)
         for (int first = pfirst; first < plast;) {
             // as many of the phase's ops (at most DS_MAX_PHASE_OPS) as leave every CTA's staged slabs inside the
             // shared-memory buffer; the rest of them form a further phase with the same input
@@ -1065,7 +1074,7 @@ bool build_decode_tables(const aq_stack_t* p, const StackPlan& plan, int M, int 
     // what no phase has copied out for the caller
     in_tails.assign(p->n_bufs, 0);
     for (int b = 1; b < p->n_bufs; ++b) {
-        if (writer[b] < 0 || recorded[b]) continue;
+        if (writer[b] < op_first || recorded[b]) continue;   // (written by this launch, read by none of its phases)
         const int64_t n = (int64_t)M * p->buf_width[b];
         if (n % 4) return false;
         in_tails[b] = 1;
@@ -1105,9 +1114,10 @@ static cudaError_t launch_ds(const DsArgs& a, int grid, cudaStream_t s) {
 }
 
 int launch_decode_stack(const aq_stack_t* p, const StackPlan& plan, int M, aq_dtype_t dt, uint8_t* ws, cudaStream_t s,
-                        cudaError_t* err, void* out, int out_buf, bool* wrote_out) {
+                        cudaError_t* err, void* out, int out_buf, bool* wrote_out, int op_first, int op_end, bool clear) {
     *err = cudaSuccess;
     *wrote_out = false;
+    if (op_end < 0) op_end = p->n_ops;
     const int grid = sm_count();
     const int dev = current_device();
     cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
@@ -1115,7 +1125,7 @@ int launch_decode_stack(const aq_stack_t* p, const StackPlan& plan, int M, aq_dt
     const bool capturing = (cap != cudaStreamCaptureStatusNone);
     // key: everything the device tables are computed from
     std::vector<uint8_t> key;
-    key_put(key, M); key_put(key, dev); key_put(key, grid); key_put(key, ws);
+    key_put(key, M); key_put(key, dev); key_put(key, grid); key_put(key, ws); key_put(key, op_first); key_put(key, op_end);
     std::lock_guard<std::mutex> lock(g_plan_mutex);
     key_put(key, g_hold);
     key_put(key, p->n_ops); key_put(key, p->n_bufs);
@@ -1134,7 +1144,7 @@ int launch_decode_stack(const aq_stack_t* p, const StackPlan& plan, int M, aq_dt
         std::vector<DsTail> tails;
         std::vector<DsCtaPhase> ctab;
         std::vector<char> in_tails;
-        if (!build_decode_tables(p, plan, M, grid, ws, phases, tails, ctab, in_tails)) return 1;
+        if (!build_decode_tables(p, plan, M, grid, ws, phases, tails, ctab, in_tails, op_first, op_end)) return 1;
         if (g_plans.size() >= MAX_PLANS) {   // make room: the oldest plan no graph refers to
             size_t oldest = g_plans.size();
             for (size_t i = 0; i < g_plans.size(); ++i)
@@ -1206,8 +1216,8 @@ int launch_decode_stack(const aq_stack_t* p, const StackPlan& plan, int M, aq_dt
         a.out_n = (int64_t)M * p->buf_width[out_buf];
         *wrote_out = true;
     }
-    // the packed sums start from zero
-    cudaError_t e = cudaMemsetAsync(ws + plan.pk_begin, 0, plan.pk_end - plan.pk_begin, s);
+    // the packed sums start from zero (once per pass: a later launch of the same pass reads what the earlier ones left)
+    cudaError_t e = clear ? cudaMemsetAsync(ws + plan.pk_begin, 0, plan.pk_end - plan.pk_begin, s) : cudaSuccess;
     if (e == cudaSuccess) {
         const bool bf = (dt == AQ_BF16);
         if (M == 1) e = bf ? launch_ds<1, true>(a, grid, s) : launch_ds<1, false>(a, grid, s);

@@ -79,6 +79,7 @@ struct StackPlan {
     std::vector<size_t> buf_off;    // per buffer: float32 [M][width]
     std::vector<size_t> in_off;     // per op: its phase's staged input [M][K] (activation dtype)
     std::vector<int> phase_first;   // first op of each phase (ops that share one input vector)
+    std::vector<char> external;     // per buffer: no op writes it and it is not buffer 0 (somebody else fills it)
     std::vector<size_t> pk_off;     // per buffer (M <= AQ_DECODE_MAX_M only): its packed 64-bit sums [M][width]
     size_t pk_begin = 0, pk_end = 0;   // the packed sums' region: zero at the start of a decode pass
     std::vector<size_t> nm_off;     // per op that opens an RMS-normalised phase (3 <= M <= AQ_DECODE_MAX_M): the CTAs'
@@ -93,9 +94,10 @@ struct StackPlan {
 
 // whole-program decode (M <= AQ_DECODE_MAX_M) in one persistent kernel: 0 = launched,
 // 1 = the program does not fit that kernel (nothing launched), -1 = CUDA error in *err
-// (out: the caller's rounded copy of buffer out_buf, or null; *wrote_out: the kernel itself writes it)
+// (out: the caller's rounded copy of buffer out_buf, or null; *wrote_out: the kernel itself writes it; op_first, op_end:
+// the ops of the program this launch runs, whole phases; clear: the packed sums are zeroed first)
 int launch_decode_stack(const aq_stack_t* p, const StackPlan& plan, int M, aq_dtype_t dt, uint8_t* ws, cudaStream_t s,
-                        cudaError_t* err, void* out, int out_buf, bool* wrote_out);
+                        cudaError_t* err, void* out, int out_buf, bool* wrote_out, int op_first = 0, int op_end = -1, bool clear = true);
 void decode_stack_forget(aq_handle_t h);   // drops cached device tables that name h
 int read_decode_status(bool clear);        // nonzero: a bounded wait in the decode-stack kernel ran out
 void set_decode_wait_ns(unsigned long long ns);   // limit of every wait in that kernel (0: the default, two seconds)
@@ -135,6 +137,8 @@ size_t attn_scratch_bytes(int n_kv);
 cudaError_t launch_attn_decode(const void* q, const void* kc, const void* vc, void* out, int M, int n_heads, int n_kv, int64_t L,
                                int64_t Lmax, float scale, aq_dtype_t dt, aq_dtype_t out_dt, void* scratch, cudaStream_t s);
 cudaError_t launch_rope(void* x, int n_heads, int D, int64_t pos, float theta, aq_dtype_t dt, cudaStream_t s);
+cudaError_t launch_attn_prepare(const float* q, const float* k, const float* v, void* q16, void* kc, void* vc, int M, int H, int Hkv,
+                                int64_t pos, int64_t Lmax, float theta, aq_dtype_t dt, cudaStream_t s);
 cudaError_t launch_kv_append(void* kc, void* vc, const void* k, const void* v, int n_kv, int D, int64_t pos, int64_t Lmax, cudaStream_t s);
 
 int current_device();               // cudaGetDevice, or -1

@@ -34,8 +34,13 @@ static bool plan_stack(const aq_stack_t* p, int M, StackPlan& plan) {
         if (p->buf_width[b] > maxw) maxw = p->buf_width[b];
     }
     plan.stage_off = off;
-    std::vector<char> written(p->n_bufs, 0);
-    written[0] = 1;
+    // A buffer that no op writes is an input of the program: buffer 0 is filled from x0, any other one by whoever runs
+    // between the ops (the attention of aq_stack_forward_attn) or by the caller, as float32 in the workspace.
+    std::vector<char> written(p->n_bufs, 1);
+    for (int i = 0; i < p->n_ops; ++i)
+        if (p->ops[i].dst >= 1 && p->ops[i].dst < p->n_bufs) written[p->ops[i].dst] = 0;
+    plan.external.assign(written.begin(), written.end());
+    plan.external[0] = 0;
     for (int i = 0; i < p->n_ops; ++i) {
         const aq_stack_op_t& o = p->ops[i];
         if (!handle_ok(o.w)) return false;
@@ -305,9 +310,17 @@ static cudaError_t run_stack(const aq_stack_t* p, const StackPlan& plan, const T
             count_launch();
         }
         if (r == 0) return cudaGetLastError();
-        // op by op: the streaming kernel accumulates with red.add, so every output starts at zero
-        e = cudaMemsetAsync(ws + plan.buf_off[1], 0, plan.stage_off - plan.buf_off[1], s);
-        if (e != cudaSuccess) return e;
+        // op by op: the streaming kernel accumulates with red.add, so every output starts at zero (inputs that somebody
+        // else has filled are left alone: runs of buffers between them are cleared)
+        for (int b = 1; b < p->n_bufs;) {
+            if (plan.external[b]) { ++b; continue; }
+            int b1 = b;
+            while (b1 + 1 < p->n_bufs && !plan.external[b1 + 1]) ++b1;
+            const size_t end = (b1 + 1 < p->n_bufs) ? plan.buf_off[b1 + 1] : plan.stage_off;
+            e = cudaMemsetAsync(ws + plan.buf_off[b], 0, end - plan.buf_off[b], s);
+            if (e != cudaSuccess) return e;
+            b = b1 + 1;
+        }
     }
     int i = 0;
     while (i < p->n_ops) {
@@ -447,6 +460,99 @@ aq_status_t aq_stack_forward(const aq_stack_t* prog, const void* x0_dev, void* o
                                      (uint8_t*)workspace_dev, s);
     if (e != cudaSuccess) return cuda_fail(e);
     return AQ_OK;
+}
+
+size_t aq_stack_attn_scratch_bytes(int n_heads, int n_kv_heads, int M) {
+    if (n_heads < 1 || n_kv_heads < 1 || n_kv_heads > 64 || M < 1 || M > AQ_DECODE_MAX_M) return 0;
+    return align_up((size_t)M * n_heads * 128 * 2, 256) + attn_scratch_bytes(n_kv_heads);
+}
+
+aq_status_t aq_stack_forward_attn(const aq_stack_t* prog, const aq_stack_attn_t* attn, int n_attn, int64_t pos, float theta,
+                                  const void* x0_dev, void* out_dev, int out_buf, int M, aq_dtype_t dtype, void* workspace_dev,
+                                  size_t ws_bytes, void* attn_scratch_dev, size_t attn_scratch_bytes_given, aq_stream_t stream) {
+    StackPlan plan;
+    if (!plan_stack(prog, M, plan)) return AQ_ERR_INVALID_ARG;
+    if (!x0_dev || !workspace_dev || (reinterpret_cast<uintptr_t>(workspace_dev) & 255u) ||
+        (reinterpret_cast<uintptr_t>(x0_dev) & 15u) || (reinterpret_cast<uintptr_t>(out_dev) & 15u))
+        return AQ_ERR_INVALID_ARG;
+    if (ws_bytes < plan.total || n_attn < 0 || (n_attn > 0 && !attn) || pos < 0 || !(theta > 1.f)) return AQ_ERR_INVALID_ARG;
+    if (out_dev && (out_buf < 0 || out_buf >= prog->n_bufs)) return AQ_ERR_INVALID_ARG;
+    if (dtype != AQ_F16 && dtype != AQ_BF16) return (dtype == AQ_F32) ? AQ_ERR_UNSUPPORTED : AQ_ERR_INVALID_ARG;
+    if (M > AQ_DECODE_MAX_M) return AQ_ERR_UNSUPPORTED;
+    size_t need = 0;
+    int prev = -1;
+    for (int i = 0; i < n_attn; ++i) {
+        const aq_stack_attn_t& t = attn[i];
+        auto buf_ok = [&](int b, int64_t w) { return b >= 1 && b < prog->n_bufs && prog->buf_width[b] == w; };
+        if (t.after_op <= prev || t.after_op >= prog->n_ops || t.n_heads < 1 || t.n_kv_heads < 1 || t.n_heads % t.n_kv_heads != 0 ||
+            !buf_ok(t.q_buf, (int64_t)t.n_heads * 128) || !buf_ok(t.k_buf, (int64_t)t.n_kv_heads * 128) ||
+            !buf_ok(t.v_buf, (int64_t)t.n_kv_heads * 128) || !buf_ok(t.dst_buf, (int64_t)t.n_heads * 128) || !plan.external[t.dst_buf] ||
+            !t.k_cache_dev || !t.v_cache_dev || (reinterpret_cast<uintptr_t>(t.k_cache_dev) & 15u) ||
+            (reinterpret_cast<uintptr_t>(t.v_cache_dev) & 15u) || pos + M > t.L_max || t.L_max > ((int64_t)1 << 31))
+            return AQ_ERR_INVALID_ARG;
+        // q, k, v come from ops at or before after_op, and the next op opens a phase (a launch ends where a phase ends)
+        bool qw = false, kw = false, vw = false;
+        for (int o = 0; o <= t.after_op; ++o) {
+            qw |= prog->ops[o].dst == t.q_buf; kw |= prog->ops[o].dst == t.k_buf; vw |= prog->ops[o].dst == t.v_buf;
+        }
+        if (!qw || !kw || !vw) return AQ_ERR_INVALID_ARG;
+        if (t.after_op + 1 < prog->n_ops && same_input(prog->ops[t.after_op + 1], prog->ops[t.after_op])) return AQ_ERR_INVALID_ARG;
+        if ((int64_t)(t.n_heads / t.n_kv_heads) * M > 16 || t.n_kv_heads > 64) return AQ_ERR_UNSUPPORTED;
+        need = std::max(need, aq_stack_attn_scratch_bytes(t.n_heads, t.n_kv_heads, M));
+        prev = t.after_op;
+    }
+    if (n_attn > 0 && (!attn_scratch_dev || (reinterpret_cast<uintptr_t>(attn_scratch_dev) & 255u) || attn_scratch_bytes_given < need))
+        return AQ_ERR_INVALID_ARG;
+    {
+        int dev = 0;
+        cudaDeviceProp prop;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return cuda_fail(cudaGetLastError());
+        if (prop.major != 10) return AQ_ERR_ARCH;
+    }
+    cudaStream_t s = (cudaStream_t)stream;
+    uint8_t* ws = reinterpret_cast<uint8_t*>(workspace_dev);
+    auto buf = [&](int b) { return reinterpret_cast<float*>(ws + plan.buf_off[b]); };
+    cudaError_t e = cudaSuccess;
+    {
+        const int64_t n = (int64_t)M * prog->buf_width[0];
+        if (dtype == AQ_F16) widen_kernel<__half><<<(unsigned)((n + 255) / 256), 256, 0, s>>>((const __half*)x0_dev, buf(0), n);
+        else widen_kernel<__nv_bfloat16><<<(unsigned)((n + 255) / 256), 256, 0, s>>>((const __nv_bfloat16*)x0_dev, buf(0), n);
+        count_launch();
+    }
+    int first = 0;
+    bool wrote_out = false;
+    for (int i = 0; i <= n_attn; ++i) {
+        const int end = (i < n_attn) ? attn[i].after_op + 1 : prog->n_ops;
+        if (end > first) {
+            bool w = false;
+            const int r = launch_decode_stack(prog, plan, M, dtype, ws, s, &e, (i == n_attn) ? out_dev : nullptr, out_buf, &w, first, end,
+                                              first == 0);
+            if (r < 0) return cuda_fail(e);
+            if (r > 0) return AQ_ERR_UNSUPPORTED;
+            wrote_out = wrote_out || w;
+        }
+        first = end;
+        if (i == n_attn) break;
+        const aq_stack_attn_t& t = attn[i];
+        uint8_t* sc = reinterpret_cast<uint8_t*>(attn_scratch_dev);
+        void* q16 = sc;
+        void* asc = sc + align_up((size_t)M * t.n_heads * 128 * 2, 256);
+        e = launch_attn_prepare(buf(t.q_buf), buf(t.k_buf), buf(t.v_buf), q16, t.k_cache_dev, t.v_cache_dev, M, t.n_heads, t.n_kv_heads, pos,
+                                t.L_max, theta, dtype, s);
+        if (e == cudaSuccess)
+            e = launch_attn_decode(q16, t.k_cache_dev, t.v_cache_dev, buf(t.dst_buf), M, t.n_heads, t.n_kv_heads, pos + M, t.L_max,
+                                   0.08838834764831845f, dtype, AQ_F32, asc, s);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    for (int k = 0; k < prog->n_ops; ++k) prog->ops[k].w->last_stream = s;
+    if (out_dev && !wrote_out) {
+        const int64_t n = (int64_t)M * prog->buf_width[out_buf];
+        if (dtype == AQ_F16) narrow_kernel<__half><<<(unsigned)((n + 255) / 256), 256, 0, s>>>(buf(out_buf), (__half*)out_dev, n);
+        else narrow_kernel<__nv_bfloat16><<<(unsigned)((n + 255) / 256), 256, 0, s>>>(buf(out_buf), (__nv_bfloat16*)out_dev, n);
+        count_launch();
+    }
+    e = cudaGetLastError();
+    return e == cudaSuccess ? AQ_OK : cuda_fail(e);
 }
 
 }  // extern "C"

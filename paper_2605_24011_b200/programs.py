@@ -52,6 +52,43 @@ def block_program(layers):
     return aq.Program(widths, ops), h, names
 
 
+def block_program_attn(layers, n_heads, n_kv_heads):
+    """block_program with the attention in its place: W_o reads a buffer that the attention step of
+    aq_stack_forward_attn fills from q, k, v and the caches.  Returns (Program, out_buf, op_names, attn), attn being
+    the list of attention steps without their caches (keys after_op, q_buf, k_buf, v_buf, dst_buf, n_heads, n_kv_heads)."""
+    first = layers[0]["shape"]
+    widths = [first["q"][1]]
+    ops, names, attn = [], [], []
+    h = 0
+
+    def new_buf(w):
+        widths.append(w)
+        return len(widths) - 1
+
+    for li, L in enumerate(layers):
+        sh = L["shape"]
+        bq, bk, bv = new_buf(sh["q"][0]), new_buf(sh["k"][0]), new_buf(sh["v"][0])
+        for nm, b in (("q", bq), ("k", bk), ("v", bv)):
+            ops.append({"w": L[nm], "src": h, "dst": b, "in_op": aq.AQ_IN_RMSNORM})
+            names.append((li, nm))
+        ba = new_buf(sh["q"][0])                      # the attention's output: no op writes it
+        attn.append({"after_op": len(ops) - 1, "q_buf": bq, "k_buf": bk, "v_buf": bv, "dst_buf": ba, "n_heads": n_heads,
+                     "n_kv_heads": n_kv_heads})
+        h1 = new_buf(sh["o"][0])
+        ops.append({"w": L["o"], "src": ba, "dst": h1, "in_op": aq.AQ_IN_PLAIN, "out_op": aq.AQ_OUT_ADD, "res": h})
+        names.append((li, "o"))
+        bg, bu = new_buf(sh["gate"][0]), new_buf(sh["up"][0])
+        for nm, b in (("gate", bg), ("up", bu)):
+            ops.append({"w": L[nm], "src": h1, "dst": b, "in_op": aq.AQ_IN_RMSNORM})
+            names.append((li, nm))
+        h2 = new_buf(sh["down"][0])
+        ops.append({"w": L["down"], "src": bg, "src2": bu, "dst": h2, "in_op": aq.AQ_IN_SILU_MUL,
+                    "out_op": aq.AQ_OUT_ADD, "res": h1})
+        names.append((li, "down"))
+        h = h2
+    return aq.Program(widths, ops), h, names, attn
+
+
 def mlp_program(gate, up, down, hidden, inter):
     """gate/up -> silu*up -> down, no norm and no residual (a bare MLP block)."""
     widths = [hidden, inter, inter, hidden]
