@@ -600,6 +600,8 @@ def main():
         line["dequant"] = dequant_leg(aq, synth, peaks, torch)
         line["attn_decode"] = attn_leg(aq, peaks, torch)
         if args.layers == 32:
+            line["decode_with_attention"] = decode_attn_leg(aq, info, peaks, torch)
+        if args.layers == 32:
             line["configs"] = configs_leg(peaks, torch, prog, out_buf, info)
         cores = len(os.sched_getaffinity(0))
         mats = oracle_layer_sample()
@@ -697,6 +699,53 @@ def attn_leg(aq, peaks, torch):
                                      "kernel": "attn_decode_kernel"}}
         del caches
     return out
+
+
+def decode_attn_leg(aq, info, peaks, torch, context=4096, steps=30):
+    """One decoded token of the same 7B-class stack WITH its attention: per block q, k, v -> rotation, cache append,
+    attention over `context` cached positions -> W_o ... (aq_stack_forward_attn: one launch of the decode kernel per
+    stretch of linears between two attention steps).  Bytes = packed weights + the keys and values read."""
+    from paper_2605_24011_b200 import programs, workloads
+    H = 32
+    prog, out_buf, names, attn = programs.block_program_attn(info["layers"], H, H)
+    g = torch.Generator(device="cuda")
+    g.manual_seed(13)
+    Lmax = context + 8
+    for t in attn:
+        t["k_cache"] = torch.randn((H, Lmax, 128), generator=g, device="cuda", dtype=torch.float16)
+        t["v_cache"] = torch.randn((H, Lmax, 128), generator=g, device="cuda", dtype=torch.float16)
+    ws = torch.empty(prog.workspace_bytes(1), dtype=torch.uint8, device="cuda")
+    scratch = torch.empty(aq.aq_stack_attn_scratch_bytes(H, H, 1), dtype=torch.uint8, device="cuda")
+    x0 = workloads.activations_device(1, 4096, torch.float16, 3, 1)
+    y = torch.empty((1, 4096), dtype=torch.float16, device="cuda")
+    pos = context - 1
+    fn = lambda: aq.aq_stack_forward_attn(prog, attn, pos, x0, y, out_buf, 1, ws, scratch)
+    l0 = aq.aq_kernel_launches()
+    fn()
+    launches = aq.aq_kernel_launches() - l0
+    ms = _timed(fn, steps, 3, torch) / steps
+    aq.aq_check()
+    # the same token replayed from a CUDA graph: device time without the host's share of 98 launches
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            fn()
+    torch.cuda.synchronize()
+    ms_graph = _timed(graph.replay, steps, 3, torch) / steps
+    aq.aq_check()
+    kv = len(attn) * 2 * H * context * 128 * 2
+    byts = info["packed_bytes"] + kv
+    for t in attn:
+        del t["k_cache"], t["v_cache"]
+    return {"workload": f"the same stack with attention over {context} cached positions per block (32 heads of 128, fp16 caches), M = 1",
+            "us_per_token": 1e3 * ms, "gbs": byts / ms / 1e6, "us_per_token_graph": 1e3 * ms_graph, "gbs_graph": byts / ms_graph / 1e6,
+            "kv_bytes": kv, "launches_per_token": launches,
+            "roofline": {"bound": "hbm", "achieved": byts / ms_graph / 1e6, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": byts / ms_graph / 1e6 / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
+                         "what": "graph replay",
+                         "kernel": "decode_stack_kernel (33 launches) + attn_decode_kernel (32) + attn_prepare_kernel (32)"}}
 
 
 def dequant_leg(aq, synth, peaks, torch):

@@ -504,10 +504,10 @@ aq_status_t aq_stack_forward_attn(const aq_stack_t* prog, const aq_stack_attn_t*
     if (n_attn > 0 && (!attn_scratch_dev || (reinterpret_cast<uintptr_t>(attn_scratch_dev) & 255u) || attn_scratch_bytes_given < need))
         return AQ_ERR_INVALID_ARG;
     {
-        int dev = 0;
-        cudaDeviceProp prop;
-        if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return cuda_fail(cudaGetLastError());
-        if (prop.major != 10) return AQ_ERR_ARCH;
+        int dev = 0, major = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
+            return cuda_fail(cudaGetLastError());
+        if (major != 10) return AQ_ERR_ARCH;
     }
     cudaStream_t s = (cudaStream_t)stream;
     uint8_t* ws = reinterpret_cast<uint8_t*>(workspace_dev);
