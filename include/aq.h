@@ -365,7 +365,8 @@ aq_status_t aq_stack_forward(const aq_stack_t* prog, const void* x0_dev, void* o
  *                      over the entries); contents irrelevant
  * The linears between two attention steps run as one launch each of the whole-program decode kernel; a program that
  * kernel cannot take returns AQ_ERR_UNSUPPORTED (the outputs are undefined then).  Other arguments, the workspace and what it
- * holds afterwards as in aq_stack_forward; calls on one device must not overlap (see aq_attn_decode).
+ * holds afterwards as in aq_stack_forward (its rules on CUDA graphs too: one eager call with the same arguments first);
+ * calls on one device must not overlap (see aq_attn_decode).
  */
 typedef struct {
     int32_t after_op;
