@@ -209,6 +209,13 @@ def run_micro(args):
             fn = lambda i: aq.aq_hsic(Gs[2 * (i % n_copies)], Gs[2 * (i % n_copies) + 1], out=res)
             work, unit = 2.0 * K * K * 4, "GB/s"
         out.update({"K_samples": K, "d": d})
+    elif args.micro == "decode_token":
+        # one decoded token of the 7B-class stack with its attention (--K cached positions per block)
+        prog0, out_buf0, names0, _, info0 = workloads.llama7b_decode_stack(n_layers=args.layers, seed=0)
+        leg = decode_attn_leg(aq, info0, _peaks(), torch, context=args.K or 4096, steps=args.steps)
+        out.update({"layers": args.layers, **leg})
+        print(json.dumps(out))
+        return
     elif args.micro == "attn_decode":
         # one decoded token of a 7B-class block (32 heads of 128) against --K cached positions; HBM-bound on the cache:
         # 2 (keys, values) x heads x positions x 128 x 2 bytes per call; caches rotate so that L2 does not hold them
@@ -485,7 +492,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
     ap.add_argument("--layers", type=int, default=32, help="decoder layers (32 = the full workload)")
     ap.add_argument("--no-extras", action="store_true", help="skip prefill / dequant / oracle legs")
-    ap.add_argument("--micro", choices=("decode_linear", "prefill_linear", "dequant", "decode_stack", "prefill_stack", "pack", "pack_opt", "rbf_gram", "hsic", "attn_decode"),
+    ap.add_argument("--micro", choices=("decode_linear", "prefill_linear", "dequant", "decode_stack", "prefill_stack", "pack", "pack_opt", "rbf_gram", "hsic", "attn_decode", "decode_token"),
                     help="time one kernel on a small case (the command ncu captures are taken from) instead of the benchmark")
     ap.add_argument("--configs", action="store_true",
                     help="time all five workload configurations once each and print one JSON object (not the benchmark line)")
