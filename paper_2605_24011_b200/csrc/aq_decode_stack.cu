@@ -1113,8 +1113,20 @@ static cudaError_t launch_ds(const DsArgs& a, int grid, cudaStream_t s) {
     return e;
 }
 
+// The part of a plan's key that depends on the program alone (ops, their matrices, buffer widths).
+void decode_program_key(const aq_stack_t* p, std::vector<uint8_t>& key) {
+    key.reserve(key.size() + (size_t)p->n_ops * (sizeof(aq_stack_op_t) + 8) + (size_t)p->n_bufs * 8 + 16);
+    key_put(key, p->n_ops); key_put(key, p->n_bufs);
+    for (int i = 0; i < p->n_ops; ++i) {
+        key_put(key, p->ops[i]);
+        key_put(key, p->ops[i].w->frags);
+    }
+    for (int b = 0; b < p->n_bufs; ++b) key_put(key, p->buf_width[b]);
+}
+
 int launch_decode_stack(const aq_stack_t* p, const StackPlan& plan, int M, aq_dtype_t dt, uint8_t* ws, cudaStream_t s,
-                        cudaError_t* err, void* out, int out_buf, bool* wrote_out, int op_first, int op_end, bool clear) {
+                        cudaError_t* err, void* out, int out_buf, bool* wrote_out, int op_first, int op_end, bool clear,
+                        const std::vector<uint8_t>* program_key) {
     *err = cudaSuccess;
     *wrote_out = false;
     if (op_end < 0) op_end = p->n_ops;
@@ -1128,12 +1140,8 @@ int launch_decode_stack(const aq_stack_t* p, const StackPlan& plan, int M, aq_dt
     key_put(key, M); key_put(key, dev); key_put(key, grid); key_put(key, ws); key_put(key, op_first); key_put(key, op_end);
     std::lock_guard<std::mutex> lock(g_plan_mutex);
     key_put(key, g_hold);
-    key_put(key, p->n_ops); key_put(key, p->n_bufs);
-    for (int i = 0; i < p->n_ops; ++i) {
-        key_put(key, p->ops[i]);
-        key_put(key, p->ops[i].w->frags);
-    }
-    for (int b = 0; b < p->n_bufs; ++b) key_put(key, p->buf_width[b]);
+    if (program_key) key.insert(key.end(), program_key->begin(), program_key->end());   // (built once for all the launches of a pass)
+    else decode_program_key(p, key);
 
     DecodePlan* dp = nullptr;
     for (DecodePlan* q : g_plans)

@@ -97,7 +97,9 @@ struct StackPlan {
 // (out: the caller's rounded copy of buffer out_buf, or null; *wrote_out: the kernel itself writes it; op_first, op_end:
 // the ops of the program this launch runs, whole phases; clear: the packed sums are zeroed first)
 int launch_decode_stack(const aq_stack_t* p, const StackPlan& plan, int M, aq_dtype_t dt, uint8_t* ws, cudaStream_t s,
-                        cudaError_t* err, void* out, int out_buf, bool* wrote_out, int op_first = 0, int op_end = -1, bool clear = true);
+                        cudaError_t* err, void* out, int out_buf, bool* wrote_out, int op_first = 0, int op_end = -1, bool clear = true,
+                        const std::vector<uint8_t>* program_key = nullptr);
+void decode_program_key(const aq_stack_t* p, std::vector<uint8_t>& key);   // the program's share of a plan's key
 void decode_stack_forget(aq_handle_t h);   // drops cached device tables that name h
 int read_decode_status(bool clear);        // nonzero: a bounded wait in the decode-stack kernel ran out
 void set_decode_wait_ns(unsigned long long ns);   // limit of every wait in that kernel (0: the default, two seconds)

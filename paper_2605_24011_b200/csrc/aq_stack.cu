@@ -521,12 +521,14 @@ aq_status_t aq_stack_forward_attn(const aq_stack_t* prog, const aq_stack_attn_t*
     }
     int first = 0;
     bool wrote_out = false;
+    std::vector<uint8_t> program_key;
+    decode_program_key(prog, program_key);
     for (int i = 0; i <= n_attn; ++i) {
         const int end = (i < n_attn) ? attn[i].after_op + 1 : prog->n_ops;
         if (end > first) {
             bool w = false;
             const int r = launch_decode_stack(prog, plan, M, dtype, ws, s, &e, (i == n_attn) ? out_dev : nullptr, out_buf, &w, first, end,
-                                              first == 0);
+                                              first == 0, &program_key);
             if (r < 0) return cuda_fail(e);
             if (r > 0) return AQ_ERR_UNSUPPORTED;
             wrote_out = wrote_out || w;
