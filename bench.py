@@ -702,7 +702,7 @@ def attn_leg(aq, peaks, torch):
         gbs = per / us / 1e3
         out[f"L{L}"] = {"us_per_call": us, "gbs": gbs,
                         "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
-                                     "traffic": 67_175_168 + 467_712 if L == 4096 else None, "peak_source": peaks["source"],
+                                     "traffic": 67_175_680 + 434_688 if L == 4096 else None, "peak_source": peaks["source"],
                                      "kernel": "attn_decode_kernel"}}
         del caches
     return out

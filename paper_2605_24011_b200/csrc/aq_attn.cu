@@ -121,11 +121,18 @@ __global__ void __launch_bounds__(AT_WARPS * 32, 1) attn_decode_kernel(const Att
     for (int nd = 0; nd < AT_D / 8; ++nd) o[nd][0] = o[nd][1] = o[nd][2] = o[nd][3] = 0.f;
     float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;   // rows g and g + 8: running maximum (log2 domain), sum
 
+    // Launched as a programmatic dependent: the kernel before this one on the stream (the one that rotates q and
+    // appends the new rows, when a stack program runs) may still be at work.  Only the last M rows of the cache and q can
+    // be its output: a CTA whose positions include those rows waits for it before its first copy, the others start
+    // their copies of older rows at once and wait before they read q (and before they write anything).
+    const bool has_new_rows = p1 > a.L - a.M;
+    if (has_new_rows) pdl_wait();
 #pragma unroll
     for (int s = 0; s < AT_STAGES - 1; ++s) {
         if (s < my_tiles) issue(s, s);
         at_commit();
     }
+    if (!has_new_rows) pdl_wait();
     // (while the first tiles are on their way) the query heads of this key/value head as the A operand: row r = head
     // hk G + r, rows >= G are zero
     // row r = token r / G, head hk G + r % G of that token; rows >= G M are zero
@@ -347,6 +354,7 @@ template <typename T>
 __global__ void attn_prepare_kernel(const float* __restrict__ q, const float* __restrict__ k, const float* __restrict__ v, T* __restrict__ q16,
                                     T* __restrict__ kc, T* __restrict__ vc, int H, int Hkv, int D, int64_t pos, int64_t Lmax, double log2_theta) {
     const int m = blockIdx.y, hh = blockIdx.x, i = threadIdx.x, half = D / 2;
+    pdl_launch_dependents();   // the attention kernel may set itself up and read older cache rows meanwhile
     auto cast = [](float x) -> T {
         if constexpr (std::is_same<T, __half>::value) return __float2half_rn(x);
         else return __float2bfloat16_rn(x);
@@ -430,10 +438,10 @@ cudaError_t launch_attn_decode(const void* q, const void* kc, const void* vc, vo
         if (rc != 0) return rc < 0 ? cudaErrorInvalidDevice : (cudaError_t)rc;
     }
     const dim3 grid((unsigned)n_kv, (unsigned)splits);
-    if (bf) attn_decode_kernel<true><<<grid, AT_WARPS * 32, AT_SMEM, s>>>(a);
-    else attn_decode_kernel<false><<<grid, AT_WARPS * 32, AT_SMEM, s>>>(a);
+    const cudaError_t e = bf ? launch_pdl(attn_decode_kernel<true>, grid, dim3(AT_WARPS * 32), AT_SMEM, s, a)
+                             : launch_pdl(attn_decode_kernel<false>, grid, dim3(AT_WARPS * 32), AT_SMEM, s, a);
     count_launch();
-    return cudaGetLastError();
+    return e;
 }
 
 cudaError_t launch_rope(void* x, int n_heads, int D, int64_t pos, float theta, aq_dtype_t dt, cudaStream_t s) {
